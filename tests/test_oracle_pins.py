@@ -1,0 +1,429 @@
+"""Pins of the CPU oracle against things other than itself: brute force on tiny
+inputs, closed forms, invariants, hand-worked cases, and the figures the paper
+prints.  CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+def read_golden(name):
+    d = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split()
+            d[k] = float(v)
+    return d
+
+
+def densify(w):
+    A = np.zeros((w.M, w.K), dtype=np.float64)
+    v = w.vals if w.dtype == W.SD_F32 else W.bf16_bits_to_f32(w.vals)
+    for i in range(w.M):
+        for p in range(w.rowptr[i], w.rowptr[i + 1]):
+            A[i, w.colind[p]] += float(v[p])
+    return A
+
+
+def dense_f64(w, X):
+    return (X if w.dtype == W.SD_F32 else W.bf16_bits_to_f32(X)).astype(np.float64)
+
+
+def brute_gemm(A, B):
+    """Dense triple loop in Python floats (IEEE double)."""
+    M, K = A.shape
+    N = B.shape[1]
+    out = [[0.0] * N for _ in range(M)]
+    for i in range(M):
+        for j in range(N):
+            s = 0.0
+            for k in range(K):
+                if A[i, k] != 0.0:
+                    s += float(A[i, k]) * float(B[k, j])
+            out[i][j] = s
+    return np.array(out, dtype=np.float64).reshape(M, N)
+
+
+# ------------------------------------------------------------------ O1
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+@pytest.mark.parametrize("N", [1, 3, 4, 32])
+def test_o1_brute_force_tiny(dtype, N):
+    rng = np.random.default_rng(7 + N)
+    M, K = 37, 29
+    lengths = rng.integers(0, 9, size=M)
+    lengths[5] = 0
+    lengths[11] = K
+    for alpha in (0.0, 1.0, -0.5):
+        for beta in (0.0, 1.0, -0.5):
+            w = W.random_csr(M, K, N, lengths, seed=100 + N, dtype=dtype, alpha=alpha, beta=beta)
+            # ld > N: pad B and C with sentinel columns
+            Bp = np.full((K, N + 3), 7, dtype=w.B.dtype)
+            Bp[:, :N] = w.B
+            Cin = None
+            if beta != 0.0:
+                Cin = np.full((M, N + 2), np.float32(99.0))
+                Cin[:, :N] = w.C0
+            Cref, S = oracle.spmm(w.rowptr, w.colind, w.vals, Bp[:, :N], N,
+                                  Cin[:, :N] if Cin is not None else None, alpha, beta)
+            A = densify(w)
+            Bd = dense_f64(w, w.B)
+            want = np.float64(np.float32(alpha)) * brute_gemm(A, Bd)
+            if beta != 0.0:
+                want = want + np.float64(np.float32(beta)) * w.C0.astype(np.float64)
+            np.testing.assert_allclose(Cref, want, rtol=1e-14, atol=1e-300)
+            np.testing.assert_allclose(S, brute_gemm(np.abs(A), np.abs(Bd)), rtol=1e-14, atol=1e-300)
+
+
+def test_o1_hand_worked_3x3():
+    # A = [[2,0,1],[0,0,0],[0,-3,4]],  B = [[1,2],[3,4],[5,6]]
+    rowptr = np.array([0, 2, 2, 4], np.int32)
+    colind = np.array([0, 2, 1, 2], np.int32)
+    vals = np.array([2, 1, -3, 4], np.float32)
+    B = np.array([[1, 2], [3, 4], [5, 6]], np.float32)
+    Cin = np.array([[10, 20], [30, 40], [50, 60]], np.float32)
+    # A*B = [[2*1+1*5, 2*2+1*6], [0,0], [-9+20, -12+24]] = [[7,10],[0,0],[11,12]]
+    Cref, S = oracle.spmm(rowptr, colind, vals, B, 2)
+    assert Cref.tolist() == [[7.0, 10.0], [0.0, 0.0], [11.0, 12.0]]
+    assert S.tolist() == [[7.0, 10.0], [0.0, 0.0], [29.0, 36.0]]
+    # alpha = 2, beta = -1:  2*AB - Cin
+    Cref, _ = oracle.spmm(rowptr, colind, vals, B, 2, Cin, 2.0, -1.0)
+    assert Cref.tolist() == [[4.0, 0.0], [-30.0, -40.0], [-28.0, -36.0]]
+    # N = 1 is SpMV with x = first column
+    Cref, _ = oracle.spmm(rowptr, colind, vals, np.ascontiguousarray(B[:, :1]), 1)
+    assert Cref.ravel().tolist() == [7.0, 0.0, 11.0]
+
+
+def test_o1_hand_worked_4x5():
+    # A (4x5): row0: (0,1)=1 (0,4)=2 ; row1: (1,0)=-1 ; row2: empty ; row3: (3,1)=0.5 (3,2)=0.25 (3,3)=-2
+    rowptr = np.array([0, 2, 3, 3, 6], np.int32)
+    colind = np.array([1, 4, 0, 1, 2, 3], np.int32)
+    vals = np.array([1, 2, -1, 0.5, 0.25, -2], np.float32)
+    B = np.array([[1, 0, 2], [0, 1, 4], [8, 8, 8], [1, 2, 3], [10, 20, 30]], np.float32)
+    # row0 = B[1] + 2 B[4] = [20, 41, 64]; row1 = -B[0] = [-1, 0, -2]; row2 = 0
+    # row3 = .5 B[1] + .25 B[2] - 2 B[3] = [0+2-2, .5+2-4, 2+2-6] = [0, -1.5, -2]
+    Cref, S = oracle.spmm(rowptr, colind, vals, B, 3)
+    assert Cref.tolist() == [[20.0, 41.0, 64.0], [-1.0, 0.0, -2.0], [0.0, 0.0, 0.0], [0.0, -1.5, -2.0]]
+    assert S[3].tolist() == [4.0, 6.5, 10.0]
+    # beta == 0 must not read C: poison it
+    poison = np.full((4, 3), np.nan, np.float32)
+    Cref2, _ = oracle.spmm(rowptr, colind, vals, B, 3, poison, 1.0, 0.0)
+    assert np.array_equal(Cref, Cref2)
+
+
+def test_o1_identity_and_permutation():
+    rng = np.random.default_rng(3)
+    n, N = 50, 5
+    B = rng.standard_normal((n, N)).astype(np.float32)
+    Cin = rng.standard_normal((n, N)).astype(np.float32)
+    rowptr = np.arange(n + 1, dtype=np.int32)
+    ones = np.ones(n, np.float32)
+    ident = np.arange(n, dtype=np.int32)
+    Cref, _ = oracle.spmm(rowptr, ident, ones, B, N, Cin, 0.75, -2.0)
+    want = np.float64(0.75) * B.astype(np.float64) + np.float64(-2.0) * Cin.astype(np.float64)
+    assert np.array_equal(Cref, want)
+    perm = rng.permutation(n).astype(np.int32)
+    Cref, _ = oracle.spmm(rowptr, perm, ones, B, N)
+    assert np.array_equal(Cref, B[perm].astype(np.float64))
+
+
+def test_o1_row_sums_col_sums_linearity():
+    w = W.g1_tiny_uniform(M=300, K=257, N=8, seed=11)
+    v64 = w.vals.astype(np.float64)
+    # B = ones  =>  every column of C is the row sum of A
+    ones = np.ones((w.K, 4), np.float32)
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, ones, 4)
+    rows = np.repeat(np.arange(w.M), np.diff(w.rowptr))
+    rs = np.zeros(w.M)
+    np.add.at(rs, rows, v64)
+    np.testing.assert_allclose(Cref, np.repeat(rs[:, None], 4, 1), rtol=1e-13, atol=1e-13)
+    # 1^T (A B) = (1^T A) B
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
+    cs = np.zeros(w.K)
+    np.add.at(cs, w.colind, v64)
+    np.testing.assert_allclose(Cref.sum(0), cs @ w.B.astype(np.float64), rtol=1e-11, atol=1e-11)
+    # width consistency: columns are independent
+    left, _ = oracle.spmm(w.rowptr, w.colind, w.vals, np.ascontiguousarray(w.B[:, :3]), 3)
+    one, _ = oracle.spmm(w.rowptr, w.colind, w.vals, np.ascontiguousarray(w.B[:, :1]), 1)
+    assert np.array_equal(left, Cref[:, :3])
+    assert np.array_equal(one, Cref[:, :1])
+    # strided view of a wider B gives the same answer
+    viewed, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B[:, :5], 5)
+    assert np.array_equal(viewed, Cref[:, :5])
+    # spmm_rows returns the same rows
+    pick = np.array([0, 7, 299, 150], np.int64)
+    sub, _ = oracle.spmm_rows(pick, w.rowptr, w.colind, w.vals, w.B, w.N)
+    assert np.array_equal(sub, Cref[pick])
+
+
+def test_o1_check_flags_errors():
+    w = W.g1_tiny_uniform(M=64, K=64, N=8, seed=5)
+    Cref, S = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
+    good = Cref.astype(np.float32)
+    r = oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, good)
+    assert r["ok"] and r["max_ratio"] < 1.0
+    bad = good.copy()
+    i = int(np.argmax(np.diff(w.rowptr) > 0))
+    bad[i, 3] += np.float32(1e-3) * max(1.0, abs(bad[i, 3]))
+    r = oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, bad)
+    assert not r["ok"] and r["violations"] == 1 and r["worst"] == (i, 3)
+    bad = good.copy()
+    bad[1, 1] = np.nan
+    assert oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, bad)["nonfinite"] == 1
+
+
+# ------------------------------------------------------------------ workload closed forms
+def test_stencil_closed_forms_small_and_eigenmodes():
+    n = 48
+    w = W.g2_stencil(n=n, N=4, beta=0.0)
+    assert w.nnz == 5 * n * n - 4 * n
+    r = np.diff(w.rowptr)
+    assert (r == 3).sum() == 4 and (r == 4).sum() == 4 * (n - 2) and (r == 5).sum() == (n - 2) ** 2
+    # A*1: 0 interior, 1 edge, 2 corner; total 4n
+    ones = np.ones((w.K, 1), np.float32)
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, ones, 1)
+    assert Cref.sum() == 4 * n
+    assert sorted(np.unique(Cref).tolist()) == [0.0, 1.0, 2.0]
+    # discrete sine modes are eigenvectors (textbook): lambda = 4 - 2cos(p pi/(n+1)) - 2cos(q pi/(n+1))
+    idx = np.arange(n * n)
+    x, y = idx % n, idx // n
+    modes = [(1, 1), (2, 5), (7, 3), (n, n)]
+    B = np.stack([np.sin(p * math.pi * (x + 1) / (n + 1)) * np.sin(q * math.pi * (y + 1) / (n + 1))
+                  for p, q in modes], axis=1).astype(np.float32)
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, B, 4)
+    lam = np.array([4 - 2 * math.cos(p * math.pi / (n + 1)) - 2 * math.cos(q * math.pi / (n + 1))
+                    for p, q in modes])
+    np.testing.assert_allclose(Cref, B.astype(np.float64) * lam[None, :], atol=2e-6)
+
+
+def test_stencil_full_size_counts():
+    n = 1024
+    w = W.g2_stencil(n=n, N=1, beta=0.0)
+    assert w.nnz == 5_238_784 == 5 * n * n - 4 * n
+    r = np.diff(w.rowptr)
+    assert (r == 3).sum() == 4 and (r == 4).sum() == 4088 and (r == 5).sum() == 1_044_484
+    info = oracle.summary(w.rowptr, w.colind, w.M, w.K, 64)
+    # occupied 16x16 blocks: diagonal + left/right neighbours + up/down neighbours
+    nb = n // 16
+    assert info.nnzb16 == n * nb + 2 * (nb - 1) * n + 2 * (n - 1) * nb
+    assert info.diag == n * n and info.unsorted_rows == 0 and info.max_r == 5
+    assert info.max_span == 2 * n + 1
+
+
+def test_gcn_normalised_adjacency_invariants():
+    w = W.g3_gcn_rmat(scale=10, edge_factor=8, N=2, seed=99)
+    d = w.meta["degree"].astype(np.float64)
+    assert np.array_equal(np.diff(w.rowptr), w.meta["degree"])
+    sq = np.sqrt(d)
+    B = np.stack([sq, -2 * sq], 1).astype(np.float32)
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, B, 2)
+    # A_hat sqrt(d) = sqrt(d): eigenvalue 1 (up to fp32 rounding of the inputs)
+    np.testing.assert_allclose(Cref, B.astype(np.float64), rtol=2e-6)
+    # symmetry: x^T (A y) = y^T (A x)
+    rng = np.random.default_rng(0)
+    X = rng.standard_normal((w.M, 2)).astype(np.float32)
+    AX, _ = oracle.spmm(w.rowptr, w.colind, w.vals, X, 2)
+    x, y = X[:, 0].astype(np.float64), X[:, 1].astype(np.float64)
+    assert abs(x @ AX[:, 1] - y @ AX[:, 0]) < 1e-9 * (np.abs(x) @ np.abs(AX[:, 1]) + 1)
+
+
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_block_workload_strip_gemm_and_bsr(dtype):
+    w = W.g4_block(Mb=24, Kb=40, N=8, nblocks=60, seed=21, dtype=dtype)
+    bi, bj, bv = w.meta["block_row"], w.meta["block_col"], w.meta["block_vals"]
+    if dtype == W.SD_BF16:
+        bv = W.bf16_bits_to_f32(W.f32_to_bf16_bits(bv).reshape(bv.shape))
+    Bd = dense_f64(w, w.B)
+    Cref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
+    for I in range(24):
+        want = np.zeros((16, w.N))
+        for b in np.flatnonzero(bi == I):
+            want += bv[b].astype(np.float64) @ Bd[16 * bj[b]:16 * bj[b] + 16]
+        np.testing.assert_allclose(Cref[16 * I:16 * I + 16], want, rtol=1e-12, atol=1e-12)
+    browptr, bcol, bval = oracle.bsr16(w.rowptr, w.colind, w.vals, w.M, w.K)
+    assert browptr[-1] == 60
+    assert np.array_equal(np.diff(browptr), np.bincount(bi, minlength=24))
+    assert np.array_equal(bcol, bj.astype(np.int32))
+    gen_vals = w.meta["block_vals"]
+    gen_vals = W.f32_to_bf16_bits(gen_vals).reshape(gen_vals.shape) if dtype == W.SD_BF16 else gen_vals
+    assert np.array_equal(bval, gen_vals)
+    info = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+    assert info.nnzb16 == 60 and oracle.rho_bsr16(info) == 1.0
+    assert info.blk_hist[8] == 60 and info.nnz_dense_blocks == w.nnz
+    assert oracle.decide(info) == oracle.BSR_TC
+
+
+# ------------------------------------------------------------------ O2
+def test_o2_against_python_sets_and_round_trip():
+    rng = np.random.default_rng(17)
+    M, K = 70, 45       # neither a multiple of 16
+    lengths = rng.integers(0, 12, size=M)
+    w = W.random_csr(M, K, 1, lengths, seed=33)
+    browptr, bcol, bval = oracle.bsr16(w.rowptr, w.colind, w.vals, M, K)
+    blocks = {}
+    for i in range(M):
+        for p in range(w.rowptr[i], w.rowptr[i + 1]):
+            blocks.setdefault((i >> 4, w.colind[p] >> 4), {})[(i & 15, w.colind[p] & 15)] = w.vals[p]
+    keys = sorted(blocks)
+    assert len(keys) == browptr[-1]
+    k = 0
+    for I in range((M + 15) // 16):
+        mine = [key for key in keys if key[0] == I]
+        assert browptr[I + 1] - browptr[I] == len(mine)
+        for (_, J) in mine:
+            assert bcol[k] == J
+            dense = np.zeros((16, 16), np.float32)
+            for (r, c), v in blocks[(I, J)].items():
+                dense[r, c] = v
+            assert np.array_equal(bval[k], dense)
+            k += 1
+    # round trip BSR -> CSR through the structure mask returns the input
+    back = []
+    for I in range((M + 15) // 16):
+        for r in range(16):
+            i = 16 * I + r
+            if i >= M:
+                break
+            for b in range(browptr[I], browptr[I + 1]):
+                for c in range(16):
+                    if (r, c) in blocks[(I, int(bcol[b]))]:
+                        back.append((i, 16 * int(bcol[b]) + c, bval[b, r, c]))
+    got_rows = np.repeat(np.arange(M), np.diff(w.rowptr))
+    assert [(int(a), int(b), float(c)) for a, b, c in back] == \
+        [(int(a), int(b), float(c)) for a, b, c in zip(got_rows, w.colind, w.vals)]
+
+
+def test_o2_stored_zero_counts_as_structure():
+    rowptr = np.array([0, 1, 2], np.int32)
+    colind = np.array([3, 40], np.int32)
+    vals = np.array([0.0, 5.0], np.float32)
+    browptr, bcol, bval = oracle.bsr16(rowptr, colind, vals, 2, 48)
+    assert browptr.tolist() == [0, 2] and bcol.tolist() == [0, 2]
+    assert bval[1, 1, 8] == 5.0 and not bval[0].any()
+
+
+# ------------------------------------------------------------------ O3
+def test_o3_against_brute_force():
+    rng = np.random.default_rng(5)
+    M, K = 90, 300
+    lengths = rng.integers(0, 40, size=M)
+    lengths[3] = 280
+    lengths[4] = 0
+    w = W.random_csr(M, K, 1, lengths, seed=44)
+    info = oracle.summary(w.rowptr, w.colind, M, K, 7)
+    assert (info.M, info.K, info.N, info.nnz) == (M, K, 7, w.nnz)
+    hist = [0] * 32
+    for r in lengths:
+        hist[0 if r == 0 else int(math.floor(math.log2(r))) + 1] += 1
+    assert list(info.row_hist) == hist
+    assert info.sum_r2 == int((lengths.astype(np.int64) ** 2).sum())
+    assert info.max_r == 280 and info.empty_rows == int((lengths == 0).sum())
+    assert info.long_rows == 1 and info.nnz_long_rows == 280
+    span = gap = diag = 0
+    mspan = 0
+    blocks = {}
+    for i in range(M):
+        cols = w.colind[w.rowptr[i]:w.rowptr[i + 1]]
+        if cols.size:
+            s = int(cols.max() - cols.min() + 1)
+            span += s
+            mspan = max(mspan, s)
+            gap += int(np.diff(cols).sum())      # sum of gaps between sorted consecutive indices
+            diag += int((cols == i).sum())
+        for c in cols:
+            blocks[(i >> 4, c >> 4)] = blocks.get((i >> 4, c >> 4), 0) + 1
+    assert (info.sum_span, info.max_span, info.sum_gap, info.diag) == (span, mspan, gap, diag)
+    assert info.unsorted_rows == 0
+    assert info.nnzb16 == len(blocks)
+    bh = [0] * 9
+    for c in blocks.values():
+        bh[min(int(math.floor(math.log2(c))), 8)] += 1
+    assert list(info.blk_hist) == bh
+    assert info.nnz_dense_blocks == sum(c for c in blocks.values() if c >= 128)
+
+
+def test_o3_unsorted_and_duplicate_rows_are_counted():
+    rowptr = np.array([0, 3, 5, 7], np.int32)
+    colind = np.array([0, 2, 1, 4, 4, 1, 9], np.int32)   # row0 unsorted, row1 duplicate, row2 fine
+    info = oracle.summary(rowptr, colind, 3, 10, 1)
+    assert info.unsorted_rows == 2
+    assert oracle.decide(info) != oracle.BSR_TC
+
+
+def test_paper_worked_example_sec3_3():
+    g = read_golden("sec3_3_shen_e40r0100.txt")
+    info = oracle.Info()
+    info.M = info.K = int(g["m"])
+    info.nnz = int(g["nnz"])
+    info.max_r = int(g["max_row_length"])
+    info.nnzb16 = int(g["nnzb16"])
+    assert round(oracle.rho_ell(info), 1) == g["rho_ell_approx"]
+    assert round(oracle.rho_bsr16(info), 1) == g["rho_bsr16_approx"]
+    assert round(info.nnz / info.nnzb16, 1) == g["nnz_per_occupied_tile_approx"]
+    assert round(100 * oracle.tile_coverage16(info), 1) == g["occupied_tile_fraction_percent_approx"]
+    assert oracle.csr_bytes(info, 4) == int(g["csr_bytes_fp32_int32"])
+
+
+def test_paper_planning_record_nemeth26():
+    g = read_golden("appE_nemeth26_working_set.txt")
+    info = oracle.Info()
+    info.M = info.K = int(g["rows"])
+    info.N = int(g["dense_width"])
+    info.nnz = int(g["rows"] * g["mean_row_length"])
+    _, m_t = oracle.working_set_bytes(oracle.csr_bytes(info, 4), info, 4)
+    assert abs(m_t / 2**20 - g["csr_working_set_mib"]) < 0.01
+
+
+# ------------------------------------------------------------------ O4
+def test_o4_merge_coords_match_closed_form():
+    rng = np.random.default_rng(2)
+    for trial in range(6):
+        S = int(rng.integers(1, 200))
+        lengths = rng.integers(0, 6, size=S)
+        if trial % 2:
+            lengths[rng.integers(0, S)] = 500
+        ptr = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+        for items in (1, 7, 64):
+            got = oracle.merge_coords(ptr, items)
+            total = S + int(ptr[-1])
+            ntiles = (total + items - 1) // items
+            assert got.size == ntiles + 1
+            # end of segment r is item number ptr[r+1] + r of the merged list
+            pos = ptr[1:].astype(np.int64) + np.arange(S)
+            want = [int(np.searchsorted(pos, min(t * items, total), side="left")) for t in range(ntiles + 1)]
+            assert got.tolist() == want
+            assert got[0] == 0 and got[-1] == S
+
+
+def test_o4_family_rule_on_the_five_shapes():
+    w = W.g1_tiny_uniform()
+    assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.ROWSPLIT
+    w = W.g2_stencil(n=64, N=4)
+    assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.ROWSPLIT
+    w = W.g3_gcn_rmat(scale=12, N=4)
+    assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.MERGE
+    w = W.g4_block(Mb=32, Kb=32, N=4, nblocks=40)
+    assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.BSR_TC
+    w = W.g5_skewed(M=1 << 14, N=4, scale_c=2.4e7 / 256, cap=800)
+    assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.MERGE
+
+
+def test_skewed_generator_counts():
+    # lengths are a deterministic rank-size law; only their assignment to rows is random
+    M = 1 << 12
+    w = W.g5_skewed(M=M, N=1, scale_c=5000.0, cap=300)
+    r = np.sort(np.diff(w.rowptr))[::-1]
+    rank = np.arange(1, M + 1, dtype=np.float64)
+    want = np.clip(np.floor(5000.0 * rank ** -1.2), 1, 300).astype(np.int64)
+    assert np.array_equal(r, want)
+    for i in range(0, M, 97):
+        cols = w.colind[w.rowptr[i]:w.rowptr[i + 1]]
+        assert np.all(np.diff(cols) > 0) and cols.min() >= 0 and cols.max() < M
