@@ -1,0 +1,174 @@
+/*
+ * sd.h -- C ABI of the structure-adaptive SpMM library for NVIDIA B200 (sm_100a).
+ *
+ *     C = alpha * A * B + beta * C
+ *
+ * A is an M x K sparse matrix in CSR (32-bit indices; fp32 values, or bf16 values
+ * that are multiplied exactly and accumulated in fp32), B is a row-major dense
+ * K x N matrix in the same dtype as A's values, C is a row-major dense M x N fp32
+ * matrix.  This is the SpMM of the paper's Sec. 2.1 ("SpMM computes C = AB with a
+ * dense matrix B of width K"; the paper's dense width K is called N here, and K is
+ * the column count of A).  N = 1 is SpMV.  alpha and beta follow the BLAS
+ * convention; the paper's operator is alpha = 1, beta = 0.
+ *
+ * The three calls mirror the preprocess / compute / cleanup harness of the
+ * paper's generated implementations (Appendix "A Generated SpMM Implementation"):
+ * sd_plan_create analyses the sparsity pattern once (Sec. 3.1: row-length
+ * statistics, column spread, occupied 16x16 tiles), chooses a representation and a
+ * schedule -- the compilation plan <R, S, theta_H> of Sec. 3, Eq. 2, with fixed
+ * integer rules in place of the paper's learned ranking and search -- and builds
+ * it; sd_spmm executes it any number of times with different dense operands;
+ * sd_plan_destroy releases it.
+ *
+ * Conventions for every call
+ *  - Pointers named rowptr, colind, vals, B, C are DEVICE pointers on the current
+ *    CUDA device unless the parameter says "host".  Sizes are element counts.
+ *  - Errors are return codes.  Nothing throws, aborts or traps.  The last error
+ *    message of the calling thread is kept for sd_last_error().
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef SD_H_
+#define SD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd_plan sd_plan_t; /* opaque, library-owned */
+
+typedef enum {
+    SD_OK = 0,
+    SD_ERR_INVALID_ARG = 1, /* null pointer, negative size, ld < N, bad enum, invalid CSR */
+    SD_ERR_UNSUPPORTED = 2, /* valid request this build cannot serve */
+    SD_ERR_ALLOC = 3,       /* device or host allocation failed */
+    SD_ERR_CUDA = 4,        /* a CUDA call failed; text in sd_last_error */
+    SD_ERR_INTERNAL = 5
+} sd_status_t;
+
+typedef enum { SD_F32 = 0, SD_BF16 = 1 } sd_dtype_t; /* dtype of vals AND of B */
+
+/* Kernel families (paper Sec. 3.2 lists the SpMM template set CSR, COO, BSR-4/8/16,
+ * Blocked-ELL, DTC; this library keeps a row-wise CSR family, an nnz-balanced
+ * family in the spirit of COO / merge-based decompositions, and BSR-16). */
+typedef enum {
+    SD_AUTO = 0,     /* decide from the structure summary */
+    SD_ROWSPLIT = 1, /* sub-warp per row, vectorised gathers of B rows */
+    SD_MERGE = 2,    /* merge-path split of (row ends + nonzeros), segmented reduction,
+                        deterministic carry-out fix-up */
+    SD_BSR_TC = 3    /* 16x16 blocks on the tensor cores (tcgen05 / TMEM / TMA) */
+} sd_family_t;
+
+/* Options of sd_plan_create_ex.  Zero-initialise, then set fields. */
+typedef struct {
+    const int32_t *rowptr; /* device, [M+1], non-decreasing, rowptr[0] == 0 */
+    const int32_t *colind; /* device, [nnz], 0 <= col < K */
+    const void *vals;      /* device, [nnz], float or bf16 per `dtype` */
+    int64_t M, K, N;       /* N: dense width the plan is tuned for (other widths still run) */
+    int32_t dtype;         /* sd_dtype_t */
+    int32_t family;        /* sd_family_t; SD_AUTO applies the rule */
+    int32_t windows;       /* column windows of the MERGE family: 0 = automatic, 1 = off, 2..64 */
+    int32_t validate;      /* != 0: check rowptr monotone and 0 <= col < K on the device first */
+    void *stream;          /* stream for the analysis kernels (plan creation still synchronises) */
+} sd_plan_desc_t;
+
+/* Integer structure summary (Sec. 3.1 "Intrinsic pattern features", Eq. 4) and the
+ * decision taken from it.  All counts are exact integers. */
+typedef struct {
+    int64_t M, K, N, nnz;
+    int64_t row_hist[32];   /* bin 0: r == 0; bin b >= 1: 2^(b-1) <= r < 2^b   (r = row length) */
+    uint64_t sum_r2;        /* sum of r_i^2 */
+    int64_t max_r;
+    int64_t empty_rows;
+    uint64_t sum_span;      /* sum over non-empty rows of (max col - min col + 1) */
+    int64_t max_span;
+    uint64_t sum_gap;       /* sum over non-empty rows of (max col - min col) */
+    int64_t diag;           /* stored entries with col == row */
+    int64_t unsorted_rows;  /* rows with an adjacent pair col[p+1] <= col[p] */
+    int64_t long_rows;      /* rows with r >= 256 */
+    int64_t nnz_long_rows;  /* nonzeros in those rows */
+    int64_t nnzb16;         /* occupied 16x16 blocks (Eq. 4, nnzb_16) */
+    int64_t blk_hist[9];    /* per-block entry count: [1],[2,3],[4,7],...,[128,255],[256+] */
+    int64_t nnz_dense_blocks; /* nonzeros in blocks holding >= 128 entries */
+    /* decision and schedule parameters (theta_H of Eq. 2) */
+    int32_t family;         /* sd_family_t actually built */
+    int32_t dtype;
+    int32_t windows;        /* column windows in use (1 = none) */
+    int32_t tile_items;     /* merge items (row ends + nonzeros) per CTA tile, MERGE only */
+    int64_t num_tiles;      /* MERGE: total tiles over all windows */
+    int64_t num_segments;   /* MERGE: rows, or (row, window) pairs when windows > 1 */
+    int64_t plan_bytes;     /* device memory owned by the plan */
+    int32_t sm_count;       /* hardware context read at plan time (Sec. 3.1) */
+    int32_t reserved;
+    int64_t l2_bytes;
+} sd_plan_info_t;
+
+/* sd_plan_create -- Sec. 3 (task <X, o, H> in, specialised implementation out) and
+ * the `preprocess` entry of the paper's harness.  fp32 values, automatic family.
+ *   rowptr, colind, vals  device pointers, BORROWED: they must stay allocated and
+ *                         unchanged until sd_plan_destroy.
+ *   M, K                  shape of A;  N  dense width to tune for.
+ * Synchronous; allocates device memory owned by the plan.  Returns NULL on failure
+ * (reason through sd_last_error). */
+sd_plan_t *sd_plan_create(const int32_t *rowptr, const int32_t *colind, const float *vals,
+                          int64_t M, int64_t K, int64_t N);
+
+/* sd_plan_create_ex -- same, with dtype, forced family, window count, validation.
+ * *out receives the plan.  SD_ERR_INVALID_ARG for null desc/out, negative sizes,
+ * null CSR pointers with M > 0, unknown enums, or (validate != 0) a malformed CSR. */
+sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
+
+/* sd_spmm -- the `compute` entry: C = alpha*A*B + beta*C on `stream`.
+ *   B    device, row-major [K, ldb], dtype of the plan, read-only, must not alias C
+ *   C    device, row-major [M, ldc] fp32, in/out; columns N..ldc-1 are never touched
+ *   ldb, ldc >= N (elements).  N is the width given at plan creation.
+ * beta == 0: C is not read (NaN/Inf in it do not propagate).  alpha == 0: C = beta*C
+ * without reading A or B.  M == 0 or N == 0: SD_OK, nothing launched.  Empty rows
+ * get beta*C.  Asynchronous: launches only, no allocation, no synchronisation.
+ * 16-byte aligned B/C with N, ldb, ldc multiples of the vector width take the
+ * vectorised kernels; anything else takes scalar kernels (never an error).
+ * A plan must not run concurrently on two streams (it owns carry-out scratch).
+ * Results are run-to-run bit-identical (no floating-point atomics). */
+sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc,
+                    float alpha, float beta, void *stream);
+
+/* sd_spmm_host -- same operation with HOST buffers: B (and C when beta != 0) are
+ * copied to plan-owned device staging buffers, sd_spmm runs, C is copied back, and
+ * the call returns after the copy completed.  The staging buffers are allocated by
+ * the first such call on a plan.  Pinned host memory gives full PCIe speed. */
+sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host,
+                         int64_t ldc, float alpha, float beta);
+
+/* sd_plan_destroy -- the `cleanup` entry.  Frees everything the plan owns.  NULL is a no-op. */
+void sd_plan_destroy(sd_plan_t *plan);
+
+/* sd_plan_get_info -- structure summary and decision (host struct out). */
+sd_status_t sd_plan_get_info(const sd_plan_t *plan, sd_plan_info_t *out);
+
+/* sd_plan_get_bsr -- copy the BSR-16 representation (Sec. 3.1, Eq. 4) to HOST arrays:
+ * browptr int32 [ceil(M/16)+1], bcol int32 [nnzb16] ascending inside a block-row,
+ * bval [nnzb16][16][16] row-major in the plan dtype, absent slots +0.  Any pointer may
+ * be NULL to skip it.  SD_ERR_UNSUPPORTED if the plan's family is not SD_BSR_TC. */
+sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bcol, void *bval);
+
+/* sd_plan_get_tiles -- MERGE family: copy merge-path tile start coordinates to a HOST
+ * array.  tile_seg[t] = number of segment ends among the first t*tile_items merged
+ * items of window w, for t = 0..ntiles_w, windows concatenated; `cap` is the capacity
+ * of tile_seg in elements and *count receives the number written (or needed).
+ * seg_ptr (optional, capacity num_segments + windows) receives each window's segment
+ * pointer array.  SD_ERR_UNSUPPORTED for other families. */
+sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t cap, int64_t *count);
+
+/* sd_last_error -- copy the calling thread's last error text into buf (NUL-terminated,
+ * at most n bytes); returns the last status code. */
+int sd_last_error(char *buf, size_t n);
+
+/* sd_version -- "major.minor" text of this build. */
+const char *sd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SD_H_ */

@@ -1,0 +1,761 @@
+// C ABI of the SpMM library: plan creation (structure scan, decision, representation
+// build), execution dispatch, teardown.  See include/sd.h for the contract.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include <cub/cub.cuh>
+
+#include "sd_common.cuh"
+#include "sd_launch.cuh"
+
+// =====================================================================================
+// error state
+// =====================================================================================
+namespace sd {
+
+static thread_local char g_err_text[512] = "";
+static thread_local int g_err_code = SD_OK;
+
+void set_error(sd_status_t code, const char *fmt, ...) {
+    g_err_code = code;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err_text, sizeof g_err_text, fmt, ap);
+    va_end(ap);
+}
+
+sd_status_t cuda_fail(cudaError_t e, const char *what) {
+    set_error(SD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return SD_ERR_CUDA;
+}
+
+// =====================================================================================
+// structure scan kernels (Sec. 3.1, intrinsic pattern features; integers only)
+// =====================================================================================
+struct ScanAccum {
+    unsigned long long row_hist[32];
+    unsigned long long sum_r2, empty_rows, sum_span, sum_gap, diag, unsorted_rows, long_rows, nnz_long_rows;
+    unsigned long long max_r, max_span;
+    unsigned long long blk_hist[9];
+    unsigned long long nnz_dense_blocks;
+    unsigned long long bad_csr;   // validation: number of offending rows / entries
+};
+
+__device__ __forceinline__ int hist_bin(long long v) { return v <= 0 ? 0 : 64 - __clzll(v); }
+
+// One warp per row.  Optionally writes the 16x16 block key of every nonzero.
+__global__ void __launch_bounds__(256)
+scan_rows_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, int64_t M,
+                 int64_t Kb, unsigned long long *__restrict__ keys, ScanAccum *__restrict__ out) {
+    constexpr unsigned FULL = 0xffffffffu;
+    __shared__ unsigned long long s_hist[32];
+    __shared__ unsigned long long s_sum[8];
+    __shared__ unsigned long long s_max[2];
+    if (threadIdx.x < 32) s_hist[threadIdx.x] = 0;
+    if (threadIdx.x < 8) s_sum[threadIdx.x] = 0;
+    if (threadIdx.x < 2) s_max[threadIdx.x] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    unsigned long long l_r2 = 0, l_empty = 0, l_span = 0, l_gap = 0, l_diag = 0, l_uns = 0, l_long = 0,
+                       l_nnzlong = 0, l_maxr = 0, l_maxspan = 0;
+    for (int64_t row = warp0; row < M; row += nwarps) {
+        const int p0 = rowptr[row], p1 = rowptr[row + 1];
+        const long long r = static_cast<long long>(p1) - p0;
+        int mn = INT_MAX, mx = INT_MIN, dg = 0, uns = 0;
+        for (int p = p0 + lane; p < p1; p += 32) {
+            const int c = colind[p];
+            mn = min(mn, c);
+            mx = max(mx, c);
+            dg += (c == row);
+            if (p + 1 < p1) uns |= (colind[p + 1] <= c);
+            if (keys) keys[p] = static_cast<unsigned long long>(row >> 4) * Kb + static_cast<unsigned>(c >> 4);
+        }
+        mn = __reduce_min_sync(FULL, mn);
+        mx = __reduce_max_sync(FULL, mx);
+        dg = __reduce_add_sync(FULL, dg);
+        uns = __reduce_or_sync(FULL, uns);
+        if (lane == 0) {
+            atomicAdd(&s_hist[hist_bin(r)], 1ULL);
+            l_r2 += static_cast<unsigned long long>(r) * static_cast<unsigned long long>(r);
+            l_maxr = max(l_maxr, static_cast<unsigned long long>(r));
+            if (r == 0) {
+                l_empty += 1;
+            } else {
+                const unsigned long long span = static_cast<unsigned long long>(static_cast<long long>(mx) - mn + 1);
+                l_span += span;
+                l_gap += span - 1;
+                l_maxspan = max(l_maxspan, span);
+                l_diag += dg;
+                l_uns += uns ? 1 : 0;
+                if (r >= 256) {
+                    l_long += 1;
+                    l_nnzlong += r;
+                }
+            }
+        }
+    }
+    if (lane == 0) {
+        atomicAdd(&s_sum[0], l_r2);
+        atomicAdd(&s_sum[1], l_empty);
+        atomicAdd(&s_sum[2], l_span);
+        atomicAdd(&s_sum[3], l_gap);
+        atomicAdd(&s_sum[4], l_diag);
+        atomicAdd(&s_sum[5], l_uns);
+        atomicAdd(&s_sum[6], l_long);
+        atomicAdd(&s_sum[7], l_nnzlong);
+        atomicMax(&s_max[0], l_maxr);
+        atomicMax(&s_max[1], l_maxspan);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32 && s_hist[threadIdx.x]) atomicAdd(&out->row_hist[threadIdx.x], s_hist[threadIdx.x]);
+    if (threadIdx.x == 0) {
+        atomicAdd(&out->sum_r2, s_sum[0]);
+        atomicAdd(&out->empty_rows, s_sum[1]);
+        atomicAdd(&out->sum_span, s_sum[2]);
+        atomicAdd(&out->sum_gap, s_sum[3]);
+        atomicAdd(&out->diag, s_sum[4]);
+        atomicAdd(&out->unsorted_rows, s_sum[5]);
+        atomicAdd(&out->long_rows, s_sum[6]);
+        atomicAdd(&out->nnz_long_rows, s_sum[7]);
+        atomicMax(&out->max_r, s_max[0]);
+        atomicMax(&out->max_span, s_max[1]);
+    }
+}
+
+// Histogram of the entry count of each occupied block.
+__global__ void block_fill_kernel(const int32_t *__restrict__ counts, int64_t nnzb, ScanAccum *__restrict__ out) {
+    __shared__ unsigned long long s_h[9];
+    __shared__ unsigned long long s_dense;
+    if (threadIdx.x < 9) s_h[threadIdx.x] = 0;
+    if (threadIdx.x == 0) s_dense = 0;
+    __syncthreads();
+    for (int64_t b = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; b < nnzb;
+         b += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int c = counts[b];
+        atomicAdd(&s_h[min(hist_bin(c) - 1, 8)], 1ULL);
+        if (c >= 128) atomicAdd(&s_dense, static_cast<unsigned long long>(c));
+    }
+    __syncthreads();
+    if (threadIdx.x < 9 && s_h[threadIdx.x]) atomicAdd(&out->blk_hist[threadIdx.x], s_h[threadIdx.x]);
+    if (threadIdx.x == 0 && s_dense) atomicAdd(&out->nnz_dense_blocks, s_dense);
+}
+
+// CSR validation: rowptr[0] == 0, rowptr non-decreasing, 0 <= col < K.
+__global__ void validate_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, int64_t M,
+                                int64_t K, int64_t nnz, ScanAccum *__restrict__ out) {
+    unsigned long long bad = 0;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    const int64_t i0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    for (int64_t i = i0; i < M; i += stride) bad += (rowptr[i + 1] < rowptr[i]);
+    for (int64_t p = i0; p < nnz; p += stride) bad += (colind[p] < 0 || colind[p] >= K);
+    if (i0 == 0) bad += (rowptr[0] != 0);
+    if (bad) atomicAdd(&out->bad_csr, bad);
+}
+
+// =====================================================================================
+// representation builders
+// =====================================================================================
+// BSR-16 block-row pointers from the sorted distinct block keys.
+__global__ void bsr_browptr_kernel(const unsigned long long *__restrict__ ukeys, int64_t nnzb, int64_t Kb,
+                                   int32_t Mb, int32_t *__restrict__ browptr) {
+    const int64_t I = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (I > Mb) return;
+    const unsigned long long want = static_cast<unsigned long long>(I) * Kb;
+    int64_t lo = 0, hi = nnzb;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (ukeys[mid] < want) lo = mid + 1;
+        else hi = mid;
+    }
+    browptr[I] = static_cast<int32_t>(lo);
+}
+
+__global__ void bsr_bcol_kernel(const unsigned long long *__restrict__ ukeys, int64_t nnzb, int64_t Kb,
+                                int32_t *__restrict__ bcol) {
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (b < nnzb) bcol[b] = static_cast<int32_t>(ukeys[b] % Kb);
+}
+
+// Scatter the values into row-major 16x16 blocks (copies only: bit-exact).  Warp per row.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bsr_fill_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, const T *__restrict__ vals,
+                int64_t M, const int32_t *__restrict__ browptr, const int32_t *__restrict__ bcol, T *__restrict__ bval) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t row = warp0; row < M; row += nwarps) {
+        const int b0 = browptr[row >> 4], b1 = browptr[(row >> 4) + 1];
+        for (int p = rowptr[row] + lane; p < rowptr[row + 1]; p += 32) {
+            const int c = colind[p];
+            const int J = c >> 4;
+            int lo = b0, hi = b1;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (bcol[mid] < J) lo = mid + 1;
+                else hi = mid;
+            }
+            bval[static_cast<int64_t>(lo) * 256 + (row & 15) * 16 + (c & 15)] = vals[p];
+        }
+    }
+}
+
+// Merge-path tile table: tile_seg[t] = seg_begin + #{ r : (ptr[r+1]-nzb) + (r-seg_begin) < t*tile }.
+__global__ void merge_table_kernel(const int32_t *__restrict__ ptr, int64_t seg_begin, int64_t seg_end, int32_t tile,
+                                   int32_t ntiles, int32_t *__restrict__ tile_seg) {
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t > ntiles) return;
+    const int64_t S = seg_end - seg_begin;
+    const int64_t nzb = ptr[seg_begin];
+    const int64_t total = S + (ptr[seg_end] - nzb);
+    const int64_t d = min(t * tile, total);
+    int64_t lo = 0, hi = S;   // number of segment ends placed before position d
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((ptr[seg_begin + mid + 1] - nzb) + mid < d) lo = mid + 1;
+        else hi = mid;
+    }
+    tile_seg[t] = static_cast<int32_t>(seg_begin + lo);
+}
+
+// A tile needs the fix-up pass iff a segment was open at its start and ends inside it.
+__global__ void merge_fixflag_kernel(const int32_t *__restrict__ ptr, const int32_t *__restrict__ tile_seg,
+                                     int64_t seg_begin, int32_t tile, int32_t ntiles, uint8_t *__restrict__ flag) {
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= ntiles) return;
+    const int64_t s0 = tile_seg[t], s1 = tile_seg[t + 1];
+    const int64_t nzb = ptr[seg_begin];
+    const int64_t nz0 = nzb + t * tile - (s0 - seg_begin);
+    flag[t] = (s1 > s0) && (nz0 > ptr[s0]);
+}
+
+}  // namespace sd
+
+// =====================================================================================
+// the plan object
+// =====================================================================================
+struct sd_plan {
+    const int32_t *rowptr = nullptr;
+    const int32_t *colind = nullptr;
+    const void *vals = nullptr;
+    int64_t M = 0, K = 0, N = 0, nnz = 0;
+    int dtype = SD_F32;
+    int device = 0;
+    sd_plan_info_t info{};
+
+    // MERGE
+    int32_t *tile_seg = nullptr;
+    int32_t *fix_tiles = nullptr;
+    float *tile_head = nullptr;
+    float *tile_tail = nullptr;
+    int32_t ntiles = 0, nfix = 0;
+
+    // BSR
+    int32_t *browptr = nullptr;
+    int32_t *bcol = nullptr;
+    void *bval = nullptr;
+    int64_t nnzb = 0;
+
+    // host-buffer entry point
+    void *stage_B = nullptr;
+    float *stage_C = nullptr;
+    cudaStream_t host_stream = nullptr;
+
+    int64_t owned = 0;
+};
+
+namespace sd {
+
+static sd_status_t dev_alloc(sd_plan *p, void **out, size_t bytes, const char *what) {
+    *out = nullptr;
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(out, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        set_error(SD_ERR_ALLOC, "cudaMalloc(%zu bytes) for %s failed: %s", bytes, what, cudaGetErrorString(e));
+        return SD_ERR_ALLOC;
+    }
+    if (p) p->owned += static_cast<int64_t>(bytes);
+    return SD_OK;
+}
+
+struct TempBuf {   // frees temporary device memory on every exit path
+    void *p = nullptr;
+    ~TempBuf() { if (p) cudaFree(p); }
+    sd_status_t get(size_t bytes, const char *what) { return dev_alloc(nullptr, &p, bytes, what); }
+};
+
+// Family rule on the integer summary.  The paper ranks templates with a learned model and a
+// measured search (Sec. 3.2-3.3) and prints no thresholds; these are fixed integer rules:
+//   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= 1.5 (Eq. 4)
+//   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4
+//   ROWSPLIT  otherwise
+static int decide_family(const sd_plan_info_t &s) {
+    if (s.nnz > 0 && s.unsorted_rows == 0 && 2 * 256 * s.nnzb16 <= 3 * s.nnz) return SD_BSR_TC;
+    const unsigned __int128 lhs = static_cast<unsigned __int128>(static_cast<uint64_t>(s.M)) * s.sum_r2;
+    const unsigned __int128 rhs =
+        static_cast<unsigned __int128>(5) * static_cast<uint64_t>(s.nnz) * static_cast<uint64_t>(s.nnz);
+    const bool skew = (s.max_r >= 256 && 10 * s.nnz_long_rows >= s.nnz) || (s.nnz > 0 && lhs >= rhs);
+    return skew ? SD_MERGE : SD_ROWSPLIT;
+}
+
+static sd_status_t build_merge(sd_plan *p, cudaStream_t st) {
+    const int64_t total = p->M + p->nnz;
+    const int64_t ntiles = (total + kMergeTile - 1) / kMergeTile;
+    if (ntiles > INT32_MAX - 1) {
+        set_error(SD_ERR_UNSUPPORTED, "too many merge tiles");
+        return SD_ERR_UNSUPPORTED;
+    }
+    p->ntiles = static_cast<int32_t>(ntiles);
+    sd_status_t s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_seg), sizeof(int32_t) * (ntiles + 1), "tile table")))
+        return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->fix_tiles), sizeof(int32_t) * (ntiles + 1), "fix-up list")))
+        return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_head), sizeof(float) * ntiles * p->N, "tile heads")))
+        return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_tail), sizeof(float) * ntiles * p->N, "tile tails")))
+        return s;
+    merge_table_kernel<<<ceil_div(ntiles + 1, 256), 256, 0, st>>>(p->rowptr, 0, p->M, kMergeTile, p->ntiles,
+                                                                p->tile_seg);
+    SD_CUDA_TRY(cudaGetLastError());
+    TempBuf flags, nsel, tmp;
+    if ((s = flags.get(ntiles, "fix-up flags"))) return s;
+    if ((s = nsel.get(sizeof(int32_t), "fix-up count"))) return s;
+    merge_fixflag_kernel<<<ceil_div(ntiles, 256), 256, 0, st>>>(p->rowptr, p->tile_seg, 0, kMergeTile, p->ntiles,
+                                                               static_cast<uint8_t *>(flags.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    size_t tb = 0;
+    cub::CountingInputIterator<int32_t> ids(0);
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb, ids, static_cast<uint8_t *>(flags.p), p->fix_tiles,
+                                           static_cast<int32_t *>(nsel.p), static_cast<int>(ntiles), st));
+    if ((s = tmp.get(tb, "select scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags.p), p->fix_tiles,
+                                           static_cast<int32_t *>(nsel.p), static_cast<int>(ntiles), st));
+    SD_CUDA_TRY(cudaMemcpyAsync(&p->nfix, nsel.p, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    p->info.tile_items = kMergeTile;
+    p->info.num_tiles = ntiles;
+    p->info.num_segments = p->M;
+    p->info.windows = 1;
+    return SD_OK;
+}
+
+template <typename T>
+static cudaError_t fill_bsr(sd_plan *p, cudaStream_t st) {
+    bsr_fill_kernel<T><<<148 * 8, 256, 0, st>>>(p->rowptr, p->colind, static_cast<const T *>(p->vals), p->M,
+                                                p->browptr, p->bcol, static_cast<T *>(p->bval));
+    return cudaGetLastError();
+}
+
+static sd_status_t build_bsr(sd_plan *p, const unsigned long long *ukeys, int64_t nnzb, cudaStream_t st) {
+    const int64_t Mb = (p->M + 15) / 16, Kb = (p->K + 15) / 16;
+    const size_t es = p->dtype == SD_F32 ? 4 : 2;
+    p->nnzb = nnzb;
+    sd_status_t s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->browptr), sizeof(int32_t) * (Mb + 1), "browptr"))) return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->bcol), sizeof(int32_t) * nnzb, "bcol"))) return s;
+    if ((s = dev_alloc(p, &p->bval, es * 256 * nnzb, "bval"))) return s;
+    SD_CUDA_TRY(cudaMemsetAsync(p->bval, 0, es * 256 * nnzb, st));
+    bsr_browptr_kernel<<<ceil_div(Mb + 1, 256), 256, 0, st>>>(ukeys, nnzb, Kb, static_cast<int32_t>(Mb), p->browptr);
+    SD_CUDA_TRY(cudaGetLastError());
+    bsr_bcol_kernel<<<ceil_div(nnzb, 256), 256, 0, st>>>(ukeys, nnzb, Kb, p->bcol);
+    SD_CUDA_TRY(cudaGetLastError());
+    SD_CUDA_TRY(p->dtype == SD_F32 ? fill_bsr<float>(p, st) : fill_bsr<__nv_bfloat16>(p, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    return SD_OK;
+}
+
+static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
+    cudaStream_t st = static_cast<cudaStream_t>(d->stream);
+    p->rowptr = d->rowptr;
+    p->colind = d->colind;
+    p->vals = d->vals;
+    p->M = d->M;
+    p->K = d->K;
+    p->N = d->N;
+    p->dtype = d->dtype;
+    SD_CUDA_TRY(cudaGetDevice(&p->device));
+    cudaDeviceProp prop;
+    SD_CUDA_TRY(cudaGetDeviceProperties(&prop, p->device));
+    sd_plan_info_t &info = p->info;
+    memset(&info, 0, sizeof info);
+    info.M = p->M;
+    info.K = p->K;
+    info.N = p->N;
+    info.dtype = p->dtype;
+    info.sm_count = prop.multiProcessorCount;
+    info.l2_bytes = prop.l2CacheSize;
+    info.windows = 1;
+
+    if (p->M > 0) {
+        int32_t last = 0;
+        SD_CUDA_TRY(cudaMemcpyAsync(&last, p->rowptr + p->M, sizeof last, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        if (last < 0) {
+            set_error(SD_ERR_INVALID_ARG, "rowptr[M] = %d is negative", last);
+            return SD_ERR_INVALID_ARG;
+        }
+        p->nnz = last;
+    }
+    info.nnz = p->nnz;
+    if (p->nnz > 0 && (!p->colind || !p->vals)) {
+        set_error(SD_ERR_INVALID_ARG, "colind / vals are null but rowptr[M] = %lld", (long long)p->nnz);
+        return SD_ERR_INVALID_ARG;
+    }
+
+    sd_status_t s;
+    TempBuf accum;
+    if ((s = accum.get(sizeof(ScanAccum), "scan accumulators"))) return s;
+    ScanAccum *dacc = static_cast<ScanAccum *>(accum.p);
+    SD_CUDA_TRY(cudaMemsetAsync(dacc, 0, sizeof(ScanAccum), st));
+
+    if (d->validate && p->M > 0) {
+        validate_kernel<<<148 * 8, 256, 0, st>>>(p->rowptr, p->colind, p->M, p->K, p->nnz, dacc);
+        SD_CUDA_TRY(cudaGetLastError());
+        ScanAccum h;
+        SD_CUDA_TRY(cudaMemcpyAsync(&h, dacc, sizeof h, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        if (h.bad_csr) {
+            set_error(SD_ERR_INVALID_ARG, "malformed CSR: %llu offending rowptr / colind entries", h.bad_csr);
+            return SD_ERR_INVALID_ARG;
+        }
+    }
+
+    // ---- scan: row statistics + 16x16 block keys -> sort -> run-length encode ----------------
+    const int64_t Kb = (p->K + 15) / 16, Mb = (p->M + 15) / 16;
+    TempBuf keys_a, keys_b, counts, nruns, cubtmp;
+    int64_t nnzb = 0;
+    if (p->M > 0) {
+        if (p->nnz > 0) {
+            if ((s = keys_a.get(sizeof(unsigned long long) * p->nnz, "block keys"))) return s;
+            if ((s = keys_b.get(sizeof(unsigned long long) * p->nnz, "sorted block keys"))) return s;
+        }
+        const int blocks = static_cast<int>(std::min<int64_t>((p->M + 7) / 8, 148 * 16));
+        scan_rows_kernel<<<blocks, 256, 0, st>>>(p->rowptr, p->colind, p->M, Kb,
+                                                static_cast<unsigned long long *>(keys_a.p), dacc);
+        SD_CUDA_TRY(cudaGetLastError());
+    }
+    if (p->nnz > 0) {
+        int bits = 1;
+        while (bits < 64 && (static_cast<unsigned __int128>(1) << bits) < static_cast<unsigned __int128>(Mb) * Kb) ++bits;
+        auto *ka = static_cast<unsigned long long *>(keys_a.p);
+        auto *kb = static_cast<unsigned long long *>(keys_b.p);
+        size_t tb = 0;
+        SD_CUDA_TRY(cub::DeviceRadixSort::SortKeys(nullptr, tb, ka, kb, p->nnz, 0, bits, st));
+        if ((s = cubtmp.get(tb, "sort scratch"))) return s;
+        SD_CUDA_TRY(cub::DeviceRadixSort::SortKeys(cubtmp.p, tb, ka, kb, p->nnz, 0, bits, st));
+        if ((s = counts.get(sizeof(int32_t) * p->nnz, "block fill counts"))) return s;
+        if ((s = nruns.get(sizeof(int64_t), "block count"))) return s;
+        size_t tb2 = 0;
+        SD_CUDA_TRY(cub::DeviceRunLengthEncode::Encode(nullptr, tb2, kb, ka, static_cast<int32_t *>(counts.p),
+                                                       static_cast<int64_t *>(nruns.p), p->nnz, st));
+        if (tb2 > tb) {
+            cudaFree(cubtmp.p);
+            cubtmp.p = nullptr;
+            if ((s = cubtmp.get(tb2, "rle scratch"))) return s;
+        }
+        // distinct keys land in keys_a (its contents are no longer needed)
+        SD_CUDA_TRY(cub::DeviceRunLengthEncode::Encode(cubtmp.p, tb2, kb, ka, static_cast<int32_t *>(counts.p),
+                                                       static_cast<int64_t *>(nruns.p), p->nnz, st));
+        SD_CUDA_TRY(cudaMemcpyAsync(&nnzb, nruns.p, sizeof nnzb, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        block_fill_kernel<<<static_cast<int>(std::min<int64_t>((nnzb + 255) / 256, 148 * 8)), 256, 0, st>>>(
+            static_cast<int32_t *>(counts.p), nnzb, dacc);
+        SD_CUDA_TRY(cudaGetLastError());
+    }
+    ScanAccum h;
+    SD_CUDA_TRY(cudaMemcpyAsync(&h, dacc, sizeof h, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    for (int i = 0; i < 32; ++i) info.row_hist[i] = static_cast<int64_t>(h.row_hist[i]);
+    info.sum_r2 = h.sum_r2;
+    info.max_r = static_cast<int64_t>(h.max_r);
+    info.empty_rows = static_cast<int64_t>(h.empty_rows);
+    info.sum_span = h.sum_span;
+    info.max_span = static_cast<int64_t>(h.max_span);
+    info.sum_gap = h.sum_gap;
+    info.diag = static_cast<int64_t>(h.diag);
+    info.unsorted_rows = static_cast<int64_t>(h.unsorted_rows);
+    info.long_rows = static_cast<int64_t>(h.long_rows);
+    info.nnz_long_rows = static_cast<int64_t>(h.nnz_long_rows);
+    info.nnzb16 = nnzb;
+    for (int i = 0; i < 9; ++i) info.blk_hist[i] = static_cast<int64_t>(h.blk_hist[i]);
+    info.nnz_dense_blocks = static_cast<int64_t>(h.nnz_dense_blocks);
+
+    // ---- decision ------------------------------------------------------------------------------
+    int family = d->family == SD_AUTO ? decide_family(info) : d->family;
+    if (family == SD_BSR_TC && (info.unsorted_rows != 0 || p->nnz == 0)) {
+        if (d->family == SD_BSR_TC && info.unsorted_rows != 0) {
+            set_error(SD_ERR_UNSUPPORTED, "BSR needs strictly ascending columns in every row (%lld rows are not)",
+                      (long long)info.unsorted_rows);
+            return SD_ERR_UNSUPPORTED;
+        }
+        family = SD_ROWSPLIT;
+    }
+    info.family = family;
+
+    // ---- representation -----------------------------------------------------------------------
+    if (family == SD_MERGE && p->M > 0) {
+        if ((s = build_merge(p, st))) return s;
+    } else if (family == SD_BSR_TC) {
+        if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
+    }
+    info.plan_bytes = p->owned;
+    return SD_OK;
+}
+
+static void free_plan(sd_plan *p) {
+    if (!p) return;
+    cudaFree(p->tile_seg);
+    cudaFree(p->fix_tiles);
+    cudaFree(p->tile_head);
+    cudaFree(p->tile_tail);
+    cudaFree(p->browptr);
+    cudaFree(p->bcol);
+    cudaFree(p->bval);
+    cudaFree(p->stage_B);
+    cudaFree(p->stage_C);
+    if (p->host_stream) cudaStreamDestroy(p->host_stream);
+    delete p;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace sd
+
+// =====================================================================================
+// extern "C"
+// =====================================================================================
+using namespace sd;
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char *sd_version(void) { return "0.1"; }
+
+int sd_last_error(char *buf, size_t n) {
+    if (buf && n) {
+        strncpy(buf, g_err_text, n - 1);
+        buf[n - 1] = '\0';
+    }
+    return g_err_code;
+}
+
+sd_status_t sd_plan_create_ex(const sd_plan_desc_t *d, sd_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!d || !out) {
+        set_error(SD_ERR_INVALID_ARG, "desc and out must not be null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (d->M < 0 || d->K < 0 || d->N < 0 || d->M > INT32_MAX - 1 || d->K > INT32_MAX - 1 || d->N > INT32_MAX / 2) {
+        set_error(SD_ERR_INVALID_ARG, "M, K, N must be in [0, 2^31)");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (d->M > 0 && !d->rowptr) {
+        set_error(SD_ERR_INVALID_ARG, "rowptr is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (d->dtype != SD_F32 && d->dtype != SD_BF16) {
+        set_error(SD_ERR_INVALID_ARG, "unknown dtype %d", d->dtype);
+        return SD_ERR_INVALID_ARG;
+    }
+    if (d->family < SD_AUTO || d->family > SD_BSR_TC) {
+        set_error(SD_ERR_INVALID_ARG, "unknown family %d", d->family);
+        return SD_ERR_INVALID_ARG;
+    }
+    if (d->windows < 0 || d->windows > 64) {
+        set_error(SD_ERR_INVALID_ARG, "windows must be in [0, 64]");
+        return SD_ERR_INVALID_ARG;
+    }
+    sd_plan *p = new (std::nothrow) sd_plan;
+    if (!p) {
+        set_error(SD_ERR_ALLOC, "host allocation failed");
+        return SD_ERR_ALLOC;
+    }
+    const sd_status_t s = create_plan(d, p);
+    if (s != SD_OK) {
+        free_plan(p);
+        return s;
+    }
+    *out = p;
+    return SD_OK;
+}
+
+sd_plan_t *sd_plan_create(const int32_t *rowptr, const int32_t *colind, const float *vals, int64_t M, int64_t K,
+                          int64_t N) {
+    sd_plan_desc_t d;
+    memset(&d, 0, sizeof d);
+    d.rowptr = rowptr;
+    d.colind = colind;
+    d.vals = vals;
+    d.M = M;
+    d.K = K;
+    d.N = N;
+    d.dtype = SD_F32;
+    d.family = SD_AUTO;
+    sd_plan_t *p = nullptr;
+    sd_plan_create_ex(&d, &p);
+    return p;
+}
+
+void sd_plan_destroy(sd_plan_t *plan) { free_plan(plan); }
+
+sd_status_t sd_plan_get_info(const sd_plan_t *plan, sd_plan_info_t *out) {
+    if (!plan || !out) {
+        set_error(SD_ERR_INVALID_ARG, "plan and out must not be null");
+        return SD_ERR_INVALID_ARG;
+    }
+    *out = plan->info;
+    return SD_OK;
+}
+
+sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bcol, void *bval) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->info.family != SD_BSR_TC) {
+        set_error(SD_ERR_UNSUPPORTED, "the plan holds no BSR representation");
+        return SD_ERR_UNSUPPORTED;
+    }
+    const int64_t Mb = (plan->M + 15) / 16;
+    const size_t es = plan->dtype == SD_F32 ? 4 : 2;
+    if (browptr) SD_CUDA_TRY(cudaMemcpy(browptr, plan->browptr, sizeof(int32_t) * (Mb + 1), cudaMemcpyDeviceToHost));
+    if (bcol && plan->nnzb)
+        SD_CUDA_TRY(cudaMemcpy(bcol, plan->bcol, sizeof(int32_t) * plan->nnzb, cudaMemcpyDeviceToHost));
+    if (bval && plan->nnzb) SD_CUDA_TRY(cudaMemcpy(bval, plan->bval, es * 256 * plan->nnzb, cudaMemcpyDeviceToHost));
+    return SD_OK;
+}
+
+sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t cap, int64_t *count) {
+    if (!plan || !count) {
+        set_error(SD_ERR_INVALID_ARG, "plan and count must not be null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->info.family != SD_MERGE) {
+        set_error(SD_ERR_UNSUPPORTED, "the plan holds no merge-path tile table");
+        return SD_ERR_UNSUPPORTED;
+    }
+    const int64_t n = plan->M > 0 ? static_cast<int64_t>(plan->ntiles) + 1 : 0;
+    *count = n;
+    if (tile_seg && cap >= n && n > 0)
+        SD_CUDA_TRY(cudaMemcpy(tile_seg, plan->tile_seg, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+    return SD_OK;
+}
+
+sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc, float alpha, float beta,
+                    void *stream) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    const int64_t M = plan->M, N = plan->N;
+    if (M == 0 || N == 0) return SD_OK;
+    if (!C || ldc < N) {
+        set_error(SD_ERR_INVALID_ARG, "C is null or ldc < N");
+        return SD_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (alpha == 0.f || plan->nnz == 0) {
+        SD_CUDA_TRY(run_scale_c(C, ldc, M, static_cast<int32_t>(N), beta, st));
+        return SD_OK;
+    }
+    if (!B || ldb < N) {
+        set_error(SD_ERR_INVALID_ARG, "B is null or ldb < N");
+        return SD_ERR_INVALID_ARG;
+    }
+    const int vw = plan->dtype == SD_F32 ? 4 : 8;
+    const bool vec = aligned16(B) && aligned16(C) && N % vw == 0 && ldb % vw == 0 && ldc % 4 == 0;
+
+    SpmmArgs a;
+    a.ptr = plan->rowptr;
+    a.colind = plan->colind;
+    a.vals = plan->vals;
+    a.seg_row = nullptr;
+    a.B = B;
+    a.C = C;
+    a.ldb = ldb;
+    a.ldc = ldc;
+    a.S = M;
+    a.N = static_cast<int32_t>(N);
+    a.alpha = alpha;
+    a.beta = beta;
+
+    switch (plan->info.family) {
+    case SD_ROWSPLIT:
+        SD_CUDA_TRY(run_rowsplit(a, plan->dtype, vec, st));
+        return SD_OK;
+    case SD_MERGE: {
+        MergeArgs m;
+        m.s = a;
+        m.tile_seg = plan->tile_seg;
+        m.tile_head = plan->tile_head;
+        m.tile_tail = plan->tile_tail;
+        m.seg_begin = 0;
+        m.seg_end = M;
+        m.ntiles = plan->ntiles;
+        SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_tiles, plan->nfix, st));
+        return SD_OK;
+    }
+    case SD_BSR_TC: {
+        BsrArgs b;
+        b.browptr = plan->browptr;
+        b.bcol = plan->bcol;
+        b.bval = plan->bval;
+        b.bval_mma = nullptr;
+        b.B = B;
+        b.C = C;
+        b.ldb = ldb;
+        b.ldc = ldc;
+        b.M = M;
+        b.K = plan->K;
+        b.Mb = static_cast<int32_t>((M + 15) / 16);
+        b.N = static_cast<int32_t>(N);
+        b.alpha = alpha;
+        b.beta = beta;
+        const bool vec4 = aligned16(B) && aligned16(C) && N % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
+                          (plan->dtype == SD_F32 || (reinterpret_cast<uintptr_t>(B) & 7u) == 0);
+        SD_CUDA_TRY(run_bsr_simt(b, plan->dtype, vec4, st));
+        return SD_OK;
+    }
+    default:
+        set_error(SD_ERR_INTERNAL, "plan has no family");
+        return SD_ERR_INTERNAL;
+    }
+}
+
+sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host, int64_t ldc, float alpha,
+                         float beta) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    const int64_t M = plan->M, N = plan->N, K = plan->K;
+    if (M == 0 || N == 0) return SD_OK;
+    if (!C_host || ldc < N || !B_host || ldb < N) {
+        set_error(SD_ERR_INVALID_ARG, "null host buffer or leading dimension < N");
+        return SD_ERR_INVALID_ARG;
+    }
+    const size_t es = plan->dtype == SD_F32 ? 4 : 2;
+    sd_status_t s;
+    if (!plan->host_stream) SD_CUDA_TRY(cudaStreamCreateWithFlags(&plan->host_stream, cudaStreamNonBlocking));
+    if (!plan->stage_B && (s = dev_alloc(plan, &plan->stage_B, es * K * N, "B staging"))) return s;
+    if (!plan->stage_C && (s = dev_alloc(plan, reinterpret_cast<void **>(&plan->stage_C), sizeof(float) * M * N,
+                                         "C staging")))
+        return s;
+    cudaStream_t st = plan->host_stream;
+    SD_CUDA_TRY(cudaMemcpy2DAsync(plan->stage_B, es * N, B_host, es * ldb, es * N, K, cudaMemcpyHostToDevice, st));
+    if (beta != 0.f)
+        SD_CUDA_TRY(cudaMemcpy2DAsync(plan->stage_C, 4 * N, C_host, 4 * ldc, 4 * N, M, cudaMemcpyHostToDevice, st));
+    if ((s = sd_spmm(plan, plan->stage_B, N, plan->stage_C, N, alpha, beta, st))) return s;
+    SD_CUDA_TRY(cudaMemcpy2DAsync(C_host, 4 * ldc, plan->stage_C, 4 * N, 4 * N, M, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    return SD_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Shared device/host helpers of the SpMM library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/sd.h"
+
+namespace sd {
+
+// ---- error reporting (thread-local text + code) --------------------------------
+void set_error(sd_status_t code, const char *fmt, ...);
+sd_status_t cuda_fail(cudaError_t e, const char *what);
+
+#define SD_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t e__ = (expr);                           \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr); \
+    } while (0)
+
+// ---- element access -------------------------------------------------------------
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Vector width in elements of a 16-byte load of T.
+template <typename T> struct vec_width;
+template <> struct vec_width<float> { static constexpr int value = 4; };
+template <> struct vec_width<__nv_bfloat16> { static constexpr int value = 8; };
+
+// Load VW consecutive elements of T (read-only path) and widen to float.
+template <typename T, int VW> struct RowLoad;
+
+template <> struct RowLoad<float, 4> {
+    __device__ __forceinline__ static void ld(const float *p, float (&o)[4]) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(p));
+        o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+    }
+};
+template <> struct RowLoad<float, 1> {
+    __device__ __forceinline__ static void ld(const float *p, float (&o)[1]) { o[0] = __ldg(p); }
+};
+template <> struct RowLoad<__nv_bfloat16, 8> {
+    __device__ __forceinline__ static void ld(const __nv_bfloat16 *p, float (&o)[8]) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(p));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {       // bf16 is the upper half of a float
+            o[2 * i] = __uint_as_float(w[i] << 16);
+            o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+};
+template <> struct RowLoad<__nv_bfloat16, 1> {
+    __device__ __forceinline__ static void ld(const __nv_bfloat16 *p, float (&o)[1]) {
+        o[0] = __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+    }
+};
+
+// How one output row leaves the registers.
+//   mode 0: C = alpha*acc + beta*C   (first and only write of the row; beta == 0 never reads C)
+//   mode 1: C = C + alpha*acc        (later column window of a row already written)
+template <int VW>
+__device__ __forceinline__ void store_cols(float *c, const float (&acc)[VW], float alpha, float beta,
+                                           int accumulate) {
+    if constexpr (VW == 1) {
+        float r = alpha * acc[0];
+        if (accumulate) r += *c;
+        else if (beta != 0.f) r += beta * *c;
+        *c = r;
+    } else {
+#pragma unroll
+        for (int q = 0; q < VW / 4; ++q) {
+            float4 *p = reinterpret_cast<float4 *>(c) + q;
+            float4 r = make_float4(alpha * acc[4 * q], alpha * acc[4 * q + 1], alpha * acc[4 * q + 2],
+                                   alpha * acc[4 * q + 3]);
+            if (accumulate) {
+                const float4 o = *p;
+                r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w;
+            } else if (beta != 0.f) {
+                const float4 o = *p;
+                r.x += beta * o.x; r.y += beta * o.y; r.z += beta * o.z; r.w += beta * o.w;
+            }
+            *p = r;
+        }
+    }
+}
+
+// Arguments common to the CSR kernels.
+struct SpmmArgs {
+    const int32_t *ptr;     // row (or segment) pointer array, [S+1]
+    const int32_t *colind;  // [nnz]
+    const void *vals;       // [nnz] float or bf16
+    const int32_t *seg_row; // nullptr: segment s is row s.  Else output row of segment s;
+                            // bit 31 set: the row was already written by an earlier window.
+    const void *B;
+    float *C;
+    int64_t ldb, ldc;
+    int64_t S;              // number of rows / segments
+    int32_t N;
+    float alpha, beta;
+};
+
+inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
+
+}  // namespace sd

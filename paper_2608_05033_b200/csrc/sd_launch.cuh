@@ -1,0 +1,49 @@
+// Host entry points of the kernel families, one translation unit each.
+#pragma once
+
+#include "sd_common.cuh"
+
+namespace sd {
+
+// Every tile holds the same number of merged items whatever the lane geometry, so one tile
+// table serves every dense width and both the vector and the scalar kernels.
+constexpr int kMergeTile = 1024;
+
+struct MergeArgs {
+    SpmmArgs s;
+    const int32_t *tile_seg;  // [ntiles + 1] segment coordinate of each tile start (global seg ids)
+    float *tile_head;         // [ntiles][N]  partial of the segment open at tile start, if it ends here
+    float *tile_tail;         // [ntiles][N]  partial of the segment still open at tile end
+    int64_t seg_begin;        // first segment of this window
+    int64_t seg_end;          // one past the last segment of this window
+    int32_t ntiles;
+};
+
+
+// Family (a).  `vec`: B, C, ldb, ldc and N allow 16-byte accesses.
+cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
+
+// C = beta * C.
+cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st);
+
+// Family (b): tile kernel, then the carry-out fix-up for the `nfix` tiles listed in fix_tiles.
+cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fix_tiles, int32_t nfix,
+                      cudaStream_t st);
+
+// Family (c).
+struct BsrArgs {
+    const int32_t *browptr;  // [Mb + 1]
+    const int32_t *bcol;     // [nnzb]
+    const void *bval;        // [nnzb][16][16] row-major, plan dtype
+    const void *bval_mma;    // [nnzb] tensor-core operand images of the same blocks
+    const void *B;
+    float *C;
+    int64_t ldb, ldc;
+    int64_t M, K;
+    int32_t Mb;
+    int32_t N;
+    float alpha, beta;
+};
+cudaError_t run_bsr_simt(const BsrArgs &a, int dtype, bool vec, cudaStream_t st);
+
+}  // namespace sd

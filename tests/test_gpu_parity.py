@@ -1,0 +1,312 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+Tolerance (fp): |C - Cref| <= rel * (|alpha| sum|a||b| + |beta||Cin|) + 1e-6, rel = 1e-5 for
+fp32 values and 1e-2 for bf16 values; integer work (plan summary, BSR, tile table) bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if torch.cuda.is_available():
+    import paper_2608_05033_b200 as sd
+    from util import DeviceWorkload, run_spmm
+else:  # collected but skipped
+    sd = None
+
+FAMILIES = {"rowsplit": 1, "merge": 2, "bsr": 3}
+
+
+def check(w, got, c_in=None, alpha=None, beta=None):
+    alpha = w.alpha if alpha is None else alpha
+    beta = w.beta if beta is None else beta
+    cin = c_in if c_in is not None else w.C0
+    r = oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, got, cin, alpha, beta)
+    assert r["ok"], r
+    return r
+
+
+def shape_lengths(kind, M, K, rng):
+    if kind == "uniform":
+        return np.clip(rng.poisson(8, M), 0, K)
+    if kind == "short":
+        return rng.integers(0, 4, M)
+    if kind == "skewed":
+        r = np.clip((2000.0 * np.arange(1, M + 1) ** -1.2).astype(np.int64), 1, min(K, 3000))
+        return rng.permutation(r)
+    if kind == "onelong":
+        r = np.zeros(M, np.int64)
+        r[M // 3] = K
+        r[M - 1] = K // 2
+        return r
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("family", ["rowsplit", "merge"])
+@pytest.mark.parametrize("kind", ["uniform", "short", "skewed", "onelong"])
+@pytest.mark.parametrize("N", [1, 4, 8, 32, 64, 128, 256, 7, 100])
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_forced_family_small(family, kind, N, dtype):
+    rng = np.random.default_rng(hash((family, kind, N)) % 2**32)
+    M, K = 1237, 3001   # ragged: not multiples of any tile
+    w = W.random_csr(M, K, N, shape_lengths(kind, M, K, rng), seed=N * 7 + 1, dtype=dtype, alpha=1.25, beta=-0.5)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=FAMILIES[family])
+    assert plan.info().family == FAMILIES[family]
+    got, intact = run_spmm(plan, w)
+    assert intact
+    check(w, got)
+    # run again: bit-identical (no float atomics)
+    got2, _ = run_spmm(plan, w)
+    assert np.array_equal(got, got2)
+    # beta == 0 must not read C: poison it
+    poison = np.full((M, N), np.nan, np.float32)
+    got3, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got3, beta=0.0)
+    plan.close()
+
+
+@pytest.mark.parametrize("family", ["rowsplit", "merge", "bsr"])
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_padding_and_misalignment(family, dtype):
+    rng = np.random.default_rng(5)
+    M, K, N = 300, 517, 32
+    w = W.random_csr(M, K, N, np.clip(rng.poisson(6, M), 0, K), seed=77, dtype=dtype, beta=0.75)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=FAMILIES[family])
+    for pad_b, pad_c, off in [(3, 5, 0), (4, 8, 0), (0, 0, 1), (1, 2, 3), (8, 4, 4)]:
+        got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_c, offset=off)
+        assert intact, (pad_b, pad_c, off)
+        check(w, got)
+    plan.close()
+
+
+@pytest.mark.parametrize("family", ["rowsplit", "merge", "bsr"])
+def test_degenerate_cases(family):
+    fam = FAMILIES[family]
+    # alpha == 0: C = beta*C, A and B untouched
+    w = W.random_csr(64, 64, 8, np.full(64, 3), seed=3, beta=2.0)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=fam)
+    got, _ = run_spmm(plan, w, alpha=0.0)
+    assert np.array_equal(got, np.float32(2.0) * w.C0)
+    plan.close()
+    # no nonzeros at all
+    w = W.random_csr(50, 40, 4, np.zeros(50, np.int64), seed=4, beta=0.0)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=fam)
+    assert plan.info().nnz == 0
+    got, _ = run_spmm(plan, w, c_fill=np.full((50, 4), np.nan, np.float32))
+    assert np.array_equal(got, np.zeros((50, 4), np.float32))
+    plan.close()
+    # M == 0 and N == 0: nothing launched, SD_OK
+    rp = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p0 = sd.Plan(rp, rp, torch.zeros(1, device="cuda"), 0, 10, 4, family=fam)
+    sd.sd_spmm(p0.handle, 0, 4, 0, 4, 1.0, 0.0)
+    p0.close()
+    w = W.random_csr(8, 8, 1, np.full(8, 2), seed=9)
+    dw = DeviceWorkload(w)
+    pn = dw.plan(family=fam, N=0)
+    sd.sd_spmm(pn.handle, 0, 0, 0, 0, 1.0, 0.0)
+    pn.close()
+
+
+def test_invalid_arguments_return_codes():
+    w = W.random_csr(16, 16, 4, np.full(16, 2), seed=1)
+    dw = DeviceWorkload(w)
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_create_ex(None, dw.colind, dw.vals, 16, 16, 4)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_create_ex(dw.rowptr, dw.colind, dw.vals, -1, 16, 4)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_create_ex(dw.rowptr, dw.colind, dw.vals, 16, 16, 4, dtype=7)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_create_ex(dw.rowptr, dw.colind, dw.vals, 16, 16, 4, family=9)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    # malformed CSR is caught by validation
+    bad = dw.colind.clone()
+    bad[3] = 99
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_create_ex(dw.rowptr, bad, dw.vals, 16, 16, 4, validate=True)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    plan = dw.plan()
+    B = torch.zeros(16, 4, device="cuda")
+    Cm = torch.zeros(16, 4, device="cuda")
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_spmm(plan.handle, B, 3, Cm, 4, 1.0, 0.0)     # ldb < N
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_spmm(plan.handle, B, 4, None, 4, 1.0, 0.0)   # null C
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_spmm(None, B, 4, Cm, 4, 1.0, 0.0)
+    assert e.value.code == sd.SD_ERR_INVALID_ARG
+    with pytest.raises(sd.SdError) as e:
+        sd.sd_plan_get_bsr(plan.handle)
+    assert e.value.code == sd.SD_ERR_UNSUPPORTED
+    sd.sd_plan_destroy(None)   # no-op
+    plan.close()
+    # the context is still healthy
+    torch.cuda.synchronize()
+
+
+def small_configs():
+    return {
+        "tiny_uniform": W.g1_tiny_uniform(),
+        "stencil": W.g2_stencil(n=96, N=64),
+        "gcn_rmat": W.g3_gcn_rmat(scale=13, N=128),
+        "block16_f32": W.g4_block(Mb=128, Kb=128, N=256, nblocks=300),
+        "block16_bf16": W.g4_block(Mb=128, Kb=128, N=256, nblocks=300, dtype=W.SD_BF16),
+        "skewed": W.g5_skewed(M=1 << 16, N=32, scale_c=2.4e7 / 64, cap=4000),
+    }
+
+
+EXPECTED_FAMILY = {"tiny_uniform": 1, "stencil": 1, "gcn_rmat": 2, "block16_f32": 3, "block16_bf16": 3, "skewed": 2}
+
+
+@pytest.mark.parametrize("name", list(EXPECTED_FAMILY))
+def test_scaled_configs_auto_plan_and_plan_parity(name):
+    w = small_configs()[name]
+    dw = DeviceWorkload(w)
+    plan = dw.plan(validate=True)
+    info = plan.info()
+    # plan metadata: bit-exact against the oracle's own summary and rule
+    ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+    mine = info.as_dict()
+    for k, v in ref.as_dict().items():
+        assert mine[k] == v, k
+    assert info.family == oracle.decide(ref) == EXPECTED_FAMILY[name]
+    if info.family == sd.SD_MERGE:
+        tiles = sd.sd_plan_get_tiles(plan.handle)
+        assert np.array_equal(tiles, oracle.merge_coords(w.rowptr, info.tile_items))
+        assert info.num_tiles == tiles.size - 1
+    if info.family == sd.SD_BSR_TC:
+        browptr, bcol, bval = sd.sd_plan_get_bsr(plan.handle)
+        rb, rc, rv = oracle.bsr16(w.rowptr, w.colind, w.vals, w.M, w.K)
+        assert np.array_equal(browptr, rb) and np.array_equal(bcol, rc)
+        assert bval.tobytes() == rv.tobytes()
+    got, intact = run_spmm(plan, w)
+    assert intact
+    check(w, got)
+    got2, _ = run_spmm(plan, w)
+    assert np.array_equal(got, got2)
+    plan.close()
+
+
+def test_partially_filled_blocks_bsr_parity():
+    # blocks on the last partial block-row / block-column, fill well below 100 %
+    rng = np.random.default_rng(8)
+    M, K, N = 1000 + 7, 500 + 3, 64
+    w = W.random_csr(M, K, N, np.clip(rng.poisson(20, M), 0, K), seed=12, beta=1.5)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_BSR_TC)
+    browptr, bcol, bval = sd.sd_plan_get_bsr(plan.handle)
+    rb, rc, rv = oracle.bsr16(w.rowptr, w.colind, w.vals, M, K)
+    assert np.array_equal(browptr, rb) and np.array_equal(bcol, rc) and bval.tobytes() == rv.tobytes()
+    got, intact = run_spmm(plan, w)
+    assert intact
+    check(w, got)
+    plan.close()
+
+
+def test_unsorted_and_duplicate_columns():
+    # CSR families accept any order and sum duplicates; BSR is refused for such input
+    rng = np.random.default_rng(4)
+    M, K, N = 200, 90, 16
+    w = W.random_csr(M, K, N, rng.integers(1, 12, M), seed=6)
+    for i in range(0, M, 3):     # reverse some rows, duplicate an entry in others
+        lo, hi = w.rowptr[i], w.rowptr[i + 1]
+        w.colind[lo:hi] = w.colind[lo:hi][::-1].copy()
+        w.vals[lo:hi] = w.vals[lo:hi][::-1].copy()
+        if hi - lo >= 2 and i % 2 == 0:
+            w.colind[lo + 1] = w.colind[lo]
+    dw = DeviceWorkload(w)
+    for fam in (sd.SD_ROWSPLIT, sd.SD_MERGE):
+        plan = dw.plan(family=fam)
+        assert plan.info().unsorted_rows == oracle.summary(w.rowptr, w.colind, M, K, N).unsorted_rows > 0
+        got, _ = run_spmm(plan, w)
+        check(w, got)
+        plan.close()
+    with pytest.raises(sd.SdError) as e:
+        dw.plan(family=sd.SD_BSR_TC)
+    assert e.value.code == sd.SD_ERR_UNSUPPORTED
+    assert dw.plan().info().family != sd.SD_BSR_TC
+
+
+def test_long_all_positive_row_stays_inside_tolerance():
+    # 200,000 same-sign terms in one row: sequential fp32 summation would drift to the edge of
+    # 1e-5; the tiled summation of the merge family must stay well inside
+    M, K, N = 64, 262144, 32
+    r = np.full(M, 3, np.int64)
+    r[17] = 200_000
+    w = W.random_csr(M, K, N, r, seed=31, positive=True)
+    dw = DeviceWorkload(w)
+    for fam in (sd.SD_MERGE, sd.SD_ROWSPLIT):
+        plan = dw.plan(family=fam)
+        got, _ = run_spmm(plan, w)
+        res = check(w, got)
+        if fam == sd.SD_MERGE:
+            assert res["max_ratio"] < 0.5
+        plan.close()
+    assert dw.plan().info().family == sd.SD_MERGE
+
+
+def test_one_row_holds_every_nonzero_and_rows_straddle_many_tiles():
+    M, K, N = 5000, 40000, 8
+    r = np.zeros(M, np.int64)
+    r[4321] = 30000
+    w = W.random_csr(M, K, N, r, seed=2)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE)
+    got, _ = run_spmm(plan, w, c_fill=np.full((M, N), np.nan, np.float32))
+    check(w, got)
+    plan.close()
+    # rows of ~2.5 tiles each, back to back
+    r = np.full(40, 2600, np.int64)
+    w = W.random_csr(40, 8192, 32, r, seed=3, beta=0.25)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE)
+    got, _ = run_spmm(plan, w)
+    check(w, got)
+    plan.close()
+
+
+def test_identity_and_permutation_are_exact():
+    n, N = 4096, 64
+    rng = np.random.default_rng(0)
+    perm = rng.permutation(n).astype(np.int32)
+    B = rng.standard_normal((n, N)).astype(np.float32)
+    w = W.Workload("perm", n, n, N, np.arange(n + 1, dtype=np.int32), perm, np.ones(n, np.float32), B, None)
+    dw = DeviceWorkload(w)
+    for fam in (sd.SD_ROWSPLIT, sd.SD_MERGE):
+        plan = dw.plan(family=fam)
+        got, _ = run_spmm(plan, w)
+        assert np.array_equal(got, B[perm])
+        plan.close()
+
+
+def test_plan_reuse_with_second_dense_operand_and_host_entry():
+    w = W.g1_tiny_uniform(M=512, K=700, N=32, seed=8)
+    dw = DeviceWorkload(w)
+    plan = dw.plan()
+    got, _ = run_spmm(plan, w)
+    check(w, got)
+    w2 = W.g1_tiny_uniform(M=512, K=700, N=32, seed=8)
+    w2.B = np.random.default_rng(1).standard_normal(w.B.shape).astype(np.float32)
+    got2, _ = run_spmm(plan, w2)
+    check(w2, got2)
+    # host buffers through sd_spmm_host
+    Bh = torch.from_numpy(w2.B).pin_memory()
+    Ch = torch.full((w.M, w.N), float("nan")).pin_memory()
+    plan.spmm_host(Bh, Ch, 1.0, 0.0)
+    assert np.array_equal(Ch.numpy(), got2)
+    Cin = np.random.default_rng(2).standard_normal((w.M, w.N)).astype(np.float32)
+    Ch = torch.from_numpy(Cin.copy()).pin_memory()
+    plan.spmm_host(Bh, Ch, 0.5, 2.0)
+    check(w2, Ch.numpy(), c_in=Cin, alpha=0.5, beta=2.0)
+    plan.close()
