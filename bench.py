@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the structure-adaptive SpMM path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--configs 1,2,3,4] [--impl reference]
+
+One *step* is one pass of the whole hot path: one sd_spmm call on each benchmark workload
+(stencil N=64 -> family (a), GCN R-MAT N=128 and skewed N=32 -> family (b), block16 N=256 in
+fp32 and bf16 -> family (c)), inputs resident in HBM, L2 flushed before every call.  The JSON
+line's `value` is sum(2*nnz*N) / sum(device time) over the step; `per_config` carries each
+workload's own GFLOP/s, effective GB/s on the compulsory-traffic model and fraction of the
+measured HBM peak.  `e2e` runs the same step through sd_spmm_host with pinned host buffers
+(B copied in, C copied out, every call).  `--impl reference` times the CPU oracle instead.
+
+With N > 1 ranks (torchrun), every rank runs the step on its own dense operands (independent
+problems, no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "SpMM GFLOP/s (2*nnz*N) and effective HBM GB/s as % of B200 peak, 1 GPU"
+
+# (label, config index, dtype)
+BENCH_SET = [("stencil_f32", 1, W.SD_F32), ("gcn_rmat_f32", 2, W.SD_F32), ("block16_f32", 3, W.SD_F32),
+             ("block16_bf16", 3, W.SD_BF16), ("skewed_f32", 4, W.SD_F32)]
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic():
+    """Per-launch DRAM bytes of the kernels, as captured with ncu (profiles/traffic.json)."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p))
+        except Exception:
+            pass
+    return {}
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) during the timed region."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _once(self):
+        nv = self.nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            try:
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            except Exception:
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                     0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+            for bit, name in names.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def start(self):
+        if self.nv is None:
+            return
+        def loop():
+            while not self._stop.is_set():
+                self._once()
+                time.sleep(self.period)
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
+
+    def stop(self) -> dict:
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- multi-rank plumbing
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(x: float, device=None) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, device=None) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(w: W.Workload, budget_flops: float, seed: int):
+    """Rows of a seeded random order until their 2*nnz*N reaches the budget."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    order = rng.permutation(w.M)
+    per_row = 2.0 * np.diff(w.rowptr)[order] * w.N
+    n = int(np.searchsorted(np.cumsum(per_row), budget_flops)) + 1
+    rows = np.sort(order[:min(n, w.M)]).astype(np.int64)
+    flops = float(2.0 * np.diff(w.rowptr)[rows].sum() * w.N)
+    return rows, flops
+
+
+def time_oracle(sets, budget_flops: float):
+    """One pass of the oracle (as it stands: double accumulation, abs-sum companion) over the
+    row samples.  Returns (seconds, flops)."""
+    import oracle
+    total_t, total_f = 0.0, 0.0
+    for w, rows, flops in sets:
+        t0 = time.perf_counter()
+        oracle.spmm_rows(rows, w.rowptr, w.colind, w.vals, w.B, w.N, w.C0, w.alpha, w.beta)
+        total_t += time.perf_counter() - t0
+        total_f += flops
+    return total_t, total_f
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the CPU oracle on a bounded row sample of the same workloads."""
+    if rank != 0:
+        return
+    import oracle
+    ws = [make_workload(args, ci, dt) for _, ci, dt in select_set(args)]
+    budget = 2.0e8   # flops per workload per step: about a second of host work per step in total
+    sets = []
+    for i, w in enumerate(ws):
+        rows, flops = oracle_sample(w, budget, 1234 + i)
+        sets.append((w, rows, flops))
+    for _ in range(args.warmup):
+        time_oracle(sets, budget)
+    ts, fl = [], 0.0
+    for _ in range(args.steps):
+        t, fl = time_oracle(sets, budget)
+        ts.append(t)
+    sec = float(np.mean(ts))
+    value = fl / sec / 1e9
+    sample = "seeded random rows, ~2e8 flops per workload per step: " + ", ".join(
+        f"{lab}:{len(r)} rows" for (lab, _, _), (_, r, _) in zip(select_set(args), sets))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args)},
+        "cpu_baseline": {"value": value, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU leg
+SMALL_KW = {1: dict(n=768), 2: dict(scale=18), 3: dict(Mb=2048, Kb=2048), 4: dict(M=1 << 20, scale_c=2.4e7 / 4, cap=50000)}
+
+
+def make_workload(args, ci, dt):
+    return W.config(ci, dtype=dt, **(SMALL_KW[ci] if args.small else {}))
+
+
+def select_set(args):
+    if not args.configs:
+        return BENCH_SET
+    want = {int(x) for x in args.configs.split(",")}
+    return [b for b in BENCH_SET if b[1] in want]
+
+
+def workload_name(args):
+    return "suite: " + " | ".join(lab for lab, _, _ in select_set(args)) + \
+        " (stencil 1024^2 grid N=64 beta=0.5; R-MAT scale 20 GCN N=128; 16x16 dense blocks 0.2% of " \
+        "4096^2 positions N=256; rank-size Zipf(1.2) rows cap 200000 N=32)"
+
+
+def run_gpu(args, rank, local_rank, world):
+    import torch
+    import paper_2608_05033_b200 as sd
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    sd.load()
+    peak, peak_kind = measured_peak()
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).to(dev)
+
+    cases = []
+    t_gen0 = time.time()
+    for lab, ci, dt in select_set(args):
+        w = make_workload(args, ci, dt)
+        if rank > 0:   # independent problems: every rank draws its own dense operands
+            rng = np.random.Generator(np.random.PCG64(W.SEED_BASE + 100 * rank + ci))
+            Bf = rng.standard_normal(size=(w.K, w.N), dtype=np.float32)
+            w.B = Bf if dt == W.SD_F32 else W.f32_to_bf16_bits(Bf).reshape(w.K, w.N)
+        rowptr, colind, vals = to_dev(w.rowptr), to_dev(w.colind), to_dev(w.vals)
+        t0 = time.time()
+        plan = sd.Plan(rowptr, colind, vals, w.M, w.K, w.N, dtype=w.dtype)
+        torch.cuda.synchronize()
+        plan_ms = (time.time() - t0) * 1e3
+        Bd = to_dev(w.B)
+        Cd = to_dev(w.C0) if w.C0 is not None else torch.zeros((w.M, w.N), dtype=torch.float32, device=dev)
+        cases.append({"label": lab, "w": w, "plan": plan, "B": Bd, "C": Cd, "plan_ms": plan_ms,
+                      "info": plan.info(), "times": []})
+    gen_s = time.time() - t_gen0
+
+    flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def one_step(record: bool):
+        evs = []
+        for c in cases:
+            flush.fill_(1.0)                         # L2 flush, outside the timed interval
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            c["plan"].spmm(c["B"], c["C"], c["w"].alpha, c["w"].beta, stream)
+            e1.record(stream)
+            evs.append((c, e0, e1))
+        torch.cuda.synchronize()
+        tot = 0.0
+        for c, e0, e1 in evs:
+            ms = e0.elapsed_time(e1)
+            tot += ms
+            if record:
+                c["times"].append(ms)
+        return tot
+
+    for _ in range(max(args.warmup, 3)):
+        one_step(False)
+    barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    wall0 = time.perf_counter()
+    step_ms = [one_step(True) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    barrier()
+    wall_ms = (time.perf_counter() - wall0) * 1e3 / args.steps
+    clocks = sampler.stop()
+
+    local_ms = float(np.mean(step_ms))
+    ms_per_step = max_over_ranks(local_ms, dev)
+    flops_local = float(sum(c["w"].flops() for c in cases))
+    bytes_local = float(sum(c["w"].compulsory_bytes() for c in cases))
+    flops_all = sum_over_ranks(flops_local, dev)
+    bytes_all = sum_over_ranks(bytes_local, dev)
+    value = flops_all / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers through sd_spmm_host, copies inside the timed region --------
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 3))
+    h2d = d2h = 0
+    hosts = []
+    for c in ([] if args.no_e2e else cases):
+        w = c["w"]
+        Bh = torch.from_numpy(w.B.view(np.int16) if w.B.dtype == np.uint16 else w.B).pin_memory()
+        Ch = (torch.from_numpy(w.C0.copy()) if w.C0 is not None else torch.zeros((w.M, w.N))).pin_memory()
+        hosts.append((Bh, Ch))
+        h2d += Bh.numel() * Bh.element_size() + (Ch.numel() * 4 if w.beta != 0.0 else 0)
+        d2h += Ch.numel() * 4
+
+    def e2e_step():
+        for c, (Bh, Ch) in zip(cases, hosts):
+            c["plan"].spmm_host(Bh, Ch, c["w"].alpha, c["w"].beta)
+
+    if e2e_steps:
+        e2e_step()
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_local = (time.perf_counter() - t0) * 1e3 / max(e2e_steps, 1) if e2e_steps else float("inf")
+    e2e_ms = max_over_ranks(e2e_local, dev)
+    e2e_value = flops_all / (e2e_ms * 1e-3) / 1e9
+
+    if rank != 0:
+        return
+
+    # ---- per-config table, roofline of the dominant kernel ------------------------------------------
+    traffic = ncu_traffic()
+    per = []
+    for c in cases:
+        w, info = c["w"], c["info"]
+        ms = float(np.mean(c["times"]))
+        gbs = w.compulsory_bytes() / (ms * 1e-3) / 1e9
+        per.append({"workload": c["label"], "family": sd.FAMILY_NAMES[info.family], "M": w.M, "N": w.N,
+                    "nnz": w.nnz, "ms": ms, "ms_min": float(np.min(c["times"])),
+                    "gflops": w.flops() / (ms * 1e-3) / 1e9, "compulsory_bytes": w.compulsory_bytes(),
+                    "effective_gbs": gbs, "frac_of_measured_hbm": gbs / peak,
+                    "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS, "launches": int(info.launches),
+                    "plan_ms": c["plan_ms"], "plan_bytes": int(info.plan_bytes)})
+    dom = max(per, key=lambda p: p["ms"])
+    roofline = {"bound": "hbm", "kernel": dom["family"] + " on " + dom["workload"],
+                "achieved": dom["effective_gbs"], "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": dom["effective_gbs"] / peak,
+                "traffic": traffic.get(dom["workload"], {}).get("dram_bytes_per_launch"),
+                "note": "achieved = compulsory-model bytes of the call / its CUDA-event time"}
+
+    # ---- CPU baseline: the oracle on a bounded sample, this machine's host cores --------------------------
+    import oracle
+    sets = []
+    for i, c in enumerate([] if args.no_e2e else cases):
+        rows, fl = oracle_sample(c["w"], 4.0e9, 1234 + i)
+        sets.append((c["w"], rows, fl))
+    tsec, fl = time_oracle(sets, 4.0e9)
+    tsec2, _ = time_oracle(sets, 4.0e9)
+    tsec = max(min(tsec, tsec2), 1e-9)
+    cpu = {"value": fl / tsec / 1e9, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": "seeded random rows, ~4e9 flops per workload: " + ", ".join(
+               f"{c['label']}:{len(r)} rows" for c, (_, r, _) in zip(cases, sets)), "seconds": tsec}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(args),
+                   "l2": "512 MB flush write before every call (outside the timed events); every workload "
+                         "but block16 also exceeds the 126 MB L2",
+                   "timing": "CUDA events on the launching stream around each sd_spmm call, summed per step"},
+        "effective_gbs": bytes_all / (ms_per_step * 1e-3) / 1e9,
+        "frac_of_measured_hbm": bytes_all / (ms_per_step * 1e-3) / 1e9 / (peak * world),
+        "wall_ms_per_step_incl_flush": wall_ms,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "GFLOP/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "gpu_launches": int(sum(p["launches"] for p in per) * args.steps),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "per_config": per,
+        "setup_seconds": gen_s,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="sd", choices=["sd", "reference"])
+    ap.add_argument("--configs", default="", help="comma list of config indices (1..4) to restrict the step")
+    ap.add_argument("--small", action="store_true",
+                    help="reduced sizes of the same workloads (dense operands still above the L2 size where "
+                         "the full-size ones are); for profiler captures, not a bench number")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer and CPU-baseline legs")
+    args = ap.parse_args()
+    rank, local_rank, world = dist_env()
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_gpu(args, rank, local_rank, world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -101,7 +101,7 @@ typedef struct {
     int64_t num_segments;   /* MERGE: rows, or (row, window) pairs when windows > 1 */
     int64_t plan_bytes;     /* device memory owned by the plan */
     int32_t sm_count;       /* hardware context read at plan time (Sec. 3.1) */
-    int32_t reserved;
+    int32_t launches;       /* kernel launches one sd_spmm call issues on the vectorised path */
     int64_t l2_bytes;
 } sd_plan_info_t;
 

@@ -41,7 +41,7 @@ class sd_plan_info_t(C.Structure):
                 ("blk_hist", C.c_int64 * 9), ("nnz_dense_blocks", C.c_int64),
                 ("family", C.c_int32), ("dtype", C.c_int32), ("windows", C.c_int32),
                 ("tile_items", C.c_int32), ("num_tiles", C.c_int64), ("num_segments", C.c_int64),
-                ("plan_bytes", C.c_int64), ("sm_count", C.c_int32), ("reserved", C.c_int32),
+                ("plan_bytes", C.c_int64), ("sm_count", C.c_int32), ("launches", C.c_int32),
                 ("l2_bytes", C.c_int64)]
 
     def as_dict(self) -> dict:

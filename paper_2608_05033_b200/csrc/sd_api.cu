@@ -504,6 +504,7 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     } else if (family == SD_BSR_TC) {
         if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
     }
+    info.launches = (family == SD_MERGE && p->M > 0) ? info.windows * (1 + (p->nfix > 0 ? 1 : 0)) : 1;
     info.plan_bytes = p->owned;
     return SD_OK;
 }

@@ -28,17 +28,28 @@ rowsplit_kernel(const SpmmArgs a) {
     // trip counts are made warp-uniform so that the shuffles below are always converged
     const int maxlen = (LPR == 32) ? len : __reduce_max_sync(FULL, len);
 
-    float acc[NV][VW];
+    // two-level accumulation: `acc` takes at most 32*LPR terms before it is folded into
+    // `tot`, so that a very long row is summed in blocks rather than as one running sum
+    float acc[NV][VW], tot[NV][VW];
 #pragma unroll
     for (int v = 0; v < NV; ++v)
 #pragma unroll
-        for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
+        for (int e = 0; e < VW; ++e) acc[v][e] = tot[v][e] = 0.f;
 
     bool colok[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) colok[v] = cbase + (v * LPR + lg) * VW < a.N;
 
     for (int base = 0; base < maxlen; base += LPR) {
+        if (base != 0 && (base / LPR) % 32 == 0) {
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+#pragma unroll
+                for (int e = 0; e < VW; ++e) {
+                    tot[v][e] += acc[v][e];
+                    acc[v][e] = 0.f;
+                }
+        }
         // the group fetches LPR (column, value) pairs with one coalesced load each ...
         int myc = 0;
         float myv = 0.f;
@@ -70,8 +81,11 @@ rowsplit_kernel(const SpmmArgs a) {
     if (row < a.S) {
         float *crow = a.C + row * a.ldc + cbase;
 #pragma unroll
-        for (int v = 0; v < NV; ++v)
-            if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], a.alpha, a.beta, 0);
+        for (int v = 0; v < NV; ++v) {
+#pragma unroll
+            for (int e = 0; e < VW; ++e) tot[v][e] += acc[v][e];
+            if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, tot[v], a.alpha, a.beta, 0);
+        }
     }
 }
 
