@@ -222,15 +222,21 @@ __global__ void merge_table_kernel(const int32_t *__restrict__ ptr, int64_t seg_
     tile_seg[t] = static_cast<int32_t>(seg_begin + lo);
 }
 
-// A tile needs the fix-up pass iff a segment was open at its start and ends inside it.
+// A tile needs the fix-up pass iff a segment was open at its start and ends inside it.  The
+// chain of carry-outs to add starts at the tile holding the segment's first nonzero.
 __global__ void merge_fixflag_kernel(const int32_t *__restrict__ ptr, const int32_t *__restrict__ tile_seg,
-                                     int64_t seg_begin, int32_t tile, int32_t ntiles, uint8_t *__restrict__ flag) {
+                                     int64_t seg_begin, int32_t tile, int32_t ntiles, uint8_t *__restrict__ flag_short,
+                                     uint8_t *__restrict__ flag_long) {
     const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (t >= ntiles) return;
     const int64_t s0 = tile_seg[t], s1 = tile_seg[t + 1];
     const int64_t nzb = ptr[seg_begin];
     const int64_t nz0 = nzb + t * tile - (s0 - seg_begin);
-    flag[t] = (s1 > s0) && (nz0 > ptr[s0]);
+    const bool fix = (s1 > s0) && (nz0 > ptr[s0]);
+    const int64_t ta = ((ptr[s0] - nzb) + (s0 - seg_begin)) / tile;
+    const bool is_long = fix && (t - ta >= kMergeLongChain);
+    flag_short[t] = fix && !is_long;
+    flag_long[t] = is_long;
 }
 
 }  // namespace sd
@@ -249,10 +255,11 @@ struct sd_plan {
 
     // MERGE
     int32_t *tile_seg = nullptr;
-    int32_t *fix_tiles = nullptr;
+    int32_t *fix_short = nullptr;
+    int32_t *fix_long = nullptr;
     float *tile_head = nullptr;
     float *tile_tail = nullptr;
-    int32_t ntiles = 0, nfix = 0;
+    int32_t ntiles = 0, nfix_short = 0, nfix_long = 0;
 
     // BSR
     int32_t *browptr = nullptr;
@@ -314,7 +321,9 @@ static sd_status_t build_merge(sd_plan *p, cudaStream_t st) {
     sd_status_t s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_seg), sizeof(int32_t) * (ntiles + 1), "tile table")))
         return s;
-    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->fix_tiles), sizeof(int32_t) * (ntiles + 1), "fix-up list")))
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->fix_short), sizeof(int32_t) * (ntiles + 1), "fix-up list")))
+        return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->fix_long), sizeof(int32_t) * (ntiles + 1), "fix-up list")))
         return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_head), sizeof(float) * ntiles * p->N, "tile heads")))
         return s;
@@ -323,21 +332,29 @@ static sd_status_t build_merge(sd_plan *p, cudaStream_t st) {
     merge_table_kernel<<<ceil_div(ntiles + 1, 256), 256, 0, st>>>(p->rowptr, 0, p->M, kMergeTile, p->ntiles,
                                                                 p->tile_seg);
     SD_CUDA_TRY(cudaGetLastError());
-    TempBuf flags, nsel, tmp;
-    if ((s = flags.get(ntiles, "fix-up flags"))) return s;
-    if ((s = nsel.get(sizeof(int32_t), "fix-up count"))) return s;
+    TempBuf flags_s, flags_l, nsel, tmp;
+    if ((s = flags_s.get(ntiles, "fix-up flags"))) return s;
+    if ((s = flags_l.get(ntiles, "fix-up flags"))) return s;
+    if ((s = nsel.get(2 * sizeof(int32_t), "fix-up counts"))) return s;
     merge_fixflag_kernel<<<ceil_div(ntiles, 256), 256, 0, st>>>(p->rowptr, p->tile_seg, 0, kMergeTile, p->ntiles,
-                                                               static_cast<uint8_t *>(flags.p));
+                                                               static_cast<uint8_t *>(flags_s.p),
+                                                               static_cast<uint8_t *>(flags_l.p));
     SD_CUDA_TRY(cudaGetLastError());
     size_t tb = 0;
     cub::CountingInputIterator<int32_t> ids(0);
-    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb, ids, static_cast<uint8_t *>(flags.p), p->fix_tiles,
-                                           static_cast<int32_t *>(nsel.p), static_cast<int>(ntiles), st));
+    int32_t *dn = static_cast<int32_t *>(nsel.p);
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb, ids, static_cast<uint8_t *>(flags_s.p), p->fix_short, dn,
+                                           static_cast<int>(ntiles), st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
-    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags.p), p->fix_tiles,
-                                           static_cast<int32_t *>(nsel.p), static_cast<int>(ntiles), st));
-    SD_CUDA_TRY(cudaMemcpyAsync(&p->nfix, nsel.p, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_s.p), p->fix_short, dn,
+                                           static_cast<int>(ntiles), st));
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_l.p), p->fix_long, dn + 1,
+                                           static_cast<int>(ntiles), st));
+    int32_t hn[2] = {0, 0};
+    SD_CUDA_TRY(cudaMemcpyAsync(hn, dn, sizeof hn, cudaMemcpyDeviceToHost, st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));
+    p->nfix_short = hn[0];
+    p->nfix_long = hn[1];
     p->info.tile_items = kMergeTile;
     p->info.num_tiles = ntiles;
     p->info.num_segments = p->M;
@@ -504,7 +521,7 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     } else if (family == SD_BSR_TC) {
         if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
     }
-    info.launches = (family == SD_MERGE && p->M > 0) ? info.windows * (1 + (p->nfix > 0 ? 1 : 0)) : 1;
+    info.launches = (family == SD_MERGE && p->M > 0) ? info.windows * (1 + (p->nfix_short > 0 ? 1 : 0) + (p->nfix_long > 0 ? 1 : 0)) : 1;
     info.plan_bytes = p->owned;
     return SD_OK;
 }
@@ -512,7 +529,8 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
 static void free_plan(sd_plan *p) {
     if (!p) return;
     cudaFree(p->tile_seg);
-    cudaFree(p->fix_tiles);
+    cudaFree(p->fix_short);
+    cudaFree(p->fix_long);
     cudaFree(p->tile_head);
     cudaFree(p->tile_tail);
     cudaFree(p->browptr);
@@ -699,7 +717,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         m.seg_begin = 0;
         m.seg_end = M;
         m.ntiles = plan->ntiles;
-        SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_tiles, plan->nfix, st));
+        SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_short, plan->nfix_short, plan->fix_long, plan->nfix_long, st));
         return SD_OK;
     }
     case SD_BSR_TC: {

@@ -26,9 +26,11 @@ cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st
 // C = beta * C.
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st);
 
-// Family (b): tile kernel, then the carry-out fix-up for the `nfix` tiles listed in fix_tiles.
-cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fix_tiles, int32_t nfix,
-                      cudaStream_t st);
+// Family (b): tile kernel, then the carry-out fix-up for the listed tiles (short chains one per
+// warp, long chains one per CTA).
+cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fix_short, int32_t nshort,
+                      const int32_t *fix_long, int32_t nlong, cudaStream_t st);
+constexpr int kMergeLongChain = 8;   // chains of at least this many tiles go to the per-CTA fix-up
 
 // Family (c).
 struct BsrArgs {

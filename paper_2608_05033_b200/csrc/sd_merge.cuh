@@ -20,32 +20,30 @@ namespace sd {
 constexpr int kMergeThreads = 256;
 constexpr int kMergeEnd = -1;  // column value that marks a segment end in the staged item list
 
-template <typename T, int VW, int LPR, int NV>
+// FULL: every lane's columns are inside N (N is a multiple of the slab width), so the
+// per-vector column tests disappear from the inner loop.
+template <typename T, int VW, int LPR, int NV, bool FULL>
 __global__ void __launch_bounds__(kMergeThreads)
 merge_tile_kernel(const MergeArgs m) {
-    constexpr unsigned FULL = 0xffffffffu;
+    constexpr unsigned FULLMASK = 0xffffffffu;
     constexpr int G = kMergeThreads / LPR;   // groups per tile
-    constexpr int TILE = kMergeTile;         // items per tile
-    constexpr int IPG = TILE / G;            // items per group
-    constexpr int IPT = TILE / kMergeThreads;  // items per thread in the staging scan
+    constexpr int TILE = kMergeTile;         // merged items per tile
+    constexpr int IPG = TILE / G;            // merged items per group
     constexpr int CPL = NV * VW;             // columns per lane
     constexpr int COLS = LPR * CPL;          // columns per CTA slab
     constexpr int CP = COLS + 1;             // padded row pitch of head_s / tail_s
 
-    __shared__ int2 items[TILE];              // (column | kMergeEnd, value bits)
-    __shared__ int32_t ptr_s[TILE + 2];       // ptr[seg0 .. seg0 + ends]
-    __shared__ uint16_t eb_s[TILE];           // ends before item k; bit 15: item k is an end
+    __shared__ int2 nz_s[TILE];               // (column, value bits) of the tile's nonzeros
+    __shared__ int32_t ptr_s[TILE + 2];       // ptr[seg0 .. seg0 + ends + 1]
     __shared__ float head_s[G * CP];
     __shared__ float tail_s[G * CP];
-    __shared__ int32_t warp_cnt[kMergeThreads / 32];
+    __shared__ int32_t gseg_s[G + 1];         // segment coordinate (relative to seg0) of each group start
     __shared__ uint8_t has_end_s[G], open_s[G];
     __shared__ int32_t first_end_s;
 
     const SpmmArgs &a = m.s;
     const T *__restrict__ vals = static_cast<const T *>(a.vals);
-    const T *__restrict__ B = static_cast<const T *>(a.B);
     const int tid = threadIdx.x;
-    const int lane = tid & 31;
     const int t = blockIdx.x;
     const int cbase = blockIdx.y * COLS;
 
@@ -57,66 +55,44 @@ merge_tile_kernel(const MergeArgs m) {
     const int64_t seg1 = __ldg(m.tile_seg + t + 1);
     const int64_t d0 = static_cast<int64_t>(t) * TILE;
     const int count = static_cast<int>(min(static_cast<int64_t>(TILE), total - d0));
-    const int64_t nz0 = nzb + d0 - (seg0 - sb);
     const int ends = static_cast<int>(seg1 - seg0);
+    const int32_t nz0 = static_cast<int32_t>(nzb + d0 - (seg0 - sb));   // first nonzero of the tile
+    const int nnz_t = count - ends;                                       // nonzeros in the tile
 
-    // ---- stage the tile: segment pointers, end markers, merged item list -----------------
-    for (int i = tid; i <= ends; i += kMergeThreads) ptr_s[i] = __ldg(a.ptr + seg0 + i);
-    for (int k = tid; k < TILE; k += kMergeThreads) eb_s[k] = 0;
+    // ---- stage segment pointers and the tile's nonzeros (coalesced) ------------------------
+    for (int i = tid; i <= ends + 1; i += kMergeThreads)
+        ptr_s[i] = __ldg(a.ptr + min(seg0 + i, m.seg_end));
+    for (int k = tid; k < nnz_t; k += kMergeThreads)
+        nz_s[k] = make_int2(__ldg(a.colind + nz0 + k), __float_as_int(to_float(vals[nz0 + k])));
     if (tid == 0) first_end_s = G;
     __syncthreads();
-    // end of segment seg0+e sits at merged position (ptr[seg0+e+1] - nzb) + (seg0+e - sb)
-    for (int e = tid; e < ends; e += kMergeThreads) {
-        const int k = static_cast<int>((ptr_s[e + 1] - nzb) + (seg0 + e - sb) - d0);
-        eb_s[k] = 0x8000u;
-    }
-    __syncthreads();
-    {   // exclusive scan of the end markers: thread -> IPT consecutive items
-        int local = 0;
-        uint16_t f[IPT];
-#pragma unroll
-        for (int i = 0; i < IPT; ++i) {
-            f[i] = eb_s[tid * IPT + i];
-            local += f[i] >> 15;
+
+    // ---- merge-path coordinate of every group start: ends e with (ptr[e+1]-nz0)+e < k -----
+    for (int gi = tid; gi <= G; gi += kMergeThreads) {
+        const int k = min(gi * IPG, count);
+        int lo = 0, hi = ends;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((ptr_s[mid + 1] - nz0) + mid < k) lo = mid + 1;
+            else hi = mid;
         }
-        int incl = local;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int n = __shfl_up_sync(FULL, incl, off);
-            if (lane >= off) incl += n;
-        }
-        if (lane == 31) warp_cnt[tid >> 5] = incl;
-        __syncthreads();
-        int before = incl - local;
-        for (int w = 0; w < (tid >> 5); ++w) before += warp_cnt[w];
-#pragma unroll
-        for (int i = 0; i < IPT; ++i) {
-            eb_s[tid * IPT + i] = static_cast<uint16_t>(before) | f[i];
-            before += f[i] >> 15;
-        }
-    }
-    __syncthreads();
-    for (int k = tid; k < count; k += kMergeThreads) {   // coalesced fill of the item list
-        const uint16_t e = eb_s[k];
-        int2 it;
-        if (e & 0x8000u) {
-            it = make_int2(kMergeEnd, 0);
-        } else {
-            const int64_t j = nz0 + k - e;
-            it = make_int2(__ldg(a.colind + j), __float_as_int(to_float(vals[j])));
-        }
-        items[k] = it;
+        gseg_s[gi] = lo;
     }
     __syncthreads();
 
-    // ---- each group walks its IPG items ----------------------------------------------------
+    // ---- each group walks its slice: whole segments in a tight loop -------------------------
     const int g = tid / LPR;
     const int lg = tid % LPR;
-    const int k0 = g * IPG;
-    const int nit = max(0, min(IPG, count - k0));
+    const int s0 = gseg_s[g], s1 = gseg_s[g + 1];
+    const int j0 = min(g * IPG, count) - s0;          // tile-relative nonzero coordinates
+    const int j1 = min((g + 1) * IPG, count) - s1;
+    const bool open = (nz0 + j0) > ptr_s[s0];         // segment s0 began before this group
+    const bool seen_end = s1 > s0;
+
     bool colok[NV];
 #pragma unroll
-    for (int v = 0; v < NV; ++v) colok[v] = cbase + (v * LPR + lg) * VW < a.N;
+    for (int v = 0; v < NV; ++v) colok[v] = FULL || (cbase + (v * LPR + lg) * VW < a.N);
+    const T *__restrict__ Bl = static_cast<const T *>(a.B) + cbase + lg * VW;   // this lane's columns
 
     float acc[NV][VW];
 #pragma unroll
@@ -124,56 +100,50 @@ merge_tile_kernel(const MergeArgs m) {
 #pragma unroll
         for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
 
-    int seg_off = 0;      // segment index relative to seg0
-    bool open = false;    // the segment at the group's start began before the group
-    bool seen_end = false;
-    if (nit > 0) {
-        seg_off = eb_s[k0] & 0x7FFF;
-        open = (nz0 + k0 - seg_off) > ptr_s[seg_off];
-    }
-    for (int k = 0; k < nit; ++k) {
-        const int2 it = items[k0 + k];
-        if (it.x != kMergeEnd) {
+    int j = j0;
+    for (int s = s0;; ++s) {
+        const int jend = (s < s1) ? (ptr_s[s + 1] - nz0) : j1;
+#pragma unroll 4
+        for (; j < jend; ++j) {
+            const int2 it = nz_s[j];
             const float av = __int_as_float(it.y);
-            const T *brow = B + static_cast<int64_t>(it.x) * a.ldb + cbase;
+            const T *brow = Bl + static_cast<int64_t>(it.x) * a.ldb;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 if (colok[v]) {
                     float b[VW];
-                    RowLoad<T, VW>::ld(brow + (v * LPR + lg) * VW, b);
+                    RowLoad<T, VW>::ld(brow + v * LPR * VW, b);
 #pragma unroll
                     for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(av, b[e], acc[v][e]);
                 }
             }
-        } else {
-            if (open && !seen_end) {
-                // tail end of a segment begun earlier: completed after the scan below
-#pragma unroll
-                for (int v = 0; v < NV; ++v)
-#pragma unroll
-                    for (int e = 0; e < VW; ++e) head_s[g * CP + (v * LPR + lg) * VW + e] = acc[v][e];
-            } else {
-                // the group saw this segment from its first nonzero: finished here
-                const int64_t s = seg0 + seg_off;
-                int64_t row = s;
-                int accumulate = 0;
-                if (a.seg_row) {
-                    const int32_t r = __ldg(a.seg_row + s);
-                    row = r & 0x7FFFFFFF;
-                    accumulate = (r >> 31) & 1;
-                }
-                float *crow = a.C + row * a.ldc + cbase;
-#pragma unroll
-                for (int v = 0; v < NV; ++v)
-                    if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], a.alpha, a.beta, accumulate);
-            }
-            seen_end = true;
-            ++seg_off;
+        }
+        if (s == s1) break;
+        if (s == s0 && open) {
+            // tail end of a segment begun earlier: completed after the combine step below
 #pragma unroll
             for (int v = 0; v < NV; ++v)
 #pragma unroll
-                for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
+                for (int e = 0; e < VW; ++e) head_s[g * CP + (v * LPR + lg) * VW + e] = acc[v][e];
+        } else {
+            // the group saw this segment from its first nonzero: finished here
+            const int64_t sg = seg0 + s;
+            int64_t row = sg;
+            int accumulate = 0;
+            if (a.seg_row) {
+                const int32_t r = __ldg(a.seg_row + sg);
+                row = r & 0x7FFFFFFF;
+                accumulate = (r >> 31) & 1;
+            }
+            float *crow = a.C + row * a.ldc + cbase;
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+                if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], a.alpha, a.beta, accumulate);
         }
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
     }
 #pragma unroll
     for (int v = 0; v < NV; ++v)
@@ -186,40 +156,54 @@ merge_tile_kernel(const MergeArgs m) {
     }
     __syncthreads();
 
-    // ---- segmented scan of the group tails across the tile (warp shuffles) --------------------
+    // ---- combine the group tails across the tile -------------------------------------------------
     // I[g] = (has_end[g] ? 0 : I[g-1]) + tail[g];  carry-in of group g is I[g-1].
-    for (int c = tid >> 5; c < COLS; c += kMergeThreads / 32) {
-        float run = 0.f;
-        for (int ch = 0; ch < G; ch += 32) {
-            const int gg = ch + lane;
-            const bool valid = gg < G;
-            float v = valid ? tail_s[gg * CP + c] : 0.f;
-            int f = valid ? has_end_s[gg] : 0;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const float v2 = __shfl_up_sync(FULL, v, off);
-                const int f2 = __shfl_up_sync(FULL, f, off);
-                if (lane >= off && !f) {
-                    v += v2;
-                    f = f2;
-                }
+    if constexpr (COLS >= 16) {
+        // enough columns to keep the threads busy: one thread per column, groups in order
+        if (tid < COLS) {
+            float run = 0.f;
+#pragma unroll 4
+            for (int gg = 0; gg < G; ++gg) {
+                const float tv = tail_s[gg * CP + tid];
+                tail_s[gg * CP + tid] = run;
+                run = has_end_s[gg] ? tv : run + tv;
             }
-            if (!f) v += run;
-            float ex = __shfl_up_sync(FULL, v, 1);
-            if (lane == 0) ex = run;
-            run = __shfl_sync(FULL, v, 31);
-            if (valid) tail_s[gg * CP + c] = ex;   // now the carry-in of group gg
+            if (cbase + tid < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + tid] = run;
         }
-        // what is still open at the end of the tile goes to the carry-out slot
-        if (lane == 0 && cbase + c < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + c] = run;
+    } else {
+        // few columns, many groups: segmented scan across groups with warp shuffles
+        const int lane = tid & 31;
+        for (int c = tid >> 5; c < COLS; c += kMergeThreads / 32) {
+            float run = 0.f;
+            for (int ch = 0; ch < G; ch += 32) {
+                const int gg = ch + lane;
+                float v = tail_s[gg * CP + c];
+                int f = has_end_s[gg];
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const float v2 = __shfl_up_sync(FULLMASK, v, off);
+                    const int f2 = __shfl_up_sync(FULLMASK, f, off);
+                    if (lane >= off && !f) {
+                        v += v2;
+                        f = f2;
+                    }
+                }
+                if (!f) v += run;
+                float ex = __shfl_up_sync(FULLMASK, v, 1);
+                if (lane == 0) ex = run;
+                run = __shfl_sync(FULLMASK, v, 31);
+                tail_s[gg * CP + c] = ex;   // now the carry-in of group gg
+            }
+            if (lane == 0 && cbase + c < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + c] = run;
+        }
     }
     __syncthreads();
 
     // ---- finish the segments whose tail end a group held -----------------------------------------
-    if (nit > 0 && open && seen_end) {
+    if (open && seen_end) {
         const int first_end = first_end_s;
         const bool tile_open = open_s[0];
-        const int64_t s = seg0 + (eb_s[k0] & 0x7FFF);
+        const int64_t sg = seg0 + s0;
         float r[NV][VW];
 #pragma unroll
         for (int v = 0; v < NV; ++v)
@@ -237,10 +221,10 @@ merge_tile_kernel(const MergeArgs m) {
                     for (int e = 0; e < VW; ++e)
                         m.tile_head[static_cast<int64_t>(t) * a.N + cbase + (v * LPR + lg) * VW + e] = r[v][e];
         } else {
-            int64_t row = s;
+            int64_t row = sg;
             int accumulate = 0;
             if (a.seg_row) {
-                const int32_t rr = __ldg(a.seg_row + s);
+                const int32_t rr = __ldg(a.seg_row + sg);
                 row = rr & 0x7FFFFFFF;
                 accumulate = (rr >> 31) & 1;
             }
@@ -254,33 +238,73 @@ merge_tile_kernel(const MergeArgs m) {
 
 // Fix-up: tile `t` closed a segment that began in an earlier tile.  Its total is the sum of
 // the carry-outs of the tiles since the one holding its first nonzero, plus this tile's head,
-// added in a fixed order (no atomics, so repeated runs give identical bits).
+// added in a fixed order (no atomics, so repeated runs give identical bits).  Chains shorter
+// than kFixLongChain tiles are handled one per warp, longer ones one per CTA.
 constexpr int kFixChains = 8;
+constexpr int kFixLongChain = 8;
+
+struct FixTarget {
+    int64_t row;
+    int accumulate;
+    int ta;   // first tile of the chain
+};
+
+__device__ __forceinline__ FixTarget fix_target(const MergeArgs &m, int t, int32_t tile_items) {
+    const SpmmArgs &a = m.s;
+    const int64_t s = m.tile_seg[t];
+    const int64_t nzb = a.ptr[m.seg_begin];
+    const int64_t first_item = (a.ptr[s] - nzb) + (s - m.seg_begin);
+    FixTarget f;
+    f.ta = static_cast<int>(first_item / tile_items);
+    f.row = s;
+    f.accumulate = 0;
+    if (a.seg_row) {
+        const int32_t rr = a.seg_row[s];
+        f.row = rr & 0x7FFFFFFF;
+        f.accumulate = (rr >> 31) & 1;
+    }
+    return f;
+}
+
+__device__ __forceinline__ void fix_store(const SpmmArgs &a, const FixTarget &f, int c, float tot) {
+    float *p = a.C + f.row * a.ldc + c;
+    float r = a.alpha * tot;
+    if (f.accumulate) r += *p;
+    else if (a.beta != 0.f) r += a.beta * *p;
+    *p = r;
+}
+
+static __global__ void __launch_bounds__(256)
+merge_fixup_short_kernel(const MergeArgs m, const int32_t *__restrict__ fix_tiles, int32_t nfix, int32_t tile_items) {
+    const int f = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (f >= nfix) return;
+    const int lane = threadIdx.x & 31;
+    const int t = fix_tiles[f];
+    const FixTarget ft = fix_target(m, t, tile_items);
+    for (int c = lane; c < m.s.N; c += 32) {
+        float sum = 0.f;
+        for (int tt = ft.ta; tt < t; ++tt) sum += m.tile_tail[static_cast<int64_t>(tt) * m.s.N + c];
+        sum += m.tile_head[static_cast<int64_t>(t) * m.s.N + c];
+        fix_store(m.s, ft, c, sum);
+    }
+}
 
 static __global__ void __launch_bounds__(32 * kFixChains)
-merge_fixup_kernel(const MergeArgs m, const int32_t *__restrict__ fix_tiles, int32_t nfix, int32_t tile_items) {
+merge_fixup_long_kernel(const MergeArgs m, const int32_t *__restrict__ fix_tiles, int32_t nfix, int32_t tile_items) {
     __shared__ float part[kFixChains][33];
     const SpmmArgs &a = m.s;
     const int f = blockIdx.x;
     if (f >= nfix) return;
     const int t = fix_tiles[f];
-    const int64_t s = m.tile_seg[t];
-    const int64_t nzb = a.ptr[m.seg_begin];
-    const int64_t first_item = (a.ptr[s] - nzb) + (s - m.seg_begin);
-    const int ta = static_cast<int>(first_item / tile_items);
-    int64_t row = s;
-    int accumulate = 0;
-    if (a.seg_row) {
-        const int32_t rr = a.seg_row[s];
-        row = rr & 0x7FFFFFFF;
-        accumulate = (rr >> 31) & 1;
-    }
+    const FixTarget ft = fix_target(m, t, tile_items);
     const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
     for (int c0 = 0; c0 < a.N; c0 += 32) {
         const int c = c0 + x;
         float sum = 0.f;
-        if (c < a.N)
-            for (int tt = ta + y; tt < t; tt += kFixChains) sum += m.tile_tail[static_cast<int64_t>(tt) * a.N + c];
+        if (c < a.N) {
+#pragma unroll 4
+            for (int tt = ft.ta + y; tt < t; tt += kFixChains) sum += m.tile_tail[static_cast<int64_t>(tt) * a.N + c];
+        }
         part[y][x] = sum;
         __syncthreads();
         if (y == 0 && c < a.N) {
@@ -288,11 +312,7 @@ merge_fixup_kernel(const MergeArgs m, const int32_t *__restrict__ fix_tiles, int
 #pragma unroll
             for (int q = 1; q < kFixChains; ++q) tot += part[q][x];
             tot += m.tile_head[static_cast<int64_t>(t) * a.N + c];
-            float *p = a.C + row * a.ldc + c;
-            float r = a.alpha * tot;
-            if (accumulate) r += *p;
-            else if (a.beta != 0.f) r += a.beta * *p;
-            *p = r;
+            fix_store(a, ft, c, tot);
         }
         __syncthreads();
     }
@@ -300,23 +320,30 @@ merge_fixup_kernel(const MergeArgs m, const int32_t *__restrict__ fix_tiles, int
 
 template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_merge_one(const MergeArgs &m, cudaStream_t st) {
-    dim3 grid(static_cast<unsigned>(m.ntiles),
-              static_cast<unsigned>((m.s.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
-    merge_tile_kernel<T, VW, LPR, NV><<<grid, kMergeThreads, 0, st>>>(m);
+    constexpr int COLS = LPR * NV * VW;
+    dim3 grid(static_cast<unsigned>(m.ntiles), static_cast<unsigned>((m.s.N + COLS - 1) / COLS));
+    if (m.s.N % COLS == 0) merge_tile_kernel<T, VW, LPR, NV, true><<<grid, kMergeThreads, 0, st>>>(m);
+    else merge_tile_kernel<T, VW, LPR, NV, false><<<grid, kMergeThreads, 0, st>>>(m);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t launch_merge(const MergeArgs &m, bool vec, int lpr, cudaStream_t st) {
+cudaError_t launch_merge(const MergeArgs &m, bool vec, int lpr, int nv, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
-    const int64_t units = (m.s.N + (vec ? VWV : 1) - 1) / (vec ? VWV : 1);
-    const bool wide = units > 32;
-#define SD_MG_CASE(L)                                                                   \
-    case L:                                                                             \
-        if (vec) return (wide && L == 32) ? launch_merge_one<T, VWV, 32, 2>(m, st)      \
-                                          : launch_merge_one<T, VWV, L, 1>(m, st);      \
-        return (wide && L == 32) ? launch_merge_one<T, 1, 32, 4>(m, st)                 \
-                                 : launch_merge_one<T, 1, L, 1>(m, st);
+    if (vec && nv == 2) {
+        switch (lpr) {
+        case 4: return launch_merge_one<T, VWV, 4, 2>(m, st);
+        case 8: return launch_merge_one<T, VWV, 8, 2>(m, st);
+        case 16: return launch_merge_one<T, VWV, 16, 2>(m, st);
+        case 32: return launch_merge_one<T, VWV, 32, 2>(m, st);
+        }
+        return cudaErrorInvalidValue;
+    }
+#define SD_MG_CASE(L)                                                \
+    case L:                                                          \
+        if (vec) return launch_merge_one<T, VWV, L, 1>(m, st);       \
+        return (nv == 4) ? launch_merge_one<T, 1, 32, 4>(m, st)      \
+                         : launch_merge_one<T, 1, L, 1>(m, st);
     switch (lpr) {
         SD_MG_CASE(1)
         SD_MG_CASE(2)

@@ -4,6 +4,8 @@
 // row, several outputs per thread in registers, shuffles share the sparse entries).
 #pragma once
 
+#include <cstdlib>
+
 #include "sd_common.cuh"
 
 namespace sd {
@@ -39,6 +41,26 @@ rowsplit_kernel(const SpmmArgs a) {
     bool colok[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) colok[v] = cbase + (v * LPR + lg) * VW < a.N;
+
+    // beta != 0: fetch the old C row now so that its latency hides behind the gathers
+    float cin[NV][VW];
+    if (a.beta != 0.f && row < a.S) {
+        const float *crow = a.C + row * a.ldc + cbase;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            if (colok[v]) {
+                if constexpr (VW == 1) {
+                    cin[v][0] = crow[(v * LPR + lg)];
+                } else {
+#pragma unroll
+                    for (int q = 0; q < VW / 4; ++q) {
+                        const float4 o = *(reinterpret_cast<const float4 *>(crow + (v * LPR + lg) * VW) + q);
+                        cin[v][4 * q] = o.x; cin[v][4 * q + 1] = o.y; cin[v][4 * q + 2] = o.z; cin[v][4 * q + 3] = o.w;
+                    }
+                }
+            }
+        }
+    }
 
     for (int base = 0; base < maxlen; base += LPR) {
         if (base != 0 && (base / LPR) % 32 == 0) {
@@ -83,8 +105,11 @@ rowsplit_kernel(const SpmmArgs a) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
 #pragma unroll
-            for (int e = 0; e < VW; ++e) tot[v][e] += acc[v][e];
-            if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, tot[v], a.alpha, a.beta, 0);
+            for (int e = 0; e < VW; ++e) {
+                tot[v][e] = a.alpha * (tot[v][e] + acc[v][e]);
+                if (a.beta != 0.f) tot[v][e] = fmaf(a.beta, cin[v][e], tot[v][e]);
+            }
+            if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, tot[v], 1.f, 0.f, 0);
         }
     }
 }
@@ -110,17 +135,35 @@ cudaError_t launch_rowsplit_one(const SpmmArgs &a, cudaStream_t st) {
 
 // Lane geometry for a dense width: VW elements per 16-byte load when `vec`, LPR lanes per
 // row (a power of two), NV vectors per lane; wider rows are covered by grid.y slabs.
+// Two vectors per lane (when the row has at least 8 vectors) halve the per-nonzero
+// instruction overhead -- index broadcast, address arithmetic -- per byte gathered.
 struct LaneGeom {
     int vw, lpr, nv;
 };
+inline int geom_nv_override() {
+    static const int v = [] {
+        const char *e = getenv("SD_GEOM_NV");   // bench-only switch: 1 forces one vector per lane
+        return e ? atoi(e) : 0;
+    }();
+    return v;
+}
 inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw) {
     LaneGeom g;
     g.vw = vec ? vecw : 1;
-    int64_t units = (N + g.vw - 1) / g.vw;
+    const int64_t units = (N + g.vw - 1) / g.vw;
+    if (!vec) {
+        int lpr = 1;
+        while (lpr < 32 && lpr < units) lpr <<= 1;
+        g.lpr = lpr;
+        g.nv = units > 32 ? 4 : 1;
+        return g;
+    }
+    const bool two = units >= 8 && geom_nv_override() != 1;
+    const int64_t per = two ? (units + 1) / 2 : units;
     int lpr = 1;
-    while (lpr < 32 && lpr < units) lpr <<= 1;
+    while (lpr < 32 && lpr < per) lpr <<= 1;
     g.lpr = lpr;
-    g.nv = (units > 32) ? (vec ? 2 : 4) : 1;
+    g.nv = (two || units > 32) ? 2 : 1;
     return g;
 }
 
@@ -128,11 +171,19 @@ template <typename T>
 cudaError_t launch_rowsplit(const SpmmArgs &a, bool vec, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
     const LaneGeom g = lane_geometry(a.N, vec, VWV);
-#define SD_RS_CASE(L)                                                                  \
-    case L:                                                                            \
-        if (vec) return (g.nv == 2) ? launch_rowsplit_one<T, VWV, 32, 2>(a, st)        \
-                                    : launch_rowsplit_one<T, VWV, L, 1>(a, st);        \
-        return (g.nv == 4) ? launch_rowsplit_one<T, 1, 32, 4>(a, st)                   \
+    if (vec && g.nv == 2) {
+        switch (g.lpr) {
+        case 4: return launch_rowsplit_one<T, VWV, 4, 2>(a, st);
+        case 8: return launch_rowsplit_one<T, VWV, 8, 2>(a, st);
+        case 16: return launch_rowsplit_one<T, VWV, 16, 2>(a, st);
+        case 32: return launch_rowsplit_one<T, VWV, 32, 2>(a, st);
+        }
+        return cudaErrorInvalidValue;
+    }
+#define SD_RS_CASE(L)                                                  \
+    case L:                                                            \
+        if (vec) return launch_rowsplit_one<T, VWV, L, 1>(a, st);      \
+        return (g.nv == 4) ? launch_rowsplit_one<T, 1, 32, 4>(a, st)   \
                            : launch_rowsplit_one<T, 1, L, 1>(a, st);
     switch (g.lpr) {
         SD_RS_CASE(1)
