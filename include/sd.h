@@ -161,6 +161,13 @@ sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bc
  * pointer array.  SD_ERR_UNSUPPORTED for other families. */
 sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t cap, int64_t *count);
 
+/* sd_plan_device_status -- every wait inside the library's kernels (mbarrier waits of the
+ * tensor-core kernel) is bounded; a wait that runs out makes its CTA record a non-zero code
+ * in a plan-owned device word, release its resources and return, so the context stays
+ * usable but C is then incomplete.  This call synchronises the device, copies the word to
+ * *status (0 = no wait ever expired) and clears it. */
+sd_status_t sd_plan_device_status(sd_plan_t *plan, int32_t *status);
+
 /* sd_last_error -- copy the calling thread's last error text into buf (NUL-terminated,
  * at most n bytes); returns the last status code. */
 int sd_last_error(char *buf, size_t n);

@@ -22,7 +22,8 @@ SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_last_error", "sd_version"]
+           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_device_status", "sd_last_error",
+           "sd_version"]
 
 
 class sd_plan_desc_t(C.Structure):
@@ -81,6 +82,8 @@ def load():
     lib.sd_plan_get_bsr.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_get_tiles.restype = C.c_int
     lib.sd_plan_get_tiles.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
+    lib.sd_plan_device_status.restype = C.c_int
+    lib.sd_plan_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     lib.sd_last_error.restype = C.c_int
     lib.sd_last_error.argtypes = [C.c_char_p, C.c_size_t]
     lib.sd_version.restype = C.c_char_p
@@ -179,6 +182,14 @@ def sd_plan_get_bsr(plan):
     return browptr, bcol, bval
 
 
+def sd_plan_device_status(plan) -> int:
+    st = C.c_int32(0)
+    rc = load().sd_plan_device_status(plan, C.byref(st))
+    if rc != SD_OK:
+        _raise(rc)
+    return st.value
+
+
 def sd_plan_get_tiles(plan) -> np.ndarray:
     n = C.c_int64(0)
     rc = load().sd_plan_get_tiles(plan, None, 0, C.byref(n))
@@ -213,6 +224,9 @@ class Plan:
         ldc = C_host.strides[0] // C_host.itemsize if isinstance(C_host, np.ndarray) else C_host.stride(0)
         sd_spmm_host(self.handle, B_host, ldb, C_host, ldc, alpha, beta)
         return C_host
+
+    def device_status(self) -> int:
+        return sd_plan_device_status(self.handle)
 
     def info(self) -> sd_plan_info_t:
         return sd_plan_get_info(self.handle)

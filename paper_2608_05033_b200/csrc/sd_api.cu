@@ -2,6 +2,7 @@
 // build), execution dispatch, teardown.  See include/sd.h for the contract.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -265,6 +266,8 @@ struct sd_plan {
     int32_t *browptr = nullptr;
     int32_t *bcol = nullptr;
     void *bval = nullptr;
+    void *bval_mma = nullptr;   // tensor-core operand images of the blocks
+    int32_t *dev_error = nullptr;
     int64_t nnzb = 0;
 
     // host-buffer entry point
@@ -383,6 +386,12 @@ static sd_status_t build_bsr(sd_plan *p, const unsigned long long *ukeys, int64_
     bsr_bcol_kernel<<<ceil_div(nnzb, 256), 256, 0, st>>>(ukeys, nnzb, Kb, p->bcol);
     SD_CUDA_TRY(cudaGetLastError());
     SD_CUDA_TRY(p->dtype == SD_F32 ? fill_bsr<float>(p, st) : fill_bsr<__nv_bfloat16>(p, st));
+    if (p->dtype == SD_BF16) {
+        if ((s = dev_alloc(p, &p->bval_mma, es * 256 * nnzb, "bval (tensor-core image)"))) return s;
+        SD_CUDA_TRY(build_bsr_mma_image(p->bval, p->bval_mma, nnzb, p->dtype, st));
+    }
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->dev_error), sizeof(int32_t), "error word"))) return s;
+    SD_CUDA_TRY(cudaMemsetAsync(p->dev_error, 0, sizeof(int32_t), st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));
     return SD_OK;
 }
@@ -536,6 +545,8 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->browptr);
     cudaFree(p->bcol);
     cudaFree(p->bval);
+    cudaFree(p->bval_mma);
+    cudaFree(p->dev_error);
     cudaFree(p->stage_B);
     cudaFree(p->stage_C);
     if (p->host_stream) cudaStreamDestroy(p->host_stream);
@@ -650,6 +661,20 @@ sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bc
     return SD_OK;
 }
 
+sd_status_t sd_plan_device_status(sd_plan_t *plan, int32_t *status) {
+    if (!plan || !status) {
+        set_error(SD_ERR_INVALID_ARG, "plan and status must not be null");
+        return SD_ERR_INVALID_ARG;
+    }
+    *status = 0;
+    SD_CUDA_TRY(cudaDeviceSynchronize());
+    if (plan->dev_error) {
+        SD_CUDA_TRY(cudaMemcpy(status, plan->dev_error, sizeof(int32_t), cudaMemcpyDeviceToHost));
+        if (*status) SD_CUDA_TRY(cudaMemset(plan->dev_error, 0, sizeof(int32_t)));
+    }
+    return SD_OK;
+}
+
 sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t cap, int64_t *count) {
     if (!plan || !count) {
         set_error(SD_ERR_INVALID_ARG, "plan and count must not be null");
@@ -725,7 +750,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         b.browptr = plan->browptr;
         b.bcol = plan->bcol;
         b.bval = plan->bval;
-        b.bval_mma = nullptr;
+        b.bval_mma = plan->bval_mma;
         b.B = B;
         b.C = C;
         b.ldb = ldb;
@@ -738,7 +763,10 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         b.beta = beta;
         const bool vec4 = aligned16(B) && aligned16(C) && N % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
                           (plan->dtype == SD_F32 || (reinterpret_cast<uintptr_t>(B) & 7u) == 0);
-        SD_CUDA_TRY(run_bsr_simt(b, plan->dtype, vec4, st));
+        if (bsr_tc_usable(b, plan->dtype) && !getenv("SD_BSR_SIMT"))
+            SD_CUDA_TRY(run_bsr_tc(b, plan->dtype, plan->dev_error, plan->info.sm_count, st));
+        else
+            SD_CUDA_TRY(run_bsr_simt(b, plan->dtype, vec4, st));
         return SD_OK;
     }
     default:

@@ -47,5 +47,9 @@ struct BsrArgs {
     float alpha, beta;
 };
 cudaError_t run_bsr_simt(const BsrArgs &a, int dtype, bool vec, cudaStream_t st);
+// Tensor-core form.  bsr_tc_usable: dtype, dense width and the TMA alignment rules allow it.
+bool bsr_tc_usable(const BsrArgs &a, int dtype);
+cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_count, cudaStream_t st);
+cudaError_t build_bsr_mma_image(const void *bval, void *img, int64_t nnzb, int dtype, cudaStream_t st);
 
 }  // namespace sd

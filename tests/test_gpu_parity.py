@@ -310,3 +310,42 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     plan.spmm_host(Bh, Ch, 0.5, 2.0)
     check(w2, Ch.numpy(), c_in=Cin, alpha=0.5, beta=2.0)
     plan.close()
+
+
+@pytest.mark.parametrize("N", [64, 128, 192, 256, 320, 512])
+@pytest.mark.parametrize("beta", [0.0, -0.75])
+def test_bsr_tensor_core_path_bf16(N, beta):
+    # bf16 blocks on the tcgen05 path: ragged M and K, empty block-rows, partially filled blocks,
+    # padded leading dimensions (kept multiples of 8 so that the TMA alignment rules hold)
+    rng = np.random.default_rng(N)
+    M, K = 16 * 37 + 5, 16 * 29 + 11
+    lengths = np.clip(rng.poisson(30, M), 0, K)
+    lengths[32:64] = 0        # two empty block-rows
+    w = W.random_csr(M, K, N, lengths, seed=N + 1, dtype=W.SD_BF16, alpha=1.5, beta=beta)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_BSR_TC)
+    for pad_b, pad_c in [(0, 0), (8, 3)]:
+        got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_c)
+        assert plan.device_status() == 0
+        assert intact
+        check(w, got)
+    got2, _ = run_spmm(plan, w, pad_b=8, pad_c=3)
+    assert np.array_equal(got, got2)
+    plan.close()
+
+
+def test_bsr_tensor_core_dense_blocks_bf16_exact_products():
+    # fully dense blocks, small integers: every product and partial sum is exact in fp32, so the
+    # tensor-core result must equal the oracle bit for bit
+    w = W.g4_block(Mb=96, Kb=80, N=256, nblocks=700, seed=5, dtype=W.SD_BF16)
+    rng = np.random.default_rng(1)
+    w.vals = W.f32_to_bf16_bits(rng.integers(-4, 5, w.vals.shape).astype(np.float32))
+    w.B = W.f32_to_bf16_bits(rng.integers(-4, 5, w.B.shape).astype(np.float32)).reshape(w.B.shape)
+    dw = DeviceWorkload(w)
+    plan = dw.plan()
+    assert plan.info().family == sd.SD_BSR_TC
+    got, _ = run_spmm(plan, w)
+    assert plan.device_status() == 0
+    ref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
+    assert np.array_equal(got.astype(np.float64), ref)
+    plan.close()
