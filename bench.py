@@ -252,7 +252,7 @@ def run_gpu(args, rank, local_rank, world):
             w.B = Bf if dt == W.SD_F32 else W.f32_to_bf16_bits(Bf).reshape(w.K, w.N)
         rowptr, colind, vals = to_dev(w.rowptr), to_dev(w.colind), to_dev(w.vals)
         t0 = time.time()
-        plan = sd.Plan(rowptr, colind, vals, w.M, w.K, w.N, dtype=w.dtype)
+        plan = sd.Plan(rowptr, colind, vals, w.M, w.K, w.N, dtype=w.dtype, windows=args.windows)
         torch.cuda.synchronize()
         plan_ms = (time.time() - t0) * 1e3
         Bd = to_dev(w.B)
@@ -345,7 +345,7 @@ def run_gpu(args, rank, local_rank, world):
                     "nnz": w.nnz, "ms": ms, "ms_min": float(np.min(c["times"])),
                     "gflops": w.flops() / (ms * 1e-3) / 1e9, "compulsory_bytes": w.compulsory_bytes(),
                     "effective_gbs": gbs, "frac_of_measured_hbm": gbs / peak,
-                    "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS, "launches": int(info.launches),
+                    "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS, "launches": int(info.launches), "windows": int(info.windows),
                     "plan_ms": c["plan_ms"], "plan_bytes": int(info.plan_bytes)})
     dom = max(per, key=lambda p: p["ms"])
     roofline = {"bound": "hbm", "kernel": dom["family"] + " on " + dom["workload"],
@@ -397,6 +397,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="sd", choices=["sd", "reference"])
     ap.add_argument("--configs", default="", help="comma list of config indices (1..4) to restrict the step")
+    ap.add_argument("--windows", type=int, default=0, help="column windows of the merge family (0 = plan's rule)")
     ap.add_argument("--small", action="store_true",
                     help="reduced sizes of the same workloads (dense operands still above the L2 size where "
                          "the full-size ones are); for profiler captures, not a bench number")

@@ -129,7 +129,9 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
  * get beta*C.  Asynchronous: launches only, no allocation, no synchronisation.
  * 16-byte aligned B/C with N, ldb, ldc multiples of the vector width take the
  * vectorised kernels; anything else takes scalar kernels (never an error).
- * A plan must not run concurrently on two streams (it owns carry-out scratch).
+ * With column windows the call issues one kernel sequence per window, in order, and C is
+ * updated window by window.  A plan must not run concurrently on two streams (it owns
+ * carry-out scratch).
  * Results are run-to-run bit-identical (no floating-point atomics). */
 sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc,
                     float alpha, float beta, void *stream);
@@ -153,13 +155,29 @@ sd_status_t sd_plan_get_info(const sd_plan_t *plan, sd_plan_info_t *out);
  * be NULL to skip it.  SD_ERR_UNSUPPORTED if the plan's family is not SD_BSR_TC. */
 sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bcol, void *bval);
 
-/* sd_plan_get_tiles -- MERGE family: copy merge-path tile start coordinates to a HOST
- * array.  tile_seg[t] = number of segment ends among the first t*tile_items merged
- * items of window w, for t = 0..ntiles_w, windows concatenated; `cap` is the capacity
- * of tile_seg in elements and *count receives the number written (or needed).
- * seg_ptr (optional, capacity num_segments + windows) receives each window's segment
- * pointer array.  SD_ERR_UNSUPPORTED for other families. */
+/* sd_plan_get_tiles -- MERGE family: copy the merge-path tile start coordinates to a HOST
+ * array.  For window w (w = 0 when the plan uses no column windows) the merged list
+ * interleaves the ends of that window's segments with its nonzeros; table entry t is the
+ * (global) index of the first segment whose end lies at or after merged position
+ * t * tile_items.  Window w owns ntiles_w + 1 consecutive entries and the windows are
+ * concatenated.  `cap` is the capacity of tile_seg in elements; *count receives the number
+ * of entries (also when tile_seg is NULL or too small).  SD_ERR_UNSUPPORTED for other
+ * families. */
 sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t cap, int64_t *count);
+
+/* sd_plan_get_segments -- MERGE family with column windows (the paper's "packed column
+ * windows", Sec. 3.4): copy the window-major representation to HOST arrays.  The columns are
+ * cut into `windows` ranges of ceil(K / windows) columns; a segment is the part of one row
+ * that falls into one window; segments are ordered by (window, row), except that the empty
+ * rows come first as zero-length segments of window 0.
+ *   seg_ptr  int32 [num_segments + 1]  start of each segment in the re-bucketed arrays
+ *   seg_row  int32 [num_segments]      output row; bit 31 set when an earlier window already
+ *                                      wrote the row (this segment then adds to C)
+ *   colind   int32 [nnz], vals [nnz]   nonzeros in window-major order (plan dtype)
+ *   win_seg  int64 [windows + 1]       first segment of each window
+ * Any pointer may be NULL.  SD_ERR_UNSUPPORTED when the plan has no windows. */
+sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_t *seg_row, int32_t *colind,
+                                 void *vals, int64_t *win_seg);
 
 /* sd_plan_device_status -- every wait inside the library's kernels (mbarrier waits of the
  * tensor-core kernel) is bounded; a wait that runs out makes its CTA record a non-zero code

@@ -65,6 +65,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.sdo_bsr16_count.restype = C.c_int64
+        _lib.sdo_window_segments.restype = C.c_int64
     return _lib
 
 
@@ -191,6 +192,25 @@ def summary(rowptr, colind, M, K, N) -> Info:
 def decide(info: Info) -> int:
     """O4: family rule on the integers of O3 (parity unpinned: thresholds are not in the paper)."""
     return int(lib().sdo_decide(C.byref(info)))
+
+
+def decide_windows(info: Info, dtype: int, l2_bytes: int) -> int:
+    """O4: number of column windows of the merge family (parity unpinned: this build's rule)."""
+    return int(lib().sdo_decide_windows(C.byref(info), C.c_int(dtype), C.c_int64(l2_bytes)))
+
+
+def window_segments(rowptr, colind, M, K, W):
+    """O4: window-major segment list.  Returns (seg_ptr, seg_row, perm, win_seg)."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    colind = np.ascontiguousarray(colind, dtype=np.int32)
+    nnz = int(rowptr[-1])
+    seg_ptr = np.zeros(nnz + M + 1, np.int32)
+    seg_row = np.zeros(nnz + M, np.int32)
+    perm = np.zeros(max(nnz, 1), np.int32)
+    win_seg = np.zeros(W + 1, np.int64)
+    S = int(lib().sdo_window_segments(C.c_int64(M), C.c_int64(K), _p(rowptr), _p(colind), C.c_int32(W),
+                                      _p(seg_ptr), _p(seg_row), _p(perm), _p(win_seg)))
+    return seg_ptr[:S + 1].copy(), seg_row[:S].copy(), perm[:nnz].copy(), win_seg
 
 
 def hist_bin(v: int) -> int:

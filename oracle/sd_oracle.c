@@ -433,3 +433,61 @@ int sdo_merge_coords(int64_t S, const int32_t *ptr, int64_t items, int64_t ntile
     }
     return t == ntiles + 1 ? 0 : 1;
 }
+
+/* Column-window count (this build's rule; the paper names "packed column windows" for SpMM in
+ * Sec. 3.4 without a rule).  parity unpinned.  No windows unless the rows are short on average
+ * (nnz < 16 M), sorted, and B exceeds 60 % of L2; then the smallest power of two that makes
+ * one window's slab of B fit in that budget. */
+int sdo_decide_windows(const sdo_info_t *o, int dtype, int64_t l2_bytes)
+{
+    int64_t es = dtype == SDO_F32 ? 4 : 2;
+    int64_t bbytes = o->K * o->N * es;
+    int64_t budget = l2_bytes / 10 * 6;
+    if (o->unsorted_rows != 0 || o->nnz >= 16 * o->M || budget <= 0 || bbytes <= budget)
+        return 1;
+    int w = 1;
+    while (w < 64 && bbytes > budget * w)
+        w <<= 1;
+    return w;
+}
+
+/* Window-major segment list.  Window of a column: col / ceil(K / W).  A segment is the part
+ * of one row inside one window.  Order: the empty rows first (zero-length segments, window
+ * 0), then for w = 0..W-1, for ascending row, the row's nonzeros of window w in storage
+ * order.  seg_row carries bit 31 when the row's first nonzero lies in an earlier window
+ * (columns are ascending), i.e. when an earlier segment already wrote the row.
+ * perm[q] = original position of the q-th re-bucketed nonzero.  Returns the segment count;
+ * seg_ptr needs room for nnz + M + 1 entries, seg_row for nnz + M, win_seg for W + 1. */
+int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const int32_t *colind,
+                            int32_t W, int32_t *seg_ptr, int32_t *seg_row, int32_t *perm,
+                            int64_t *win_seg)
+{
+    int64_t wcols = (K + W - 1) / W, S = 0, q = 0;
+    for (int64_t i = 0; i < M; ++i)
+        if (rowptr[i + 1] == rowptr[i]) {
+            seg_ptr[S] = 0;
+            seg_row[S] = (int32_t)i;
+            ++S;
+        }
+    for (int32_t w = 0; w < W; ++w) {
+        win_seg[w] = (w == 0) ? 0 : S;
+        for (int64_t i = 0; i < M; ++i) {
+            int started = 0;
+            for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                if (colind[p] / wcols != w)
+                    continue;
+                if (!started) {
+                    int64_t first_w = colind[rowptr[i]] / wcols;
+                    seg_ptr[S] = (int32_t)q;
+                    seg_row[S] = (int32_t)i | (first_w != w ? (int32_t)0x80000000u : 0);
+                    ++S;
+                    started = 1;
+                }
+                perm[q++] = (int32_t)p;
+            }
+        }
+    }
+    win_seg[W] = S;
+    seg_ptr[S] = (int32_t)q;
+    return S;
+}

@@ -22,7 +22,7 @@ SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_device_status", "sd_last_error",
+           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_last_error",
            "sd_version"]
 
 
@@ -82,6 +82,8 @@ def load():
     lib.sd_plan_get_bsr.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_get_tiles.restype = C.c_int
     lib.sd_plan_get_tiles.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
+    lib.sd_plan_get_segments.restype = C.c_int
+    lib.sd_plan_get_segments.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_device_status.restype = C.c_int
     lib.sd_plan_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     lib.sd_last_error.restype = C.c_int
@@ -180,6 +182,22 @@ def sd_plan_get_bsr(plan):
     if rc != SD_OK:
         _raise(rc)
     return browptr, bcol, bval
+
+
+def sd_plan_get_segments(plan):
+    """Returns (seg_ptr, seg_row, colind, vals, win_seg) of a plan with column windows."""
+    info = sd_plan_get_info(plan)
+    S, nnz, W = info.num_segments, info.nnz, info.windows
+    seg_ptr = np.zeros(S + 1, np.int32)
+    seg_row = np.zeros(S, np.int32)
+    colind = np.zeros(nnz, np.int32)
+    vals = np.zeros(nnz, np.float32 if info.dtype == SD_F32 else np.uint16)
+    win_seg = np.zeros(W + 1, np.int64)
+    rc = load().sd_plan_get_segments(plan, seg_ptr.ctypes.data, seg_row.ctypes.data, colind.ctypes.data,
+                                     vals.ctypes.data, win_seg.ctypes.data)
+    if rc != SD_OK:
+        _raise(rc)
+    return seg_ptr, seg_row, colind, vals, win_seg
 
 
 def sd_plan_device_status(plan) -> int:

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include <cub/cub.cuh>
 
@@ -240,6 +241,88 @@ __global__ void merge_fixflag_kernel(const int32_t *__restrict__ ptr, const int3
     flag_long[t] = is_long;
 }
 
+// ---- column windows (the paper's "packed column windows" for SpMM, Sec. 3.4) ------------------
+// The column range is cut into W windows of wcols columns.  Nonzeros are re-bucketed by window
+// (stable, so rows stay ascending inside a window); a segment is the run of one row inside one
+// window.  Windows are executed one after the other, so the slab of B a window touches can stay
+// in L2 while every nonzero of that window is processed.
+__global__ void __launch_bounds__(256)
+window_keys_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, int64_t M, int32_t wcols,
+                   uint32_t *__restrict__ wkey, int32_t *__restrict__ rowid) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t row = warp0; row < M; row += nwarps)
+        for (int p = rowptr[row] + lane; p < rowptr[row + 1]; p += 32) {
+            wkey[p] = static_cast<uint32_t>(colind[p] / wcols);
+            rowid[p] = static_cast<int32_t>(row);
+        }
+}
+
+template <typename T>
+__global__ void window_gather_kernel(const int32_t *__restrict__ perm, const int32_t *__restrict__ colind,
+                                     const T *__restrict__ vals, const int32_t *__restrict__ rowid, int64_t nnz,
+                                     int32_t *__restrict__ w_col, T *__restrict__ w_val, int32_t *__restrict__ w_row) {
+    const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (q >= nnz) return;
+    const int32_t p = perm[q];
+    w_col[q] = colind[p];
+    w_val[q] = vals[p];
+    w_row[q] = rowid[p];
+}
+
+__global__ void window_headflag_kernel(const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ w_row,
+                                       int64_t nnz, uint8_t *__restrict__ flag) {
+    const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (q >= nnz) return;
+    flag[q] = (q == 0) || (w_row[q] != w_row[q - 1]) || (wkey_sorted[q] != wkey_sorted[q - 1]);
+}
+
+__global__ void window_emptyflag_kernel(const int32_t *__restrict__ rowptr, int64_t M, uint8_t *__restrict__ flag) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < M) flag[i] = rowptr[i + 1] == rowptr[i];
+}
+
+// seg_ptr[0..E) = 0 for the empty rows (their ids are already in seg_row[0..E)); for the other
+// segments the output row and the "row already written by an earlier window" bit.
+__global__ void window_segrow_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind,
+                                     const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ w_row,
+                                     int32_t wcols, int64_t E, int64_t S, int64_t nnz, int32_t *__restrict__ seg_ptr,
+                                     int32_t *__restrict__ seg_row) {
+    const int64_t s = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (s > S) return;
+    if (s == S) {
+        seg_ptr[S] = static_cast<int32_t>(nnz);
+        return;
+    }
+    if (s < E) {
+        seg_ptr[s] = 0;
+        return;
+    }
+    const int32_t q = seg_ptr[s];
+    const int32_t row = w_row[q];
+    const uint32_t first_win = static_cast<uint32_t>(colind[rowptr[row]] / wcols);
+    seg_row[s] = row | (wkey_sorted[q] != first_win ? static_cast<int32_t>(0x80000000u) : 0);
+}
+
+// win_seg[w] = first segment whose window is >= w (empty rows belong to window 0).
+__global__ void window_bounds_kernel(const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ seg_ptr,
+                                     int64_t E, int64_t S, int32_t W, int64_t *__restrict__ win_seg) {
+    const int w = threadIdx.x;
+    if (w > W) return;
+    if (w == 0) {
+        win_seg[0] = 0;
+        return;
+    }
+    int64_t lo = E, hi = S;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (wkey_sorted[seg_ptr[mid]] < static_cast<uint32_t>(w)) lo = mid + 1;
+        else hi = mid;
+    }
+    win_seg[w] = lo;
+}
+
 }  // namespace sd
 
 // =====================================================================================
@@ -254,13 +337,28 @@ struct sd_plan {
     int device = 0;
     sd_plan_info_t info{};
 
-    // MERGE
+    // MERGE: segment arrays the kernels read (the caller's CSR when windows == 1)
+    const int32_t *m_ptr = nullptr;
+    const int32_t *m_col = nullptr;
+    const void *m_vals = nullptr;
+    const int32_t *m_seg_row = nullptr;
+    int32_t *w_ptr = nullptr;      // plan-owned when windows > 1
+    int32_t *w_col = nullptr;
+    void *w_vals = nullptr;
+    int32_t *w_seg_row = nullptr;
+    int64_t num_segments = 0;
+    struct Window {
+        int64_t seg_begin, seg_end;
+        int64_t tile_base;         // first tile of the window in the concatenated tile numbering
+        int32_t ntiles, nshort, nlong;
+    };
+    std::vector<Window> wins;
     int32_t *tile_seg = nullptr;
     int32_t *fix_short = nullptr;
     int32_t *fix_long = nullptr;
     float *tile_head = nullptr;
     float *tile_tail = nullptr;
-    int32_t ntiles = 0, nfix_short = 0, nfix_long = 0;
+    int64_t ntiles = 0;
 
     // BSR
     int32_t *browptr = nullptr;
@@ -313,16 +411,167 @@ static int decide_family(const sd_plan_info_t &s) {
     return skew ? SD_MERGE : SD_ROWSPLIT;
 }
 
-static sd_status_t build_merge(sd_plan *p, cudaStream_t st) {
-    const int64_t total = p->M + p->nnz;
-    const int64_t ntiles = (total + kMergeTile - 1) / kMergeTile;
-    if (ntiles > INT32_MAX - 1) {
+// Number of column windows: none unless the rows are short on average (nnz < 16 M, so the
+// extra read-modify-write of C per (row, window) pair stays below the gather traffic saved),
+// the columns are sorted, and B does not fit in 60 % of L2; then the smallest power of two
+// that makes one window's slab of B fit.
+static int decide_windows(const sd_plan_info_t &s, int dtype) {
+    const int64_t es = dtype == SD_F32 ? 4 : 2;
+    const int64_t bbytes = s.K * s.N * es;
+    const int64_t budget = s.l2_bytes / 10 * 6;
+    if (s.unsorted_rows != 0 || s.nnz >= 16 * s.M || budget <= 0 || bbytes <= budget) return 1;
+    int w = 1;
+    while (w < 64 && bbytes > budget * w) w <<= 1;
+    return w;
+}
+
+__global__ void iota_kernel(int32_t *out, int64_t n) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = static_cast<int32_t>(i);
+}
+
+template <typename T>
+static cudaError_t launch_window_gather(const int32_t *perm, sd_plan *p, const int32_t *rowid, int32_t *w_row,
+                                        cudaStream_t st) {
+    window_gather_kernel<T><<<ceil_div(p->nnz, 256), 256, 0, st>>>(perm, p->colind, static_cast<const T *>(p->vals), rowid,
+                                                                  p->nnz, p->w_col, static_cast<T *>(p->w_vals), w_row);
+    return cudaGetLastError();
+}
+
+// Re-buckets the nonzeros by column window and builds the (row, window) segment list.
+static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &win_seg, cudaStream_t st) {
+    const int64_t nnz = p->nnz, M = p->M;
+    const int32_t wcols = static_cast<int32_t>((p->K + W - 1) / W);
+    const size_t es = p->dtype == SD_F32 ? 4 : 2;
+    const int64_t E = p->info.empty_rows;
+    sd_status_t s;
+    TempBuf wkey, wkey_sorted, rowid, w_row, ids, perm, tmp, flag, nsel, dwin;
+    if ((s = wkey.get(4 * nnz, "window keys"))) return s;
+    if ((s = wkey_sorted.get(4 * nnz, "window keys"))) return s;
+    if ((s = rowid.get(4 * nnz, "row ids"))) return s;
+    if ((s = w_row.get(4 * nnz, "row ids"))) return s;
+    if ((s = ids.get(4 * nnz, "positions"))) return s;
+    if ((s = perm.get(4 * nnz, "permutation"))) return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_col), 4 * nnz, "window-major colind"))) return s;
+    if ((s = dev_alloc(p, &p->w_vals, es * nnz, "window-major values"))) return s;
+
+    window_keys_kernel<<<148 * 8, 256, 0, st>>>(p->rowptr, p->colind, M, wcols, static_cast<uint32_t *>(wkey.p),
+                                               static_cast<int32_t *>(rowid.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    iota_kernel<<<ceil_div(nnz, 256), 256, 0, st>>>(static_cast<int32_t *>(ids.p), nnz);
+    SD_CUDA_TRY(cudaGetLastError());
+    int bits = 1;
+    while ((1 << bits) < W) ++bits;
+    size_t tb = 0;
+    SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, tb, static_cast<uint32_t *>(wkey.p),
+                                                static_cast<uint32_t *>(wkey_sorted.p), static_cast<int32_t *>(ids.p),
+                                                static_cast<int32_t *>(perm.p), nnz, 0, bits, st));
+    if ((s = tmp.get(tb, "sort scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(tmp.p, tb, static_cast<uint32_t *>(wkey.p),
+                                                static_cast<uint32_t *>(wkey_sorted.p), static_cast<int32_t *>(ids.p),
+                                                static_cast<int32_t *>(perm.p), nnz, 0, bits, st));
+    SD_CUDA_TRY(p->dtype == SD_F32
+                    ? launch_window_gather<float>(static_cast<int32_t *>(perm.p), p, static_cast<int32_t *>(rowid.p),
+                                                  static_cast<int32_t *>(w_row.p), st)
+                    : launch_window_gather<uint16_t>(static_cast<int32_t *>(perm.p), p, static_cast<int32_t *>(rowid.p),
+                                                     static_cast<int32_t *>(w_row.p), st));
+    // segment heads -> segment count and start positions
+    const int64_t nflag = nnz > M ? nnz : M;
+    if ((s = flag.get(nflag, "segment flags"))) return s;
+    if ((s = nsel.get(sizeof(int32_t), "segment count"))) return s;
+    window_headflag_kernel<<<ceil_div(nnz, 256), 256, 0, st>>>(static_cast<uint32_t *>(wkey_sorted.p),
+                                                              static_cast<int32_t *>(w_row.p), nnz,
+                                                              static_cast<uint8_t *>(flag.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    // upper bound on segments: nnz + E; allocate exactly after counting
+    cub::CountingInputIterator<int32_t> cnt(0);
+    TempBuf heads;
+    if ((s = heads.get(4 * nnz, "segment heads"))) return s;
+    size_t tb2 = 0;
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb2, cnt, static_cast<uint8_t *>(flag.p), static_cast<int32_t *>(heads.p),
+                                           static_cast<int32_t *>(nsel.p), static_cast<int>(nnz), st));
+    TempBuf tmp2;
+    if ((s = tmp2.get(tb2, "select scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp2.p, tb2, cnt, static_cast<uint8_t *>(flag.p), static_cast<int32_t *>(heads.p),
+                                           static_cast<int32_t *>(nsel.p), static_cast<int>(nnz), st));
+    int32_t nheads = 0;
+    SD_CUDA_TRY(cudaMemcpyAsync(&nheads, nsel.p, sizeof nheads, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    const int64_t S = E + nheads;
+    p->num_segments = S;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_ptr), 4 * (S + 1), "segment pointers"))) return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_seg_row), 4 * (S + 1), "segment rows"))) return s;
+    SD_CUDA_TRY(cudaMemcpyAsync(p->w_ptr + E, heads.p, 4 * static_cast<size_t>(nheads), cudaMemcpyDeviceToDevice, st));
+    if (E > 0) {   // ids of the empty rows, ascending, at the front
+        window_emptyflag_kernel<<<ceil_div(M, 256), 256, 0, st>>>(p->rowptr, M, static_cast<uint8_t *>(flag.p));
+        SD_CUDA_TRY(cudaGetLastError());
+        size_t tb3 = 0;
+        SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb3, cnt, static_cast<uint8_t *>(flag.p), p->w_seg_row,
+                                               static_cast<int32_t *>(nsel.p), static_cast<int>(M), st));
+        TempBuf tmp3;
+        if ((s = tmp3.get(tb3, "select scratch"))) return s;
+        SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp3.p, tb3, cnt, static_cast<uint8_t *>(flag.p), p->w_seg_row,
+                                               static_cast<int32_t *>(nsel.p), static_cast<int>(M), st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    window_segrow_kernel<<<ceil_div(S + 1, 256), 256, 0, st>>>(p->rowptr, p->colind, static_cast<uint32_t *>(wkey_sorted.p),
+                                                              static_cast<int32_t *>(w_row.p), wcols, E, S, nnz, p->w_ptr,
+                                                              p->w_seg_row);
+    SD_CUDA_TRY(cudaGetLastError());
+    if ((s = dwin.get(sizeof(int64_t) * (W + 1), "window bounds"))) return s;
+    window_bounds_kernel<<<1, 128, 0, st>>>(static_cast<uint32_t *>(wkey_sorted.p), p->w_ptr, E, S, W,
+                                           static_cast<int64_t *>(dwin.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    win_seg.assign(W + 1, 0);
+    SD_CUDA_TRY(cudaMemcpyAsync(win_seg.data(), dwin.p, sizeof(int64_t) * (W + 1), cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    win_seg[W] = S;
+    return SD_OK;
+}
+
+static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
+    sd_status_t s;
+    std::vector<int64_t> win_seg;
+    if (W > 1) {
+        if ((s = build_windows(p, W, win_seg, st))) return s;
+        p->m_ptr = p->w_ptr;
+        p->m_col = p->w_col;
+        p->m_vals = p->w_vals;
+        p->m_seg_row = p->w_seg_row;
+    } else {
+        W = 1;
+        p->m_ptr = p->rowptr;
+        p->m_col = p->colind;
+        p->m_vals = p->vals;
+        p->m_seg_row = nullptr;
+        p->num_segments = p->M;
+        win_seg = {0, p->M};
+    }
+    // nonzero positions of the window boundaries
+    std::vector<int32_t> win_nz(W + 1, 0);
+    for (int w = 0; w <= W; ++w)
+        SD_CUDA_TRY(cudaMemcpyAsync(&win_nz[w], p->m_ptr + win_seg[w], sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    int64_t ntiles = 0;
+    p->wins.clear();
+    for (int w = 0; w < W; ++w) {
+        sd_plan::Window win;
+        win.seg_begin = win_seg[w];
+        win.seg_end = win_seg[w + 1];
+        const int64_t total = (win.seg_end - win.seg_begin) + (win_nz[w + 1] - win_nz[w]);
+        win.ntiles = static_cast<int32_t>((total + kMergeTile - 1) / kMergeTile);
+        win.tile_base = ntiles;
+        win.nshort = win.nlong = 0;
+        ntiles += win.ntiles;
+        p->wins.push_back(win);
+    }
+    if (ntiles > INT32_MAX / 2) {
         set_error(SD_ERR_UNSUPPORTED, "too many merge tiles");
         return SD_ERR_UNSUPPORTED;
     }
-    p->ntiles = static_cast<int32_t>(ntiles);
-    sd_status_t s;
-    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_seg), sizeof(int32_t) * (ntiles + 1), "tile table")))
+    p->ntiles = ntiles;
+    // tile tables are concatenated: window w owns entries [tile_base + w, tile_base + w + ntiles_w]
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_seg), sizeof(int32_t) * (ntiles + W), "tile table")))
         return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->fix_short), sizeof(int32_t) * (ntiles + 1), "fix-up list")))
         return s;
@@ -332,36 +581,46 @@ static sd_status_t build_merge(sd_plan *p, cudaStream_t st) {
         return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_tail), sizeof(float) * ntiles * p->N, "tile tails")))
         return s;
-    merge_table_kernel<<<ceil_div(ntiles + 1, 256), 256, 0, st>>>(p->rowptr, 0, p->M, kMergeTile, p->ntiles,
-                                                                p->tile_seg);
-    SD_CUDA_TRY(cudaGetLastError());
+    int32_t max_tiles = 1;
+    for (auto &win : p->wins) max_tiles = std::max(max_tiles, win.ntiles);
     TempBuf flags_s, flags_l, nsel, tmp;
-    if ((s = flags_s.get(ntiles, "fix-up flags"))) return s;
-    if ((s = flags_l.get(ntiles, "fix-up flags"))) return s;
+    if ((s = flags_s.get(max_tiles, "fix-up flags"))) return s;
+    if ((s = flags_l.get(max_tiles, "fix-up flags"))) return s;
     if ((s = nsel.get(2 * sizeof(int32_t), "fix-up counts"))) return s;
-    merge_fixflag_kernel<<<ceil_div(ntiles, 256), 256, 0, st>>>(p->rowptr, p->tile_seg, 0, kMergeTile, p->ntiles,
-                                                               static_cast<uint8_t *>(flags_s.p),
-                                                               static_cast<uint8_t *>(flags_l.p));
-    SD_CUDA_TRY(cudaGetLastError());
     size_t tb = 0;
     cub::CountingInputIterator<int32_t> ids(0);
     int32_t *dn = static_cast<int32_t *>(nsel.p);
-    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb, ids, static_cast<uint8_t *>(flags_s.p), p->fix_short, dn,
-                                           static_cast<int>(ntiles), st));
+    SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb, ids, static_cast<uint8_t *>(flags_s.p), p->fix_short, dn, max_tiles,
+                                           st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
-    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_s.p), p->fix_short, dn,
-                                           static_cast<int>(ntiles), st));
-    SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_l.p), p->fix_long, dn + 1,
-                                           static_cast<int>(ntiles), st));
-    int32_t hn[2] = {0, 0};
-    SD_CUDA_TRY(cudaMemcpyAsync(hn, dn, sizeof hn, cudaMemcpyDeviceToHost, st));
-    SD_CUDA_TRY(cudaStreamSynchronize(st));
-    p->nfix_short = hn[0];
-    p->nfix_long = hn[1];
+    int launches = 0;
+    for (int w = 0; w < W; ++w) {
+        sd_plan::Window &win = p->wins[w];
+        if (win.ntiles == 0) continue;
+        int32_t *table = p->tile_seg + win.tile_base + w;
+        merge_table_kernel<<<ceil_div(win.ntiles + 1, 256), 256, 0, st>>>(p->m_ptr, win.seg_begin, win.seg_end, kMergeTile,
+                                                                         win.ntiles, table);
+        SD_CUDA_TRY(cudaGetLastError());
+        merge_fixflag_kernel<<<ceil_div(win.ntiles, 256), 256, 0, st>>>(p->m_ptr, table, win.seg_begin, kMergeTile,
+                                                                       win.ntiles, static_cast<uint8_t *>(flags_s.p),
+                                                                       static_cast<uint8_t *>(flags_l.p));
+        SD_CUDA_TRY(cudaGetLastError());
+        SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_s.p),
+                                               p->fix_short + win.tile_base, dn, win.ntiles, st));
+        SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp.p, tb, ids, static_cast<uint8_t *>(flags_l.p),
+                                               p->fix_long + win.tile_base, dn + 1, win.ntiles, st));
+        int32_t hn[2] = {0, 0};
+        SD_CUDA_TRY(cudaMemcpyAsync(hn, dn, sizeof hn, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        win.nshort = hn[0];
+        win.nlong = hn[1];
+        launches += 1 + (win.nshort > 0) + (win.nlong > 0);
+    }
     p->info.tile_items = kMergeTile;
     p->info.num_tiles = ntiles;
-    p->info.num_segments = p->M;
-    p->info.windows = 1;
+    p->info.num_segments = p->num_segments;
+    p->info.windows = W;
+    p->info.launches = launches;
     return SD_OK;
 }
 
@@ -525,18 +784,24 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     info.family = family;
 
     // ---- representation -----------------------------------------------------------------------
-    if (family == SD_MERGE && p->M > 0) {
-        if ((s = build_merge(p, st))) return s;
+    info.launches = 1;
+    if (family == SD_MERGE && p->M > 0 && p->nnz > 0) {
+        int W = d->windows == 0 ? decide_windows(info, p->dtype) : d->windows;
+        if (info.unsorted_rows != 0) W = 1;   // windows need ascending columns
+        if ((s = build_merge(p, W, st))) return s;
     } else if (family == SD_BSR_TC) {
         if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
     }
-    info.launches = (family == SD_MERGE && p->M > 0) ? info.windows * (1 + (p->nfix_short > 0 ? 1 : 0) + (p->nfix_long > 0 ? 1 : 0)) : 1;
     info.plan_bytes = p->owned;
     return SD_OK;
 }
 
 static void free_plan(sd_plan *p) {
     if (!p) return;
+    cudaFree(p->w_ptr);
+    cudaFree(p->w_col);
+    cudaFree(p->w_vals);
+    cudaFree(p->w_seg_row);
     cudaFree(p->tile_seg);
     cudaFree(p->fix_short);
     cudaFree(p->fix_long);
@@ -684,10 +949,33 @@ sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t 
         set_error(SD_ERR_UNSUPPORTED, "the plan holds no merge-path tile table");
         return SD_ERR_UNSUPPORTED;
     }
-    const int64_t n = plan->M > 0 ? static_cast<int64_t>(plan->ntiles) + 1 : 0;
+    const int64_t n = plan->wins.empty() ? 0 : plan->ntiles + static_cast<int64_t>(plan->wins.size());
     *count = n;
     if (tile_seg && cap >= n && n > 0)
         SD_CUDA_TRY(cudaMemcpy(tile_seg, plan->tile_seg, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+    return SD_OK;
+}
+
+sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_t *seg_row, int32_t *colind,
+                                 void *vals, int64_t *win_seg) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->info.family != SD_MERGE || plan->wins.size() < 2) {
+        set_error(SD_ERR_UNSUPPORTED, "the plan holds no column-window segment list");
+        return SD_ERR_UNSUPPORTED;
+    }
+    const int64_t S = plan->num_segments;
+    const size_t es = plan->dtype == SD_F32 ? 4 : 2;
+    if (seg_ptr) SD_CUDA_TRY(cudaMemcpy(seg_ptr, plan->w_ptr, 4 * (S + 1), cudaMemcpyDeviceToHost));
+    if (seg_row) SD_CUDA_TRY(cudaMemcpy(seg_row, plan->w_seg_row, 4 * S, cudaMemcpyDeviceToHost));
+    if (colind) SD_CUDA_TRY(cudaMemcpy(colind, plan->w_col, 4 * plan->nnz, cudaMemcpyDeviceToHost));
+    if (vals) SD_CUDA_TRY(cudaMemcpy(vals, plan->w_vals, es * plan->nnz, cudaMemcpyDeviceToHost));
+    if (win_seg) {
+        for (size_t w = 0; w < plan->wins.size(); ++w) win_seg[w] = plan->wins[w].seg_begin;
+        win_seg[plan->wins.size()] = S;
+    }
     return SD_OK;
 }
 
@@ -734,15 +1022,25 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         SD_CUDA_TRY(run_rowsplit(a, plan->dtype, vec, st));
         return SD_OK;
     case SD_MERGE: {
-        MergeArgs m;
-        m.s = a;
-        m.tile_seg = plan->tile_seg;
-        m.tile_head = plan->tile_head;
-        m.tile_tail = plan->tile_tail;
-        m.seg_begin = 0;
-        m.seg_end = M;
-        m.ntiles = plan->ntiles;
-        SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_short, plan->nfix_short, plan->fix_long, plan->nfix_long, st));
+        a.ptr = plan->m_ptr;
+        a.colind = plan->m_col;
+        a.vals = plan->m_vals;
+        a.seg_row = plan->m_seg_row;
+        a.S = plan->num_segments;
+        for (size_t w = 0; w < plan->wins.size(); ++w) {   // windows run in order on the stream
+            const sd_plan::Window &win = plan->wins[w];
+            if (win.ntiles == 0) continue;
+            MergeArgs m;
+            m.s = a;
+            m.tile_seg = plan->tile_seg + win.tile_base + w;
+            m.tile_head = plan->tile_head + win.tile_base * N;
+            m.tile_tail = plan->tile_tail + win.tile_base * N;
+            m.seg_begin = win.seg_begin;
+            m.seg_end = win.seg_end;
+            m.ntiles = win.ntiles;
+            SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_short + win.tile_base, win.nshort,
+                                  plan->fix_long + win.tile_base, win.nlong, st));
+        }
         return SD_OK;
     }
     case SD_BSR_TC: {

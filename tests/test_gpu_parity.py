@@ -349,3 +349,46 @@ def test_bsr_tensor_core_dense_blocks_bf16_exact_products():
     ref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
     assert np.array_equal(got.astype(np.float64), ref)
     plan.close()
+
+
+@pytest.mark.parametrize("kind", ["uniform", "short", "skewed", "onelong"])
+@pytest.mark.parametrize("windows", [2, 8, 5])
+@pytest.mark.parametrize("N,dtype", [(32, W.SD_F32), (8, W.SD_F32), (128, W.SD_BF16), (7, W.SD_F32)])
+def test_merge_with_column_windows(kind, windows, N, dtype):
+    rng = np.random.default_rng(windows * 100 + N)
+    M, K = 1500, 3001
+    lengths = shape_lengths(kind, M, K, rng)
+    lengths[100:110] = 0     # empty rows must still receive beta*C
+    w = W.random_csr(M, K, N, lengths, seed=N + windows, dtype=dtype, alpha=0.5, beta=1.25)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE, windows=windows)
+    info = plan.info()
+    assert info.windows == windows
+    # plan metadata against the oracle's own window-major construction
+    seg_ptr, seg_row, colind, vals, win_seg = sd.sd_plan_get_segments(plan.handle)
+    rp, rr, perm, rw = oracle.window_segments(w.rowptr, w.colind, M, K, windows)
+    assert np.array_equal(seg_ptr, rp) and np.array_equal(seg_row, rr) and np.array_equal(win_seg, rw)
+    assert np.array_equal(colind, w.colind[perm]) and vals.tobytes() == w.vals[perm].tobytes()
+    tiles = sd.sd_plan_get_tiles(plan.handle)
+    want = np.concatenate([oracle.merge_coords(rp[rw[i]:rw[i + 1] + 1], info.tile_items) + rw[i]
+                           for i in range(windows)])
+    assert np.array_equal(tiles, want.astype(np.int32))
+    got, intact = run_spmm(plan, w)
+    assert intact
+    check(w, got)
+    got2, _ = run_spmm(plan, w)
+    assert np.array_equal(got, got2)
+    poison = np.full((M, N), np.nan, np.float32)
+    got3, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got3, beta=0.0)
+    plan.close()
+
+
+def test_automatic_window_choice_matches_the_rule():
+    w = W.g5_skewed(M=1 << 16, N=32, scale_c=2.4e7 / 64, cap=4000)
+    dw = DeviceWorkload(w)
+    plan = dw.plan()
+    info = plan.info()
+    ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+    assert info.windows == oracle.decide_windows(ref, oracle.F32, info.l2_bytes) == 1   # B fits in L2 here
+    plan.close()

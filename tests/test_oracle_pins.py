@@ -427,3 +427,53 @@ def test_skewed_generator_counts():
     for i in range(0, M, 97):
         cols = w.colind[w.rowptr[i]:w.rowptr[i + 1]]
         assert np.all(np.diff(cols) > 0) and cols.min() >= 0 and cols.max() < M
+
+
+def test_o4_window_segments_against_python_sets():
+    rng = np.random.default_rng(9)
+    M, K = 60, 101
+    lengths = rng.integers(0, 9, size=M)
+    lengths[7] = 0
+    lengths[20] = 90
+    wl = W.random_csr(M, K, 1, lengths, seed=3)
+    seg_ptr, seg_row, perm, win_seg = oracle.window_segments(wl.rowptr, wl.colind, M, K, 4)
+    wcols = -(-K // 4)
+    # brute force: dictionary (window, row) -> positions
+    groups = {}
+    for i in range(M):
+        for p in range(wl.rowptr[i], wl.rowptr[i + 1]):
+            groups.setdefault((wl.colind[p] // wcols, i), []).append(p)
+    empties = [i for i in range(M) if lengths[i] == 0]
+    keys = sorted(groups)
+    assert len(seg_row) == len(empties) + len(keys)
+    assert [int(r) for r in seg_row[:len(empties)]] == empties
+    assert np.all(seg_ptr[:len(empties) + 1] == 0)
+    q = 0
+    for s, (win, row) in enumerate(keys, start=len(empties)):
+        assert seg_ptr[s] == q
+        first_w = wl.colind[wl.rowptr[row]] // wcols
+        assert (int(seg_row[s]) & 0x7FFFFFFF) == row
+        assert bool(int(seg_row[s]) & 0x80000000) == (first_w != win)
+        assert perm[q:q + len(groups[(win, row)])].tolist() == groups[(win, row)]
+        q += len(groups[(win, row)])
+    assert seg_ptr[-1] == q == wl.nnz
+    assert sorted(perm.tolist()) == list(range(wl.nnz))
+    for wdx in range(5):
+        want = len(empties) + sum(1 for k in keys if k[0] < wdx) if wdx > 0 else 0
+        assert win_seg[wdx] == want
+
+
+def test_o4_window_rule():
+    info = oracle.Info()
+    info.M = info.K = 4_194_304
+    info.N = 32
+    info.nnz = 59_839_586
+    assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 8     # 512 MiB of B, 75.6 MiB budget
+    info.nnz = 16 * info.M
+    assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 1     # long rows on average
+    info.nnz = 59_839_586
+    info.unsorted_rows = 1
+    assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 1
+    info.unsorted_rows = 0
+    info.K = 100_000
+    assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 1     # B fits
