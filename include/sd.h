@@ -168,13 +168,16 @@ sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t 
 /* sd_plan_get_segments -- MERGE family with column windows (the paper's "packed column
  * windows", Sec. 3.4): copy the window-major representation to HOST arrays.  The columns are
  * cut into `windows` ranges of ceil(K / windows) columns; a segment is the part of one row
- * that falls into one window; segments are ordered by (window, row), except that the empty
- * rows come first as zero-length segments of window 0.
+ * that falls into one window.  Inside a window the segments with more than 32 nonzeros come
+ * first (they go to the merge-path kernel), then those with none or 2..32 (one lane group per
+ * segment), then those with exactly one; rows ascend inside each class, except that the empty
+ * rows are zero-length segments at the head of window 0's middle class.
  *   seg_ptr  int32 [num_segments + 1]  start of each segment in the re-bucketed arrays
  *   seg_row  int32 [num_segments]      output row; bit 31 set when an earlier window already
  *                                      wrote the row (this segment then adds to C)
  *   colind   int32 [nnz], vals [nnz]   nonzeros in window-major order (plan dtype)
- *   win_seg  int64 [windows + 1]       first segment of each window
+ *   win_seg  int64 [3*windows + 1]     per window: first segment of each of the three classes;
+ *                                      last entry = num_segments
  * Any pointer may be NULL.  SD_ERR_UNSUPPORTED when the plan has no windows. */
 sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_t *seg_row, int32_t *colind,
                                  void *vals, int64_t *win_seg);

@@ -199,18 +199,19 @@ def decide_windows(info: Info, dtype: int, l2_bytes: int) -> int:
     return int(lib().sdo_decide_windows(C.byref(info), C.c_int(dtype), C.c_int64(l2_bytes)))
 
 
-def window_segments(rowptr, colind, M, K, W):
-    """O4: window-major segment list.  Returns (seg_ptr, seg_row, perm, win_seg)."""
+def window_segments(rowptr, colind, M, K, W, short_len=32):
+    """O4: window-major segment list ordered by (window, class, row).
+    Returns (seg_ptr, seg_row, perm, bounds[3W+1])."""
     rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
     colind = np.ascontiguousarray(colind, dtype=np.int32)
     nnz = int(rowptr[-1])
     seg_ptr = np.zeros(nnz + M + 1, np.int32)
     seg_row = np.zeros(nnz + M, np.int32)
     perm = np.zeros(max(nnz, 1), np.int32)
-    win_seg = np.zeros(W + 1, np.int64)
+    bounds = np.zeros(3 * W + 1, np.int64)
     S = int(lib().sdo_window_segments(C.c_int64(M), C.c_int64(K), _p(rowptr), _p(colind), C.c_int32(W),
-                                      _p(seg_ptr), _p(seg_row), _p(perm), _p(win_seg)))
-    return seg_ptr[:S + 1].copy(), seg_row[:S].copy(), perm[:nnz].copy(), win_seg
+                                      C.c_int32(short_len), _p(seg_ptr), _p(seg_row), _p(perm), _p(bounds)))
+    return seg_ptr[:S + 1].copy(), seg_row[:S].copy(), perm[:nnz].copy(), bounds
 
 
 def hist_bin(v: int) -> int:

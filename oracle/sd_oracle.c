@@ -452,42 +452,72 @@ int sdo_decide_windows(const sdo_info_t *o, int dtype, int64_t l2_bytes)
 }
 
 /* Window-major segment list.  Window of a column: col / ceil(K / W).  A segment is the part
- * of one row inside one window.  Order: the empty rows first (zero-length segments, window
- * 0), then for w = 0..W-1, for ascending row, the row's nonzeros of window w in storage
- * order.  seg_row carries bit 31 when the row's first nonzero lies in an earlier window
- * (columns are ascending), i.e. when an earlier segment already wrote the row.
- * perm[q] = original position of the q-th re-bucketed nonzero.  Returns the segment count;
- * seg_ptr needs room for nnz + M + 1 entries, seg_row for nnz + M, win_seg for W + 1. */
+ * of one row inside one window.  First ordering: the empty rows (zero-length segments of
+ * window 0), then for w = 0..W-1, for ascending row, the row's nonzeros of window w in storage
+ * order.  Final ordering: a stable sort of that list by (window, class), class 0 = more than
+ * short_len nonzeros, class 1 = none or 2..short_len, class 2 = exactly one.
+ * seg_row carries bit 31 when the row's first nonzero lies in an earlier window (columns are
+ * ascending), i.e. when an earlier segment already wrote the row.  perm[q] = original position
+ * of the q-th re-bucketed nonzero.  bounds[3w], bounds[3w+1], bounds[3w+2] = first segment
+ * of class 0 / 1 / 2 of window w; bounds[3W] = segment count.  Returns the segment count; seg_ptr needs room for
+ * nnz + M + 1 entries, seg_row for nnz + M, bounds for 3W + 1. */
 int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const int32_t *colind,
-                            int32_t W, int32_t *seg_ptr, int32_t *seg_row, int32_t *perm,
-                            int64_t *win_seg)
+                            int32_t W, int32_t short_len, int32_t *seg_ptr, int32_t *seg_row,
+                            int32_t *perm, int64_t *bounds)
 {
-    int64_t wcols = (K + W - 1) / W, S = 0, q = 0;
+    int64_t wcols = (K + W - 1) / W, nnz = M > 0 ? rowptr[M] : 0;
+    int64_t cap = nnz + M + 1, S = 0;
+    /* first ordering */
+    int64_t *first = (int64_t *)malloc(sizeof(int64_t) * (size_t)cap); /* first original position */
+    int32_t *len = (int32_t *)malloc(sizeof(int32_t) * (size_t)cap);
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)cap);
+    int32_t *key = (int32_t *)malloc(sizeof(int32_t) * (size_t)cap);
     for (int64_t i = 0; i < M; ++i)
         if (rowptr[i + 1] == rowptr[i]) {
-            seg_ptr[S] = 0;
-            seg_row[S] = (int32_t)i;
+            first[S] = 0;
+            len[S] = 0;
+            row[S] = (int32_t)i;
+            key[S] = 1;
             ++S;
         }
-    for (int32_t w = 0; w < W; ++w) {
-        win_seg[w] = (w == 0) ? 0 : S;
+    for (int32_t w = 0; w < W; ++w)
         for (int64_t i = 0; i < M; ++i) {
-            int started = 0;
-            for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
-                if (colind[p] / wcols != w)
-                    continue;
-                if (!started) {
-                    int64_t first_w = colind[rowptr[i]] / wcols;
-                    seg_ptr[S] = (int32_t)q;
-                    seg_row[S] = (int32_t)i | (first_w != w ? (int32_t)0x80000000u : 0);
-                    ++S;
-                    started = 1;
+            int64_t n = 0, f = -1;
+            for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p)
+                if (colind[p] / wcols == w) {
+                    if (n == 0)
+                        f = p;
+                    ++n;
                 }
-                perm[q++] = (int32_t)p;
-            }
+            if (n == 0)
+                continue;
+            int64_t first_w = colind[rowptr[i]] / wcols;
+            first[S] = f;
+            len[S] = (int32_t)n;
+            row[S] = (int32_t)i | (first_w != w ? (int32_t)0x80000000u : 0);
+            key[S] = 3 * w + (n > short_len ? 0 : (n == 1 ? 2 : 1));
+            ++S;
+        }
+    /* stable sort by key: one pass per key value */
+    int64_t out = 0, q = 0;
+    for (int32_t k = 0; k < 3 * W; ++k) {
+        bounds[k] = out;
+        for (int64_t s = 0; s < S; ++s) {
+            if (key[s] != k)
+                continue;
+            seg_ptr[out] = (int32_t)q;
+            seg_row[out] = row[s];
+            /* columns ascend inside a row, so the run is contiguous in the original arrays */
+            for (int64_t t = 0; t < len[s]; ++t)
+                perm[q++] = (int32_t)(first[s] + t);
+            ++out;
         }
     }
-    win_seg[W] = S;
+    bounds[3 * W] = S;
     seg_ptr[S] = (int32_t)q;
+    free(first);
+    free(len);
+    free(row);
+    free(key);
     return S;
 }

@@ -192,7 +192,7 @@ def sd_plan_get_segments(plan):
     seg_row = np.zeros(S, np.int32)
     colind = np.zeros(nnz, np.int32)
     vals = np.zeros(nnz, np.float32 if info.dtype == SD_F32 else np.uint16)
-    win_seg = np.zeros(W + 1, np.int64)
+    win_seg = np.zeros(3 * W + 1, np.int64)
     rc = load().sd_plan_get_segments(plan, seg_ptr.ctypes.data, seg_row.ctypes.data, colind.ctypes.data,
                                      vals.ctypes.data, win_seg.ctypes.data)
     if rc != SD_OK:

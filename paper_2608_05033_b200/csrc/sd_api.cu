@@ -259,16 +259,10 @@ window_keys_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict
         }
 }
 
-template <typename T>
-__global__ void window_gather_kernel(const int32_t *__restrict__ perm, const int32_t *__restrict__ colind,
-                                     const T *__restrict__ vals, const int32_t *__restrict__ rowid, int64_t nnz,
-                                     int32_t *__restrict__ w_col, T *__restrict__ w_val, int32_t *__restrict__ w_row) {
+__global__ void window_rows_kernel(const int32_t *__restrict__ perm, const int32_t *__restrict__ rowid, int64_t nnz,
+                                   int32_t *__restrict__ w_row) {
     const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (q >= nnz) return;
-    const int32_t p = perm[q];
-    w_col[q] = colind[p];
-    w_val[q] = vals[p];
-    w_row[q] = rowid[p];
+    if (q < nnz) w_row[q] = rowid[perm[q]];
 }
 
 __global__ void window_headflag_kernel(const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ w_row,
@@ -283,44 +277,97 @@ __global__ void window_emptyflag_kernel(const int32_t *__restrict__ rowptr, int6
     if (i < M) flag[i] = rowptr[i + 1] == rowptr[i];
 }
 
-// seg_ptr[0..E) = 0 for the empty rows (their ids are already in seg_row[0..E)); for the other
-// segments the output row and the "row already written by an earlier window" bit.
-__global__ void window_segrow_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind,
-                                     const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ w_row,
-                                     int32_t wcols, int64_t E, int64_t S, int64_t nnz, int32_t *__restrict__ seg_ptr,
-                                     int32_t *__restrict__ seg_row) {
+// First ordering of the segments: the E empty rows (their ids are already in seg_row[0..E)),
+// then the runs of (window, row) in window-major order.  Each gets its start and length in
+// the window-sorted nonzero order, its output row with the "already written" bit, and the
+// sort key 3 * window + class (class 0: more than `short_len` nonzeros, class 1: 0 or
+// 2..short_len nonzeros, class 2: exactly one).
+__global__ void window_segments_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind,
+                                       const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ w_row,
+                                       const int32_t *__restrict__ heads, int32_t wcols, int32_t short_len, int64_t E,
+                                       int64_t S, int64_t nnz, int32_t *__restrict__ seg_start,
+                                       int32_t *__restrict__ seg_len, int32_t *__restrict__ seg_row,
+                                       uint32_t *__restrict__ seg_key) {
     const int64_t s = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (s > S) return;
-    if (s == S) {
-        seg_ptr[S] = static_cast<int32_t>(nnz);
-        return;
-    }
+    if (s >= S) return;
     if (s < E) {
-        seg_ptr[s] = 0;
+        seg_start[s] = 0;
+        seg_len[s] = 0;
+        seg_key[s] = 1;   // window 0, short class
         return;
     }
-    const int32_t q = seg_ptr[s];
+    const int64_t h = s - E;
+    const int32_t q = heads[h];
+    const int32_t len = static_cast<int32_t>((h + 1 < S - E ? heads[h + 1] : nnz) - q);
     const int32_t row = w_row[q];
+    const uint32_t win = wkey_sorted[q];
     const uint32_t first_win = static_cast<uint32_t>(colind[rowptr[row]] / wcols);
-    seg_row[s] = row | (wkey_sorted[q] != first_win ? static_cast<int32_t>(0x80000000u) : 0);
+    seg_start[s] = q;
+    seg_len[s] = len;
+    seg_row[s] = row | (win != first_win ? static_cast<int32_t>(0x80000000u) : 0);
+    seg_key[s] = 3 * win + (len > short_len ? 0u : (len == 1 ? 2u : 1u));
 }
 
-// win_seg[w] = first segment whose window is >= w (empty rows belong to window 0).
-__global__ void window_bounds_kernel(const uint32_t *__restrict__ wkey_sorted, const int32_t *__restrict__ seg_ptr,
-                                     int64_t E, int64_t S, int32_t W, int64_t *__restrict__ win_seg) {
-    const int w = threadIdx.x;
-    if (w > W) return;
-    if (w == 0) {
-        win_seg[0] = 0;
-        return;
-    }
-    int64_t lo = E, hi = S;
+__global__ void window_reorder_kernel(const int32_t *__restrict__ order, const int32_t *__restrict__ seg_len,
+                                      const int32_t *__restrict__ seg_row, int64_t S, int32_t *__restrict__ len2,
+                                      int32_t *__restrict__ row2) {
+    const int64_t s = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    len2[s] = seg_len[order[s]];
+    row2[s] = seg_row[order[s]];
+}
+
+// Final gather of the nonzeros: output position q belongs to the segment found by binary
+// search in the new segment pointers; its source is that segment's run in window-sorted order.
+template <typename T>
+__global__ void window_gather_kernel(const int32_t *__restrict__ seg_ptr2, const int32_t *__restrict__ order,
+                                     const int32_t *__restrict__ seg_start, const int32_t *__restrict__ perm,
+                                     const int32_t *__restrict__ colind, const T *__restrict__ vals, int64_t S, int64_t nnz,
+                                     int32_t *__restrict__ w_col, T *__restrict__ w_val) {
+    const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (q >= nnz) return;
+    int64_t lo = 0, hi = S;   // last segment with seg_ptr2[s] <= q and a non-zero length covers q
     while (lo < hi) {
         const int64_t mid = (lo + hi) >> 1;
-        if (wkey_sorted[seg_ptr[mid]] < static_cast<uint32_t>(w)) lo = mid + 1;
+        if (seg_ptr2[mid + 1] <= q) lo = mid + 1;
         else hi = mid;
     }
-    win_seg[w] = lo;
+    const int32_t p = perm[seg_start[order[lo]] + (q - seg_ptr2[lo])];
+    w_col[q] = colind[p];
+    w_val[q] = vals[p];
+}
+
+// Chunks of the long segments: segment s (class 0) is cut into ceil(len / chunk) pieces.
+__global__ void chunk_count_kernel(const uint32_t *__restrict__ key_sorted, const int32_t *__restrict__ len2, int64_t S,
+                                   int32_t chunk, int32_t *__restrict__ nch) {
+    const int64_t s = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (s > S) return;
+    nch[s] = (s < S && key_sorted[s] % 3 == 0) ? (len2[s] + chunk - 1) / chunk : 0;
+}
+
+// chunk_ptr of window w starts at seg_chunk[first long segment] + w and holds one terminator.
+__global__ void chunk_fill_kernel(const int32_t *__restrict__ seg_ptr, const int32_t *__restrict__ seg_chunk,
+                                  int64_t seg_begin, int64_t seg_end, int32_t chunk, int32_t w,
+                                  int32_t *__restrict__ chunk_ptr) {
+    const int64_t s = seg_begin + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (s >= seg_end) return;
+    const int32_t c0 = seg_chunk[s], c1 = seg_chunk[s + 1];
+    for (int32_t c = c0; c < c1; ++c) chunk_ptr[c + w] = seg_ptr[s] + (c - c0) * chunk;
+    if (s == seg_end - 1) chunk_ptr[c1 + w] = seg_ptr[s + 1];
+}
+
+// bounds[k] = first segment (in the final order) whose key is >= k, for k = 0..2W.
+__global__ void window_bounds_kernel(const uint32_t *__restrict__ key_sorted, int64_t S, int32_t nkeys,
+                                     int64_t *__restrict__ bounds) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k > nkeys) return;
+    int64_t lo = 0, hi = S;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (key_sorted[mid] < static_cast<uint32_t>(k)) lo = mid + 1;
+        else hi = mid;
+    }
+    bounds[k] = lo;
 }
 
 }  // namespace sd
@@ -347,9 +394,17 @@ struct sd_plan {
     void *w_vals = nullptr;
     int32_t *w_seg_row = nullptr;
     int64_t num_segments = 0;
+    int32_t *seg_chunk = nullptr;   // [S + 1] first chunk of every segment (long segments own chunks)
+    int32_t *chunk_ptr = nullptr;   // per window: nonzero boundaries of its chunks, one terminator each
+    float *chunk_out = nullptr;     // [chunks][N] partial sums of the chunks
+    int64_t num_chunks = 0;
     struct Window {
-        int64_t seg_begin, seg_end;
-        int64_t tile_base;         // first tile of the window in the concatenated tile numbering
+        int64_t seg_begin, seg_end;     // segments of the merge-path kernel (all of them without windows)
+        int64_t short_begin, short_end; // segments of the group-per-segment kernel (windows only)
+        int64_t single_begin, single_end; // one-nonzero segments (windows only)
+        int32_t single_nz;              // position of the first of them in the re-bucketed nonzeros
+        int64_t chunk_begin, chunk_end; // chunks of the long segments (windows only)
+        int64_t tile_base;              // first tile of the window in the concatenated tile numbering
         int32_t ntiles, nshort, nlong;
     };
     std::vector<Window> wins;
@@ -430,22 +485,20 @@ __global__ void iota_kernel(int32_t *out, int64_t n) {
     if (i < n) out[i] = static_cast<int32_t>(i);
 }
 
-template <typename T>
-static cudaError_t launch_window_gather(const int32_t *perm, sd_plan *p, const int32_t *rowid, int32_t *w_row,
-                                        cudaStream_t st) {
-    window_gather_kernel<T><<<ceil_div(p->nnz, 256), 256, 0, st>>>(perm, p->colind, static_cast<const T *>(p->vals), rowid,
-                                                                  p->nnz, p->w_col, static_cast<T *>(p->w_vals), w_row);
-    return cudaGetLastError();
-}
+constexpr int kChunkNnz = 128;      // long segments are cut into pieces of at most this many nonzeros
+constexpr int kShortSegment = 32;   // segments up to this many nonzeros go to the group-per-segment kernel
 
-// Re-buckets the nonzeros by column window and builds the (row, window) segment list.
-static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &win_seg, cudaStream_t st) {
+// Re-buckets the nonzeros by column window and builds the (row, window) segment list, ordered by
+// (window, class, row): inside a window the long segments come first (merge-path kernel), then the
+// short ones (group-per-segment kernel), then those of exactly one nonzero (flat kernel).
+// bounds[3w .. 3w+3] delimit the three classes of window w.
+static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds, cudaStream_t st) {
     const int64_t nnz = p->nnz, M = p->M;
     const int32_t wcols = static_cast<int32_t>((p->K + W - 1) / W);
     const size_t es = p->dtype == SD_F32 ? 4 : 2;
     const int64_t E = p->info.empty_rows;
     sd_status_t s;
-    TempBuf wkey, wkey_sorted, rowid, w_row, ids, perm, tmp, flag, nsel, dwin;
+    TempBuf wkey, wkey_sorted, rowid, w_row, ids, perm, tmp, flag, nsel, heads;
     if ((s = wkey.get(4 * nnz, "window keys"))) return s;
     if ((s = wkey_sorted.get(4 * nnz, "window keys"))) return s;
     if ((s = rowid.get(4 * nnz, "row ids"))) return s;
@@ -470,26 +523,22 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &win_se
     SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(tmp.p, tb, static_cast<uint32_t *>(wkey.p),
                                                 static_cast<uint32_t *>(wkey_sorted.p), static_cast<int32_t *>(ids.p),
                                                 static_cast<int32_t *>(perm.p), nnz, 0, bits, st));
-    SD_CUDA_TRY(p->dtype == SD_F32
-                    ? launch_window_gather<float>(static_cast<int32_t *>(perm.p), p, static_cast<int32_t *>(rowid.p),
-                                                  static_cast<int32_t *>(w_row.p), st)
-                    : launch_window_gather<uint16_t>(static_cast<int32_t *>(perm.p), p, static_cast<int32_t *>(rowid.p),
-                                                     static_cast<int32_t *>(w_row.p), st));
-    // segment heads -> segment count and start positions
+    window_rows_kernel<<<ceil_div(nnz, 256), 256, 0, st>>>(static_cast<int32_t *>(perm.p), static_cast<int32_t *>(rowid.p),
+                                                          nnz, static_cast<int32_t *>(w_row.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    // runs of (window, row): head flags -> head positions
     const int64_t nflag = nnz > M ? nnz : M;
     if ((s = flag.get(nflag, "segment flags"))) return s;
     if ((s = nsel.get(sizeof(int32_t), "segment count"))) return s;
+    if ((s = heads.get(4 * nnz, "segment heads"))) return s;
     window_headflag_kernel<<<ceil_div(nnz, 256), 256, 0, st>>>(static_cast<uint32_t *>(wkey_sorted.p),
                                                               static_cast<int32_t *>(w_row.p), nnz,
                                                               static_cast<uint8_t *>(flag.p));
     SD_CUDA_TRY(cudaGetLastError());
-    // upper bound on segments: nnz + E; allocate exactly after counting
     cub::CountingInputIterator<int32_t> cnt(0);
-    TempBuf heads;
-    if ((s = heads.get(4 * nnz, "segment heads"))) return s;
     size_t tb2 = 0;
     SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb2, cnt, static_cast<uint8_t *>(flag.p), static_cast<int32_t *>(heads.p),
-                                           static_cast<int32_t *>(nsel.p), static_cast<int>(nnz), st));
+                                           static_cast<int32_t *>(nsel.p), static_cast<int>(nflag), st));
     TempBuf tmp2;
     if ((s = tmp2.get(tb2, "select scratch"))) return s;
     SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp2.p, tb2, cnt, static_cast<uint8_t *>(flag.p), static_cast<int32_t *>(heads.p),
@@ -499,39 +548,110 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &win_se
     SD_CUDA_TRY(cudaStreamSynchronize(st));
     const int64_t S = E + nheads;
     p->num_segments = S;
+
+    TempBuf seg_start, seg_len, seg_row1, seg_key, seg_key_sorted, seg_ids, order, len2, dbounds;
+    if ((s = seg_start.get(4 * S, "segment starts"))) return s;
+    if ((s = seg_len.get(4 * S, "segment lengths"))) return s;
+    if ((s = seg_row1.get(4 * S, "segment rows"))) return s;
+    if ((s = seg_key.get(4 * S, "segment keys"))) return s;
+    if ((s = seg_key_sorted.get(4 * S, "segment keys"))) return s;
+    if ((s = seg_ids.get(4 * S, "segment ids"))) return s;
+    if ((s = order.get(4 * S, "segment order"))) return s;
+    if ((s = len2.get(4 * (S + 1), "segment lengths"))) return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_ptr), 4 * (S + 1), "segment pointers"))) return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_seg_row), 4 * (S + 1), "segment rows"))) return s;
-    SD_CUDA_TRY(cudaMemcpyAsync(p->w_ptr + E, heads.p, 4 * static_cast<size_t>(nheads), cudaMemcpyDeviceToDevice, st));
-    if (E > 0) {   // ids of the empty rows, ascending, at the front
+    if (E > 0) {   // ids of the empty rows, ascending, at the front of the first ordering
         window_emptyflag_kernel<<<ceil_div(M, 256), 256, 0, st>>>(p->rowptr, M, static_cast<uint8_t *>(flag.p));
         SD_CUDA_TRY(cudaGetLastError());
-        size_t tb3 = 0;
-        SD_CUDA_TRY(cub::DeviceSelect::Flagged(nullptr, tb3, cnt, static_cast<uint8_t *>(flag.p), p->w_seg_row,
-                                               static_cast<int32_t *>(nsel.p), static_cast<int>(M), st));
-        TempBuf tmp3;
-        if ((s = tmp3.get(tb3, "select scratch"))) return s;
-        SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp3.p, tb3, cnt, static_cast<uint8_t *>(flag.p), p->w_seg_row,
-                                               static_cast<int32_t *>(nsel.p), static_cast<int>(M), st));
-        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        SD_CUDA_TRY(cub::DeviceSelect::Flagged(tmp2.p, tb2, cnt, static_cast<uint8_t *>(flag.p),
+                                               static_cast<int32_t *>(seg_row1.p), static_cast<int32_t *>(nsel.p),
+                                               static_cast<int>(M), st));
     }
-    window_segrow_kernel<<<ceil_div(S + 1, 256), 256, 0, st>>>(p->rowptr, p->colind, static_cast<uint32_t *>(wkey_sorted.p),
-                                                              static_cast<int32_t *>(w_row.p), wcols, E, S, nnz, p->w_ptr,
-                                                              p->w_seg_row);
+    window_segments_kernel<<<ceil_div(S, 256), 256, 0, st>>>(
+        p->rowptr, p->colind, static_cast<uint32_t *>(wkey_sorted.p), static_cast<int32_t *>(w_row.p),
+        static_cast<int32_t *>(heads.p), wcols, kShortSegment, E, S, nnz, static_cast<int32_t *>(seg_start.p),
+        static_cast<int32_t *>(seg_len.p), static_cast<int32_t *>(seg_row1.p), static_cast<uint32_t *>(seg_key.p));
     SD_CUDA_TRY(cudaGetLastError());
-    if ((s = dwin.get(sizeof(int64_t) * (W + 1), "window bounds"))) return s;
-    window_bounds_kernel<<<1, 128, 0, st>>>(static_cast<uint32_t *>(wkey_sorted.p), p->w_ptr, E, S, W,
-                                           static_cast<int64_t *>(dwin.p));
+    // stable sort of the segments by (window, class)
+    iota_kernel<<<ceil_div(S, 256), 256, 0, st>>>(static_cast<int32_t *>(seg_ids.p), S);
     SD_CUDA_TRY(cudaGetLastError());
-    win_seg.assign(W + 1, 0);
-    SD_CUDA_TRY(cudaMemcpyAsync(win_seg.data(), dwin.p, sizeof(int64_t) * (W + 1), cudaMemcpyDeviceToHost, st));
+    int kbits = 1;
+    while ((1 << kbits) < 3 * W) ++kbits;
+    size_t tb3 = 0;
+    SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, tb3, static_cast<uint32_t *>(seg_key.p),
+                                                static_cast<uint32_t *>(seg_key_sorted.p),
+                                                static_cast<int32_t *>(seg_ids.p), static_cast<int32_t *>(order.p), S, 0,
+                                                kbits, st));
+    TempBuf tmp3;
+    if ((s = tmp3.get(tb3, "sort scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(tmp3.p, tb3, static_cast<uint32_t *>(seg_key.p),
+                                                static_cast<uint32_t *>(seg_key_sorted.p),
+                                                static_cast<int32_t *>(seg_ids.p), static_cast<int32_t *>(order.p), S, 0,
+                                                kbits, st));
+    window_reorder_kernel<<<ceil_div(S, 256), 256, 0, st>>>(static_cast<int32_t *>(order.p),
+                                                           static_cast<int32_t *>(seg_len.p),
+                                                           static_cast<int32_t *>(seg_row1.p), S,
+                                                           static_cast<int32_t *>(len2.p), p->w_seg_row);
+    SD_CUDA_TRY(cudaGetLastError());
+    SD_CUDA_TRY(cudaMemsetAsync(static_cast<int32_t *>(len2.p) + S, 0, 4, st));
+    size_t tb4 = 0;
+    SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(nullptr, tb4, static_cast<int32_t *>(len2.p), p->w_ptr,
+                                              static_cast<int>(S + 1), st));
+    TempBuf tmp4;
+    if ((s = tmp4.get(tb4, "scan scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(tmp4.p, tb4, static_cast<int32_t *>(len2.p), p->w_ptr,
+                                              static_cast<int>(S + 1), st));
+    if (p->dtype == SD_F32)
+        window_gather_kernel<float><<<ceil_div(nnz, 256), 256, 0, st>>>(
+            p->w_ptr, static_cast<int32_t *>(order.p), static_cast<int32_t *>(seg_start.p), static_cast<int32_t *>(perm.p),
+            p->colind, static_cast<const float *>(p->vals), S, nnz, p->w_col, static_cast<float *>(p->w_vals));
+    else
+        window_gather_kernel<uint16_t><<<ceil_div(nnz, 256), 256, 0, st>>>(
+            p->w_ptr, static_cast<int32_t *>(order.p), static_cast<int32_t *>(seg_start.p), static_cast<int32_t *>(perm.p),
+            p->colind, static_cast<const uint16_t *>(p->vals), S, nnz, p->w_col, static_cast<uint16_t *>(p->w_vals));
+    SD_CUDA_TRY(cudaGetLastError());
+    if ((s = dbounds.get(sizeof(int64_t) * (3 * W + 1), "window bounds"))) return s;
+    window_bounds_kernel<<<1, 256, 0, st>>>(static_cast<uint32_t *>(seg_key_sorted.p), S, 3 * W,
+                                           static_cast<int64_t *>(dbounds.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    bounds.assign(3 * W + 1, 0);
+    SD_CUDA_TRY(cudaMemcpyAsync(bounds.data(), dbounds.p, sizeof(int64_t) * (3 * W + 1), cudaMemcpyDeviceToHost, st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));
-    win_seg[W] = S;
+
+    // chunks of the long segments: counts -> exclusive scan -> boundaries
+    TempBuf nch;
+    if ((s = nch.get(4 * (S + 1), "chunk counts"))) return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->seg_chunk), 4 * (S + 1), "segment chunks"))) return s;
+    chunk_count_kernel<<<ceil_div(S + 1, 256), 256, 0, st>>>(static_cast<uint32_t *>(seg_key_sorted.p),
+                                                            static_cast<int32_t *>(len2.p), S, kChunkNnz,
+                                                            static_cast<int32_t *>(nch.p));
+    SD_CUDA_TRY(cudaGetLastError());
+    SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(tmp4.p, tb4, static_cast<int32_t *>(nch.p), p->seg_chunk,
+                                              static_cast<int>(S + 1), st));
+    int32_t total_chunks = 0;
+    SD_CUDA_TRY(cudaMemcpyAsync(&total_chunks, p->seg_chunk + S, 4, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    p->num_chunks = total_chunks;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_ptr), 4 * (static_cast<int64_t>(total_chunks) + W + 1),
+                       "chunk boundaries")))
+        return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * total_chunks * p->N, "chunk sums")))
+        return s;
+    for (int w = 0; w < W; ++w) {
+        const int64_t sb = bounds[3 * w], se = bounds[3 * w + 1];
+        if (se > sb) {
+            chunk_fill_kernel<<<ceil_div(se - sb, 256), 256, 0, st>>>(p->w_ptr, p->seg_chunk, sb, se, kChunkNnz, w,
+                                                                     p->chunk_ptr);
+            SD_CUDA_TRY(cudaGetLastError());
+        }
+    }
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
     return SD_OK;
 }
 
 static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
     sd_status_t s;
-    std::vector<int64_t> win_seg;
+    std::vector<int64_t> win_seg;   // per window: start of the long class, start of the short class
     if (W > 1) {
         if ((s = build_windows(p, W, win_seg, st))) return s;
         p->m_ptr = p->w_ptr;
@@ -545,20 +665,27 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
         p->m_vals = p->vals;
         p->m_seg_row = nullptr;
         p->num_segments = p->M;
-        win_seg = {0, p->M};
+        win_seg = {0, p->M, p->M, p->M};
     }
-    // nonzero positions of the window boundaries
-    std::vector<int32_t> win_nz(W + 1, 0);
-    for (int w = 0; w <= W; ++w)
-        SD_CUDA_TRY(cudaMemcpyAsync(&win_nz[w], p->m_ptr + win_seg[w], sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    // nonzero positions of the class boundaries
+    std::vector<int32_t> win_nz(3 * W + 1, 0);
+    for (int k = 0; k <= 3 * W; ++k)
+        SD_CUDA_TRY(cudaMemcpyAsync(&win_nz[k], p->m_ptr + win_seg[k], sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));
     int64_t ntiles = 0;
     p->wins.clear();
     for (int w = 0; w < W; ++w) {
         sd_plan::Window win;
-        win.seg_begin = win_seg[w];
-        win.seg_end = win_seg[w + 1];
-        const int64_t total = (win.seg_end - win.seg_begin) + (win_nz[w + 1] - win_nz[w]);
+        win.seg_begin = win_seg[3 * w];
+        win.seg_end = win_seg[3 * w + 1];
+        win.short_begin = win_seg[3 * w + 1];
+        win.short_end = win_seg[3 * w + 2];
+        win.single_begin = win_seg[3 * w + 2];
+        win.single_end = win_seg[3 * w + 3];
+        win.single_nz = win_nz[3 * w + 2];
+        win.chunk_begin = win.chunk_end = 0;
+        int64_t total = (win.seg_end - win.seg_begin) + (win_nz[3 * w + 1] - win_nz[3 * w]);
+        if (W > 1) total = 0;   // with windows the long segments run as chunks, not as merge-path tiles
         win.ntiles = static_cast<int32_t>((total + kMergeTile - 1) / kMergeTile);
         win.tile_base = ntiles;
         win.nshort = win.nlong = 0;
@@ -594,13 +721,28 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
                                            st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
     int launches = 0;
+    if (W > 1) {   // chunk ranges of the long segments
+        std::vector<int32_t> cb(2 * W, 0);
+        for (int w = 0; w < W; ++w) {
+            SD_CUDA_TRY(cudaMemcpyAsync(&cb[2 * w], p->seg_chunk + p->wins[w].seg_begin, 4, cudaMemcpyDeviceToHost, st));
+            SD_CUDA_TRY(cudaMemcpyAsync(&cb[2 * w + 1], p->seg_chunk + p->wins[w].seg_end, 4, cudaMemcpyDeviceToHost, st));
+        }
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        for (int w = 0; w < W; ++w) {
+            p->wins[w].chunk_begin = cb[2 * w];
+            p->wins[w].chunk_end = cb[2 * w + 1];
+            if (cb[2 * w + 1] > cb[2 * w]) launches += 2;
+        }
+    }
     for (int w = 0; w < W; ++w) {
         sd_plan::Window &win = p->wins[w];
-        if (win.ntiles == 0) continue;
+        if (win.short_end > win.short_begin) launches += 1;
+        if (win.single_end > win.single_begin) launches += 1;
         int32_t *table = p->tile_seg + win.tile_base + w;
         merge_table_kernel<<<ceil_div(win.ntiles + 1, 256), 256, 0, st>>>(p->m_ptr, win.seg_begin, win.seg_end, kMergeTile,
                                                                          win.ntiles, table);
         SD_CUDA_TRY(cudaGetLastError());
+        if (win.ntiles == 0) continue;
         merge_fixflag_kernel<<<ceil_div(win.ntiles, 256), 256, 0, st>>>(p->m_ptr, table, win.seg_begin, kMergeTile,
                                                                        win.ntiles, static_cast<uint8_t *>(flags_s.p),
                                                                        static_cast<uint8_t *>(flags_l.p));
@@ -802,6 +944,9 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->w_col);
     cudaFree(p->w_vals);
     cudaFree(p->w_seg_row);
+    cudaFree(p->seg_chunk);
+    cudaFree(p->chunk_ptr);
+    cudaFree(p->chunk_out);
     cudaFree(p->tile_seg);
     cudaFree(p->fix_short);
     cudaFree(p->fix_long);
@@ -973,8 +1118,12 @@ sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_
     if (colind) SD_CUDA_TRY(cudaMemcpy(colind, plan->w_col, 4 * plan->nnz, cudaMemcpyDeviceToHost));
     if (vals) SD_CUDA_TRY(cudaMemcpy(vals, plan->w_vals, es * plan->nnz, cudaMemcpyDeviceToHost));
     if (win_seg) {
-        for (size_t w = 0; w < plan->wins.size(); ++w) win_seg[w] = plan->wins[w].seg_begin;
-        win_seg[plan->wins.size()] = S;
+        for (size_t w = 0; w < plan->wins.size(); ++w) {
+            win_seg[3 * w] = plan->wins[w].seg_begin;
+            win_seg[3 * w + 1] = plan->wins[w].short_begin;
+            win_seg[3 * w + 2] = plan->wins[w].single_begin;
+        }
+        win_seg[3 * plan->wins.size()] = S;
     }
     return SD_OK;
 }
@@ -1029,6 +1178,36 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         a.S = plan->num_segments;
         for (size_t w = 0; w < plan->wins.size(); ++w) {   // windows run in order on the stream
             const sd_plan::Window &win = plan->wins[w];
+            if (win.short_end > win.short_begin) {   // short segments: one lane group per segment
+                SpmmArgs sa = a;
+                sa.ptr = a.ptr + win.short_begin;
+                sa.seg_row = a.seg_row + win.short_begin;
+                sa.S = win.short_end - win.short_begin;
+                SD_CUDA_TRY(run_segments(sa, plan->dtype, vec, false, st));
+            }
+            if (win.chunk_end > win.chunk_begin) {
+                // long segments: every chunk is summed by one lane group into its own scratch row,
+                // then each segment adds its chunks in order and updates its row of C
+                SpmmArgs ca = a;
+                ca.ptr = plan->chunk_ptr + win.chunk_begin + w;
+                ca.seg_row = nullptr;
+                ca.S = win.chunk_end - win.chunk_begin;
+                ca.C = plan->chunk_out + win.chunk_begin * N;
+                ca.ldc = N;
+                ca.alpha = 1.f;
+                ca.beta = 0.f;
+                SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, st));
+                SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->seg_chunk, a.seg_row, win.seg_begin, win.seg_end, C,
+                                             ldc, static_cast<int32_t>(N), alpha, beta, st));
+            }
+            if (win.single_end > win.single_begin) {   // one-nonzero segments: flat
+                SpmmArgs sa = a;
+                sa.seg_row = a.seg_row + win.single_begin;
+                sa.colind = a.colind + win.single_nz;
+                sa.vals = static_cast<const uint8_t *>(a.vals) + static_cast<size_t>(win.single_nz) * (plan->dtype == SD_F32 ? 4 : 2);
+                sa.S = win.single_end - win.single_begin;
+                SD_CUDA_TRY(run_single(sa, plan->dtype, vec, st));
+            }
             if (win.ntiles == 0) continue;
             MergeArgs m;
             m.s = a;

@@ -1,11 +1,34 @@
 #include "sd_launch.cuh"
 #include "sd_rowsplit.cuh"
+#include "sd_segment.cuh"
 
 namespace sd {
 
 cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
     if (dtype == SD_F32) return launch_rowsplit<float>(a, vec, st);
     return launch_rowsplit<__nv_bfloat16>(a, vec, st);
+}
+
+cudaError_t run_segments(const SpmmArgs &a, int dtype, bool vec, bool scratch, cudaStream_t st) {
+    if (dtype == SD_F32) return launch_seg<float>(a, vec, scratch, st);
+    return launch_seg<__nv_bfloat16>(a, vec, scratch, st);
+}
+
+cudaError_t run_single(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
+    if (dtype == SD_F32) return launch_single<float>(a, vec, st);
+    return launch_single<__nv_bfloat16>(a, vec, st);
+}
+
+cudaError_t run_chunk_reduce(const float *chunk_out, const int32_t *seg_chunk, const int32_t *seg_row, int64_t seg_begin,
+                             int64_t seg_end, float *C, int64_t ldc, int32_t N, float alpha, float beta, cudaStream_t st) {
+    const int64_t n = seg_end - seg_begin;
+    if (N % 4 == 0)   // scratch rows are then 16-byte aligned
+        chunk_reduce_kernel<4><<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, seg_begin,
+                                                                                 seg_end, C, ldc, N, alpha, beta, 0);
+    else
+        chunk_reduce_kernel<1><<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, seg_begin,
+                                                                                 seg_end, C, ldc, N, alpha, beta, 0);
+    return cudaGetLastError();
 }
 
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st) {

@@ -103,7 +103,32 @@ merge_tile_kernel(const MergeArgs m) {
     int j = j0;
     for (int s = s0;; ++s) {
         const int jend = (s < s1) ? (ptr_s[s + 1] - nz0) : j1;
-#pragma unroll 4
+        // batches of four nonzeros: the four gathers are in flight together
+        for (; j + 4 <= jend; j += 4) {
+            int2 it[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) it[u] = nz_s[j + u];
+            float b[4][NV][VW];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const T *brow = Bl + static_cast<int64_t>(it[u].x) * a.ldb;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    if (colok[v]) {
+                        RowLoad<T, VW>::ld(brow + v * LPR * VW, b[u][v]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < VW; ++e) b[u][v][e] = 0.f;
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < NV; ++v)
+#pragma unroll
+                    for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(__int_as_float(it[u].y), b[u][v][e], acc[v][e]);
+        }
         for (; j < jend; ++j) {
             const int2 it = nz_s[j];
             const float av = __int_as_float(it.y);
@@ -332,7 +357,6 @@ cudaError_t launch_merge(const MergeArgs &m, bool vec, int lpr, int nv, cudaStre
     constexpr int VWV = vec_width<T>::value;
     if (vec && nv == 2) {
         switch (lpr) {
-        case 4: return launch_merge_one<T, VWV, 4, 2>(m, st);
         case 8: return launch_merge_one<T, VWV, 8, 2>(m, st);
         case 16: return launch_merge_one<T, VWV, 16, 2>(m, st);
         case 32: return launch_merge_one<T, VWV, 32, 2>(m, st);

@@ -135,8 +135,10 @@ cudaError_t launch_rowsplit_one(const SpmmArgs &a, cudaStream_t st) {
 
 // Lane geometry for a dense width: VW elements per 16-byte load when `vec`, LPR lanes per
 // row (a power of two), NV vectors per lane; wider rows are covered by grid.y slabs.
-// Two vectors per lane (when the row has at least 8 vectors) halve the per-nonzero
-// instruction overhead -- index broadcast, address arithmetic -- per byte gathered.
+// Two vectors per lane halve the per-nonzero instruction overhead (index broadcast, address
+// arithmetic) per byte gathered; they are used only when a group still covers a full 128-byte
+// line with one load instruction (at least 8 lanes), because a gather instruction costs one
+// L1 tag cycle per distinct line it touches.
 struct LaneGeom {
     int vw, lpr, nv;
 };
@@ -158,7 +160,7 @@ inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw) {
         g.nv = units > 32 ? 4 : 1;
         return g;
     }
-    const bool two = units >= 8 && geom_nv_override() != 1;
+    const bool two = units >= 16 && geom_nv_override() != 1;
     const int64_t per = two ? (units + 1) / 2 : units;
     int lpr = 1;
     while (lpr < 32 && lpr < per) lpr <<= 1;
@@ -173,7 +175,6 @@ cudaError_t launch_rowsplit(const SpmmArgs &a, bool vec, cudaStream_t st) {
     const LaneGeom g = lane_geometry(a.N, vec, VWV);
     if (vec && g.nv == 2) {
         switch (g.lpr) {
-        case 4: return launch_rowsplit_one<T, VWV, 4, 2>(a, st);
         case 8: return launch_rowsplit_one<T, VWV, 8, 2>(a, st);
         case 16: return launch_rowsplit_one<T, VWV, 16, 2>(a, st);
         case 32: return launch_rowsplit_one<T, VWV, 32, 2>(a, st);

@@ -1,0 +1,287 @@
+// Group-per-segment kernels of the window-major schedule (family (b) with column windows):
+//   seg_kernel     one lane group per segment, or per chunk of a long segment
+//   single_kernel  segments of exactly one nonzero, without a pointer array
+//   chunk_reduce   adds the chunk sums of every long segment in order and updates C
+// Groups are independent: their shuffles name only the group's own lanes, so two groups of a
+// warp may run different trip counts, and the grid-stride loops need no warp-wide agreement.
+#pragma once
+
+#include "sd_common.cuh"
+#include "sd_rowsplit.cuh"
+
+namespace sd {
+
+constexpr int kSegThreads = 256;
+
+inline int sm_count_cached() {
+    static const int n = [] {
+        int dev = 0, v = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        return v;
+    }();
+    return n;
+}
+
+// SCRATCH: the segments are chunks; chunk c writes its plain sum to row c of a.C (the scratch
+// matrix).  Otherwise a.seg_row gives the output row and whether an earlier window wrote it.
+template <typename T, int VW, int LPR, int NV, bool SCRATCH>
+__global__ void __launch_bounds__(kSegThreads)
+seg_kernel(const SpmmArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int lg = threadIdx.x % LPR;
+    const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << (lane & ~(LPR - 1)));
+    const int cbase = blockIdx.y * (LPR * NV * VW);
+    const T *__restrict__ vals = static_cast<const T *>(a.vals);
+    const T *__restrict__ Bl = static_cast<const T *>(a.B) + cbase + lg * VW;
+    bool colok[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) colok[v] = cbase + (v * LPR + lg) * VW < a.N;
+    constexpr int QW = (NV * VW >= 8) ? 2 : 4;
+    constexpr int QU = LPR < QW ? LPR : QW;   // gathers in flight per lane (more would cost occupancy)
+
+    const int64_t gstride = static_cast<int64_t>(gridDim.x) * (kSegThreads / LPR);
+    for (int64_t s = (static_cast<int64_t>(blockIdx.x) * kSegThreads + threadIdx.x) / LPR; s < a.S; s += gstride) {
+        const int p0 = __ldg(a.ptr + s), p1 = __ldg(a.ptr + s + 1);
+        int32_t r = 0;
+        if (!SCRATCH) r = __ldg(a.seg_row + s);
+        float acc[NV][VW];
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
+        for (int p = p0; p < p1; p += LPR) {
+            int myc = 0;
+            float myv = 0.f;   // 0 beyond the segment's end: such products vanish
+            if (p + lg < p1) {
+                myc = __ldg(a.colind + p + lg);
+                myv = to_float(vals[p + lg]);
+            }
+            for (int q0 = 0; q0 < LPR && p + q0 < p1; q0 += QU) {
+                int cq[QU];
+                float aq[QU];
+#pragma unroll
+                for (int qq = 0; qq < QU; ++qq) {
+                    cq[qq] = (LPR == 1) ? myc : __shfl_sync(gmask, myc, q0 + qq, LPR);
+                    aq[qq] = (LPR == 1) ? myv : __shfl_sync(gmask, myv, q0 + qq, LPR);
+                }
+                float b[QU][NV][VW];
+#pragma unroll
+                for (int qq = 0; qq < QU; ++qq) {
+                    const bool valid = p + q0 + qq < p1;
+                    const T *brow = Bl + static_cast<int64_t>(cq[qq]) * a.ldb;
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        if (valid && colok[v]) {
+                            RowLoad<T, VW>::ld(brow + v * LPR * VW, b[qq][v]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < VW; ++e) b[qq][v][e] = 0.f;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int qq = 0; qq < QU; ++qq)
+#pragma unroll
+                    for (int v = 0; v < NV; ++v)
+#pragma unroll
+                        for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(aq[qq], b[qq][v][e], acc[v][e]);
+            }
+        }
+        if (SCRATCH) {
+            float *crow = a.C + s * a.ldc + cbase;
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+                if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], 1.f, 0.f, 0);
+        } else {
+            float *crow = a.C + static_cast<int64_t>(r & 0x7FFFFFFF) * a.ldc + cbase;
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+                if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], a.alpha, a.beta, r < 0 ? 1 : 0);
+        }
+    }
+}
+
+constexpr int kSingleBatch = 4;   // segments per lane group: their loads are all in flight together
+
+template <typename T, int VW, int LPR, int NV>
+__global__ void __launch_bounds__(kSegThreads)
+single_kernel(const SpmmArgs a) {
+    const int lg = threadIdx.x % LPR;
+    const int64_t g = (static_cast<int64_t>(blockIdx.x) * kSegThreads + threadIdx.x) / LPR;
+    const int cbase = blockIdx.y * (LPR * NV * VW);
+    const int64_t s0 = g * kSingleBatch;
+    if (s0 >= a.S) return;
+    const T *__restrict__ vals = static_cast<const T *>(a.vals);
+    int32_t r[kSingleBatch];
+    int c[kSingleBatch];
+    float av[kSingleBatch];
+#pragma unroll
+    for (int u = 0; u < kSingleBatch; ++u) {
+        const bool ok = s0 + u < a.S;
+        r[u] = ok ? __ldg(a.seg_row + s0 + u) : 0;
+        c[u] = ok ? __ldg(a.colind + s0 + u) : 0;
+        av[u] = ok ? a.alpha * to_float(vals[s0 + u]) : 0.f;
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int col = (v * LPR + lg) * VW;
+        if (cbase + col >= a.N) continue;
+        float b[kSingleBatch][VW], o[kSingleBatch][VW];
+#pragma unroll
+        for (int u = 0; u < kSingleBatch; ++u) {
+            RowLoad<T, VW>::ld(static_cast<const T *>(a.B) + static_cast<int64_t>(c[u]) * a.ldb + cbase + col, b[u]);
+            const bool need_c = (s0 + u < a.S) && (r[u] < 0 || a.beta != 0.f);
+            const float *crow = a.C + static_cast<int64_t>(r[u] & 0x7FFFFFFF) * a.ldc + cbase + col;
+            if constexpr (VW == 1) {
+                o[u][0] = need_c ? *crow : 0.f;
+            } else {
+#pragma unroll
+                for (int q = 0; q < VW / 4; ++q) {
+                    const float4 t = need_c ? *(reinterpret_cast<const float4 *>(crow) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    o[u][4 * q] = t.x; o[u][4 * q + 1] = t.y; o[u][4 * q + 2] = t.z; o[u][4 * q + 3] = t.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kSingleBatch; ++u) {
+            if (s0 + u >= a.S) continue;
+            const float beta = r[u] < 0 ? 1.f : a.beta;
+#pragma unroll
+            for (int e = 0; e < VW; ++e) b[u][e] = fmaf(beta, o[u][e], av[u] * b[u][e]);
+            store_cols<VW>(a.C + static_cast<int64_t>(r[u] & 0x7FFFFFFF) * a.ldc + cbase + col, b[u], 1.f, 0.f, 0);
+        }
+    }
+}
+
+// One warp per long segment: chain q of the warp adds every nchain-th chunk row, the chains
+// are then added in a fixed order (no atomics: repeated runs give identical bits).  CW columns
+// per lane (4 when N is a multiple of 4: 16-byte loads of the scratch rows).
+template <int CW>
+__global__ void __launch_bounds__(256)
+chunk_reduce_kernel(const float *__restrict__ chunk_out, const int32_t *__restrict__ seg_chunk,
+                    const int32_t *__restrict__ seg_row, int64_t seg_begin, int64_t seg_end, float *__restrict__ C,
+                    int64_t ldc, int32_t N, float alpha, float beta, int vec_c) {
+    const int lane = threadIdx.x & 31;
+    const int64_t s = seg_begin + static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+    if (s >= seg_end) return;
+    const int units = (N + CW - 1) / CW;
+    int lpc = 1;                       // lanes per chain: a power of two covering min(units, 32)
+    while (lpc < 32 && lpc < units) lpc <<= 1;
+    const int nchain = 32 / lpc, chain = lane / lpc, cl = lane % lpc;
+    const int32_t c0 = __ldg(seg_chunk + s), c1 = __ldg(seg_chunk + s + 1);
+    const int32_t r = __ldg(seg_row + s);
+    const bool accumulate = r < 0;
+    float *crow = C + static_cast<int64_t>(r & 0x7FFFFFFF) * ldc;
+    for (int ub = 0; ub < units; ub += lpc) {
+        const int col = (ub + cl) * CW;
+        float sum[CW];
+#pragma unroll
+        for (int e = 0; e < CW; ++e) sum[e] = 0.f;
+        if (col < N) {
+#pragma unroll 4
+            for (int32_t c = c0 + chain; c < c1; c += nchain) {
+                const float *p = chunk_out + static_cast<int64_t>(c) * N + col;
+                if constexpr (CW == 4) {
+                    const float4 t = *reinterpret_cast<const float4 *>(p);
+                    sum[0] += t.x; sum[1] += t.y; sum[2] += t.z; sum[3] += t.w;
+                } else {
+                    sum[0] += *p;
+                }
+            }
+        }
+        for (int off = lpc; off < 32; off <<= 1)
+#pragma unroll
+            for (int e = 0; e < CW; ++e) sum[e] += __shfl_xor_sync(0xffffffffu, sum[e], off);
+        if (chain == 0 && col < N) {
+#pragma unroll
+            for (int e = 0; e < CW; ++e) {
+                float v = alpha * sum[e];
+                if (accumulate) v += crow[col + e];
+                else if (beta != 0.f) v = fmaf(beta, crow[col + e], v);
+                crow[col + e] = v;
+            }
+        }
+    }
+    (void)vec_c;
+}
+
+template <typename T, int VW, int LPR, int NV>
+cudaError_t launch_seg_one(const SpmmArgs &a, bool scratch, cudaStream_t st) {
+    const int per_cta = kSegThreads / LPR;
+    const int64_t need = (a.S + per_cta - 1) / per_cta;
+    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * 8;   // 8 CTAs of 256 threads fill an SM
+    dim3 grid(static_cast<unsigned>(need < cap ? need : cap),
+              static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
+    if (scratch) seg_kernel<T, VW, LPR, NV, true><<<grid, kSegThreads, 0, st>>>(a);
+    else seg_kernel<T, VW, LPR, NV, false><<<grid, kSegThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_seg(const SpmmArgs &a, bool vec, bool scratch, cudaStream_t st) {
+    constexpr int VWV = vec_width<T>::value;
+    const LaneGeom g = lane_geometry(a.N, vec, VWV);
+    if (vec && g.nv == 2) {
+        switch (g.lpr) {
+        case 8: return launch_seg_one<T, VWV, 8, 2>(a, scratch, st);
+        case 16: return launch_seg_one<T, VWV, 16, 2>(a, scratch, st);
+        case 32: return launch_seg_one<T, VWV, 32, 2>(a, scratch, st);
+        }
+        return cudaErrorInvalidValue;
+    }
+#define SD_SEG_CASE(L)                                                       \
+    case L:                                                                  \
+        if (vec) return launch_seg_one<T, VWV, L, 1>(a, scratch, st);        \
+        return (g.nv == 4) ? launch_seg_one<T, 1, 32, 4>(a, scratch, st)     \
+                           : launch_seg_one<T, 1, L, 1>(a, scratch, st);
+    switch (g.lpr) {
+        SD_SEG_CASE(1)
+        SD_SEG_CASE(2)
+        SD_SEG_CASE(4)
+        SD_SEG_CASE(8)
+        SD_SEG_CASE(16)
+        SD_SEG_CASE(32)
+    }
+#undef SD_SEG_CASE
+    return cudaErrorInvalidValue;
+}
+
+template <typename T, int VW, int LPR, int NV>
+cudaError_t launch_single_one(const SpmmArgs &a, cudaStream_t st) {
+    const int per_cta = kSegThreads / LPR * kSingleBatch;
+    dim3 grid(static_cast<unsigned>((a.S + per_cta - 1) / per_cta),
+              static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
+    single_kernel<T, VW, LPR, NV><<<grid, kSegThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_single(const SpmmArgs &a, bool vec, cudaStream_t st) {
+    constexpr int VWV = vec_width<T>::value;
+    const LaneGeom g = lane_geometry(a.N, vec, VWV);
+    if (vec && g.nv == 2) {
+        switch (g.lpr) {
+        case 8: return launch_single_one<T, VWV, 8, 2>(a, st);
+        case 16: return launch_single_one<T, VWV, 16, 2>(a, st);
+        case 32: return launch_single_one<T, VWV, 32, 2>(a, st);
+        }
+        return cudaErrorInvalidValue;
+    }
+#define SD_SG_CASE(L)                                                \
+    case L:                                                          \
+        if (vec) return launch_single_one<T, VWV, L, 1>(a, st);      \
+        return (g.nv == 4) ? launch_single_one<T, 1, 32, 4>(a, st)   \
+                           : launch_single_one<T, 1, L, 1>(a, st);
+    switch (g.lpr) {
+        SD_SG_CASE(1)
+        SD_SG_CASE(2)
+        SD_SG_CASE(4)
+        SD_SG_CASE(8)
+        SD_SG_CASE(16)
+        SD_SG_CASE(32)
+    }
+#undef SD_SG_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace sd

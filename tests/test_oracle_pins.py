@@ -436,7 +436,8 @@ def test_o4_window_segments_against_python_sets():
     lengths[7] = 0
     lengths[20] = 90
     wl = W.random_csr(M, K, 1, lengths, seed=3)
-    seg_ptr, seg_row, perm, win_seg = oracle.window_segments(wl.rowptr, wl.colind, M, K, 4)
+    short_len = 5
+    seg_ptr, seg_row, perm, bounds = oracle.window_segments(wl.rowptr, wl.colind, M, K, 4, short_len)
     wcols = -(-K // 4)
     # brute force: dictionary (window, row) -> positions
     groups = {}
@@ -444,23 +445,36 @@ def test_o4_window_segments_against_python_sets():
         for p in range(wl.rowptr[i], wl.rowptr[i + 1]):
             groups.setdefault((wl.colind[p] // wcols, i), []).append(p)
     empties = [i for i in range(M) if lengths[i] == 0]
-    keys = sorted(groups)
-    assert len(seg_row) == len(empties) + len(keys)
-    assert [int(r) for r in seg_row[:len(empties)]] == empties
-    assert np.all(seg_ptr[:len(empties) + 1] == 0)
+    # expected order: by (window, class), long first; inside window 0's short class the empty
+    # rows come before the other rows; rows ascending inside a class
+    want = []
+    for win in range(4):
+        runs = sorted((row, ps) for (w2, row), ps in groups.items() if w2 == win)
+        want += [(win, row, ps) for row, ps in runs if len(ps) > short_len]
+        if win == 0:
+            want += [(0, row, []) for row in empties]
+        want += [(win, row, ps) for row, ps in runs if 2 <= len(ps) <= short_len]
+        want += [(win, row, ps) for row, ps in runs if len(ps) == 1]
+    assert len(seg_row) == len(want) == bounds[-1]
     q = 0
-    for s, (win, row) in enumerate(keys, start=len(empties)):
+    for s, (win, row, ps) in enumerate(want):
         assert seg_ptr[s] == q
-        first_w = wl.colind[wl.rowptr[row]] // wcols
         assert (int(seg_row[s]) & 0x7FFFFFFF) == row
-        assert bool(int(seg_row[s]) & 0x80000000) == (first_w != win)
-        assert perm[q:q + len(groups[(win, row)])].tolist() == groups[(win, row)]
-        q += len(groups[(win, row)])
+        if ps:
+            first_w = wl.colind[wl.rowptr[row]] // wcols
+            assert bool(int(seg_row[s]) & 0x80000000) == (first_w != win)
+        assert perm[q:q + len(ps)].tolist() == ps
+        q += len(ps)
     assert seg_ptr[-1] == q == wl.nnz
     assert sorted(perm.tolist()) == list(range(wl.nnz))
-    for wdx in range(5):
-        want = len(empties) + sum(1 for k in keys if k[0] < wdx) if wdx > 0 else 0
-        assert win_seg[wdx] == want
+    pos = 0
+    for win in range(4):
+        nlong = sum(1 for x in want if x[0] == win and len(x[2]) > short_len)
+        nsingle = sum(1 for x in want if x[0] == win and len(x[2]) == 1)
+        nall = sum(1 for x in want if x[0] == win)
+        assert bounds[3 * win] == pos and bounds[3 * win + 1] == pos + nlong
+        assert bounds[3 * win + 2] == pos + nall - nsingle
+        pos += nall
 
 
 def test_o4_window_rule():
