@@ -189,6 +189,30 @@ sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_
  * *status (0 = no wait ever expired) and clears it. */
 sd_status_t sd_plan_device_status(sd_plan_t *plan, int32_t *status);
 
+/* sd_spmm_merge_static -- (no counterpart in the paper: an addition of this library.)
+ * C = alpha*A*B + beta*C with the merge-path kernels, fp32, straight from the CSR arrays and
+ * WITHOUT ANY ALLOCATION.  It is meant for callers that cannot let a library allocate device
+ * memory: processes whose framework has already claimed the GPU's free memory for its own
+ * pool, so that a late cudaMalloc fails or fragments it; latency-critical loops that cannot
+ * take cudaMalloc's device-wide synchronisation; code under a fixed memory budget.  A plan
+ * allocates its tile table and carry-out rows; here they live in one fixed 4 MiB array inside
+ * the library's device image (every GPU that loads the library holds it until exit).
+ *   rowptr [M+1], colind [nnz], vals [nnz]   device, as for sd_plan_create; nnz = rowptr[M]
+ *                                            is passed in so that nothing is read back
+ *   B device [K, ldb] fp32, C device [M, ldc] fp32, ldb, ldc >= N; alpha/beta as sd_spmm.
+ * Size limit: with T = ceil((M + nnz) / 1024) tiles, 4*(T+1) rounded up to 256, plus 8*T*N
+ * bytes, must fit in 4 MiB (N = 32: about 16 million rows + nonzeros); beyond that the call
+ * returns SD_ERR_UNSUPPORTED with the numbers in sd_last_error and launches nothing.
+ * The first call on each device looks up the array's device address; make that first call
+ * before any stream capture begins on the device.  All calls share the one array, which keeps
+ * the previous call's contents (the call clears the part that must start from zero): two calls
+ * whose kernels overlap on the GPU -- different streams, or different host threads -- race on
+ * it and corrupt each other's results, so serialise them.  Asynchronous on `stream`. */
+sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, const float *vals,
+                                 int64_t M, int64_t K, int64_t N, int64_t nnz, const float *B,
+                                 int64_t ldb, float *C, int64_t ldc, float alpha, float beta,
+                                 void *stream);
+
 /* sd_last_error -- copy the calling thread's last error text into buf (NUL-terminated,
  * at most n bytes); returns the last status code. */
 int sd_last_error(char *buf, size_t n);

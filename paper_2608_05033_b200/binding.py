@@ -22,7 +22,7 @@ SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_last_error",
+           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_last_error",
            "sd_version"]
 
 
@@ -86,6 +86,9 @@ def load():
     lib.sd_plan_get_segments.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_device_status.restype = C.c_int
     lib.sd_plan_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+    lib.sd_spmm_merge_static.restype = C.c_int
+    lib.sd_spmm_merge_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
+                                         C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_void_p]
     lib.sd_last_error.restype = C.c_int
     lib.sd_last_error.argtypes = [C.c_char_p, C.c_size_t]
     lib.sd_version.restype = C.c_char_p
@@ -156,6 +159,16 @@ def sd_spmm(plan, B, ldb: int, Cmat, ldc: int, alpha: float, beta: float, stream
 
 def sd_spmm_host(plan, B_host, ldb: int, C_host, ldc: int, alpha: float, beta: float):
     rc = load().sd_spmm_host(plan, _ptr(B_host), ldb, _ptr(C_host), ldc, alpha, beta)
+    if rc != SD_OK:
+        _raise(rc)
+
+
+def sd_spmm_merge_static(rowptr, colind, vals, M: int, K: int, N: int, nnz: int, B, ldb: int, Cmat, ldc: int,
+                         alpha: float, beta: float, stream=None):
+    """Merge-path SpMM without a plan and without any allocation (fixed 4 MiB scratch inside the
+    library; see include/sd.h for the size limit and the sharing rules)."""
+    rc = load().sd_spmm_merge_static(_ptr(rowptr), _ptr(colind), _ptr(vals), M, K, N, nnz, _ptr(B), ldb, _ptr(Cmat),
+                                     ldc, alpha, beta, _stream_handle(stream))
     if rc != SD_OK:
         _raise(rc)
 
