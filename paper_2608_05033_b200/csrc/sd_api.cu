@@ -398,6 +398,9 @@ struct sd_plan {
     int32_t *chunk_ptr = nullptr;   // per window: nonzero boundaries of its chunks, one terminator each
     float *chunk_out = nullptr;     // [chunks][N] partial sums of the chunks
     int64_t num_chunks = 0;
+    // window-major plans run the three independent segment classes of a window side by side
+    cudaStream_t aux[2] = {nullptr, nullptr};
+    cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr};
     struct Window {
         int64_t seg_begin, seg_end;     // segments of the merge-path kernel (all of them without windows)
         int64_t short_begin, short_end; // segments of the group-per-segment kernel (windows only)
@@ -721,6 +724,13 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
                                            st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
     int launches = 0;
+    if (W > 1) {
+        for (int i = 0; i < 2; ++i) {
+            SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
+            SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
+        }
+        SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+    }
     if (W > 1) {   // chunk ranges of the long segments
         std::vector<int32_t> cb(2 * W, 0);
         for (int w = 0; w < W; ++w) {
@@ -960,6 +970,11 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->stage_B);
     cudaFree(p->stage_C);
     if (p->host_stream) cudaStreamDestroy(p->host_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (p->aux[i]) cudaStreamDestroy(p->aux[i]);
+        if (p->ev_join[i]) cudaEventDestroy(p->ev_join[i]);
+    }
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     delete p;
 }
 
@@ -1176,14 +1191,24 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         a.vals = plan->m_vals;
         a.seg_row = plan->m_seg_row;
         a.S = plan->num_segments;
-        for (size_t w = 0; w < plan->wins.size(); ++w) {   // windows run in order on the stream
+        const bool side = plan->wins.size() > 1 && plan->aux[0] && !getenv("SD_NO_SIDE_STREAMS");
+        for (size_t w = 0; w < plan->wins.size(); ++w) {   // windows run in order
             const sd_plan::Window &win = plan->wins[w];
-            if (win.short_end > win.short_begin) {   // short segments: one lane group per segment
-                SpmmArgs sa = a;
-                sa.ptr = a.ptr + win.short_begin;
-                sa.seg_row = a.seg_row + win.short_begin;
-                sa.S = win.short_end - win.short_begin;
-                SD_CUDA_TRY(run_segments(sa, plan->dtype, vec, false, st));
+            // Inside a window every row belongs to one segment, so the three classes touch disjoint
+            // rows of C and may run side by side: short and one-nonzero segments go to two plan-owned
+            // streams forked from the caller's stream and joined before the next window.
+            const bool has_short = win.short_end > win.short_begin, has_single = win.single_end > win.single_begin;
+            cudaStream_t s_short = st, s_single = st;
+            if (side && (has_short || has_single)) {
+                SD_CUDA_TRY(cudaEventRecord(plan->ev_fork, st));
+                if (has_short) {
+                    s_short = plan->aux[0];
+                    SD_CUDA_TRY(cudaStreamWaitEvent(s_short, plan->ev_fork, 0));
+                }
+                if (has_single) {
+                    s_single = plan->aux[1];
+                    SD_CUDA_TRY(cudaStreamWaitEvent(s_single, plan->ev_fork, 0));
+                }
             }
             if (win.chunk_end > win.chunk_begin) {
                 // long segments: every chunk is summed by one lane group into its own scratch row,
@@ -1200,13 +1225,28 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
                 SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->seg_chunk, a.seg_row, win.seg_begin, win.seg_end, C,
                                              ldc, static_cast<int32_t>(N), alpha, beta, st));
             }
-            if (win.single_end > win.single_begin) {   // one-nonzero segments: flat
+            if (has_short) {   // short segments: one lane group per segment
+                SpmmArgs sa = a;
+                sa.ptr = a.ptr + win.short_begin;
+                sa.seg_row = a.seg_row + win.short_begin;
+                sa.S = win.short_end - win.short_begin;
+                SD_CUDA_TRY(run_segments(sa, plan->dtype, vec, false, s_short));
+            }
+            if (has_single) {   // one-nonzero segments: flat
                 SpmmArgs sa = a;
                 sa.seg_row = a.seg_row + win.single_begin;
                 sa.colind = a.colind + win.single_nz;
                 sa.vals = static_cast<const uint8_t *>(a.vals) + static_cast<size_t>(win.single_nz) * (plan->dtype == SD_F32 ? 4 : 2);
                 sa.S = win.single_end - win.single_begin;
-                SD_CUDA_TRY(run_single(sa, plan->dtype, vec, st));
+                SD_CUDA_TRY(run_single(sa, plan->dtype, vec, s_single));
+            }
+            if (s_short != st) {
+                SD_CUDA_TRY(cudaEventRecord(plan->ev_join[0], s_short));
+                SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[0], 0));
+            }
+            if (s_single != st) {
+                SD_CUDA_TRY(cudaEventRecord(plan->ev_join[1], s_single));
+                SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[1], 0));
             }
             if (win.ntiles == 0) continue;
             MergeArgs m;

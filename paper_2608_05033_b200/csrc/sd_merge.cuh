@@ -103,14 +103,15 @@ merge_tile_kernel(const MergeArgs m) {
     int j = j0;
     for (int s = s0;; ++s) {
         const int jend = (s < s1) ? (ptr_s[s + 1] - nz0) : j1;
-        // batches of four nonzeros: the four gathers are in flight together
-        for (; j + 4 <= jend; j += 4) {
-            int2 it[4];
+        // batches of WB nonzeros: their gathers are all in flight together
+        constexpr int WB = 4;
+        for (; j + WB <= jend; j += WB) {
+            int2 it[WB];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) it[u] = nz_s[j + u];
-            float b[4][NV][VW];
+            for (int u = 0; u < WB; ++u) it[u] = nz_s[j + u];
+            float b[WB][NV][VW];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < WB; ++u) {
                 const T *brow = Bl + static_cast<int64_t>(it[u].x) * a.ldb;
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
@@ -123,7 +124,7 @@ merge_tile_kernel(const MergeArgs m) {
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < WB; ++u)
 #pragma unroll
                 for (int v = 0; v < NV; ++v)
 #pragma unroll

@@ -138,7 +138,9 @@ cudaError_t launch_rowsplit_one(const SpmmArgs &a, cudaStream_t st) {
 // Two vectors per lane halve the per-nonzero instruction overhead (index broadcast, address
 // arithmetic) per byte gathered; they are used only when a group still covers a full 128-byte
 // line with one load instruction (at least 8 lanes), because a gather instruction costs one
-// L1 tag cycle per distinct line it touches.
+// L1 tag cycle per distinct line it touches.  The row-split kernel gains from them (short rows:
+// fewer instructions per byte); the merge-path and segment kernels measure faster with one
+// vector per lane and more lanes per row (`prefer_two` = false).
 struct LaneGeom {
     int vw, lpr, nv;
 };
@@ -149,7 +151,7 @@ inline int geom_nv_override() {
     }();
     return v;
 }
-inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw) {
+inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw, bool prefer_two = true) {
     LaneGeom g;
     g.vw = vec ? vecw : 1;
     const int64_t units = (N + g.vw - 1) / g.vw;
@@ -160,7 +162,7 @@ inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw) {
         g.nv = units > 32 ? 4 : 1;
         return g;
     }
-    const bool two = units >= 16 && geom_nv_override() != 1;
+    const bool two = prefer_two && units >= 16 && geom_nv_override() != 1;
     const int64_t per = two ? (units + 1) / 2 : units;
     int lpr = 1;
     while (lpr < 32 && lpr < per) lpr <<= 1;

@@ -67,7 +67,10 @@ seg_kernel(const SpmmArgs a) {
                 float b[QU][NV][VW];
 #pragma unroll
                 for (int qq = 0; qq < QU; ++qq) {
-                    const bool valid = p + q0 + qq < p1;
+                    // chunks: an entry beyond the end has column 0 and value 0, so it may be gathered
+                    // unconditionally (only a segment's last chunk has such entries); short segments
+                    // would waste most of their gathers that way and keep the test
+                    const bool valid = SCRATCH || (p + q0 + qq < p1);
                     const T *brow = Bl + static_cast<int64_t>(cq[qq]) * a.ldb;
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
@@ -220,7 +223,7 @@ cudaError_t launch_seg_one(const SpmmArgs &a, bool scratch, cudaStream_t st) {
 template <typename T>
 cudaError_t launch_seg(const SpmmArgs &a, bool vec, bool scratch, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
-    const LaneGeom g = lane_geometry(a.N, vec, VWV);
+    const LaneGeom g = lane_geometry(a.N, vec, VWV, false);
     if (vec && g.nv == 2) {
         switch (g.lpr) {
         case 8: return launch_seg_one<T, VWV, 8, 2>(a, scratch, st);
@@ -258,7 +261,7 @@ cudaError_t launch_single_one(const SpmmArgs &a, cudaStream_t st) {
 template <typename T>
 cudaError_t launch_single(const SpmmArgs &a, bool vec, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
-    const LaneGeom g = lane_geometry(a.N, vec, VWV);
+    const LaneGeom g = lane_geometry(a.N, vec, VWV, false);
     if (vec && g.nv == 2) {
         switch (g.lpr) {
         case 8: return launch_single_one<T, VWV, 8, 2>(a, st);
