@@ -797,10 +797,11 @@ static sd_status_t build_bsr(sd_plan *p, const unsigned long long *ukeys, int64_
     bsr_bcol_kernel<<<ceil_div(nnzb, 256), 256, 0, st>>>(ukeys, nnzb, Kb, p->bcol);
     SD_CUDA_TRY(cudaGetLastError());
     SD_CUDA_TRY(p->dtype == SD_F32 ? fill_bsr<float>(p, st) : fill_bsr<__nv_bfloat16>(p, st));
-    if (p->dtype == SD_BF16) {
-        if ((s = dev_alloc(p, &p->bval_mma, es * 256 * nnzb, "bval (tensor-core image)"))) return s;
-        SD_CUDA_TRY(build_bsr_mma_image(p->bval, p->bval_mma, nnzb, p->dtype, st));
-    }
+    // tensor-core operand images: bf16 512 bytes per block, fp32 a hi and a lo image of 1 KB each
+    if ((s = dev_alloc(p, &p->bval_mma, (p->dtype == SD_BF16 ? 512 : 2048) * static_cast<size_t>(nnzb),
+                       "bval (tensor-core image)")))
+        return s;
+    SD_CUDA_TRY(build_bsr_mma_image(p->bval, p->bval_mma, nnzb, p->dtype, st));
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->dev_error), sizeof(int32_t), "error word"))) return s;
     SD_CUDA_TRY(cudaMemsetAsync(p->dev_error, 0, sizeof(int32_t), st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));

@@ -6,16 +6,23 @@
 // tcgen05.mma needs M = 64 or 128, while a block is only 16 rows high, so the product is
 // taken transposed: D[c, r] = sum_k  B[16J + k, n0 + c] * Ablk[r, k]  with
 //     M = 128 dense columns c   (MMA operand "A" = a 16 x 128 slab of B, MN-major, 128B swizzle,
-//                                exactly the image a 2-D TMA box load leaves in shared memory)
-//     N = 16 block rows r       (MMA operand "B" = the block, K-major)
-//     K = 16 block columns k    (one instruction per block for bf16).
+//                                exactly the image a TMA box load leaves in shared memory)
+//     N = 16 block rows r       (MMA operand "B" = the block, K-major, unswizzled 8-row cores)
+//     K = 16 (bf16, kind::f16) or 8 (fp32 as tf32, kind::tf32: two steps per block).
 // The accumulator D sits in TMEM with the dense column on the lane axis, so an epilogue warp
 // reading lane l, column r holds C[16I + r, n0 + l]: for a fixed r the 32 lanes of a warp write
 // 32 consecutive floats of C.
 //
-// Persistent CTAs, two per SM.  Warp 0: TMA producer.  Warp 1: TMEM owner + MMA issuer.
-// Warps 2..5: epilogue (TMEM -> registers -> alpha/beta -> C).  Every wait is bounded: on
-// expiry the CTA records an error word, drains, frees its TMEM and returns.
+// fp32 values cannot go through one tf32 pass (10 mantissa bits: 2^-11 operand rounding, far
+// outside the 1e-5 tolerance).  Both operands are split x = hi + lo with hi = x with its low 13
+// mantissa bits cleared (exact in tf32) and lo = x - hi (exact in fp32); three products
+// hi*hi + lo*hi + hi*lo are accumulated in fp32, the dropped lo*lo term is below 2^-22 |x||y|.
+// The blocks are split at plan time; the slab of B is split in shared memory by converter warps.
+//
+// Persistent CTAs.  Warp 0: TMA producer.  Warp 1: TMEM owner + MMA issuer.  Warps 2..5:
+// epilogue (TMEM -> registers -> alpha/beta -> C).  Warps 6..9 (fp32 only): converters.  A ring
+// slot ("stage") holds up to `sb` blocks that share one barrier round trip.  Every wait is
+// bounded: on expiry the CTA records an error word, drains, frees its TMEM and returns.
 #pragma once
 
 #include <cuda.h>
@@ -25,23 +32,21 @@
 
 namespace sd {
 
-constexpr int kTcThreads = 192;
-constexpr int kTcStages = 22;                // most ring slots a CTA may use
-constexpr int kTcDefaultStages = 10;         // ring slots per CTA: two CTAs share an SM, because one
-constexpr int kTcCtasPerSm = 2;              // producer/issuer pair is bound by its own handshake latency
-
-constexpr int kTcStageBytes = 9 * 1024;      // 4 boxes of 2 KB (B slab, 256 columns) + the block image
-constexpr int kTcBlockOff = 8 * 1024;        // offset of the block image inside a stage
+constexpr int kTcMaxStages = 24;             // most ring slots a CTA may use
 constexpr int kTcSlabCols = 256;             // dense columns per work item (two M = 128 tiles)
 constexpr int kTcTmemCols = 64;              // 2 accumulator slots x 2 tiles x 16 columns
-constexpr int kTcBatchItems = 64;             // work items whose metadata is staged at once
-constexpr int kTcBatchBlocks = 2048;          // block columns staged per batch
+constexpr int kTcBatchItems = 64;            // work items whose metadata is staged at once
+constexpr int kTcBatchBlocks = 2048;         // block columns staged per batch
 constexpr uint32_t kTcSpinLimit = 1u << 20;  // mbarrier polls before a wait gives up
+
+// shared-memory bytes of one block inside a stage
+constexpr int kTcBlkBytesBf16 = 8192 + 1024;          // slab 16 x 256 bf16, block image (512 B, padded)
+constexpr int kTcBlkBytesTf32 = 16384 + 16384 + 2048; // slab hi (in place of raw), slab lo, block hi + lo
 
 struct TcArgs {
     const int32_t *browptr;
     const int32_t *bcol;
-    const void *bmma;       // [nnzb] MMA-ready block images
+    const void *bmma;       // [nnzb] MMA-ready block images (bf16: 512 B, fp32: hi 1 KB + lo 1 KB)
     float *C;
     int64_t ldc;
     int64_t M;
@@ -50,11 +55,9 @@ struct TcArgs {
     int32_t nslab;          // ceil(N / 256)
     float alpha, beta;
     int32_t *error;         // device word: 0 = fine, else the first wait that expired
-    uint32_t lbo_a, sbo_a, lbo_b, sbo_b;   // shared-memory descriptor strides (bytes)
-    int32_t map3d;          // the tensor map is the 3-D view {64 columns, K rows, N/64 groups}
-    int32_t box_bytes;      // bytes one 3-D box copy delivers
-    int32_t debug;          // bench-only experiment switches (0 in production)
-    int32_t stages;         // ring slots in use (<= kTcStages)
+    int32_t box_bytes;      // bytes one TMA box copy delivers
+    int32_t stages;         // ring slots in use
+    int32_t sb;             // blocks per ring slot
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -81,34 +84,16 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ int g_tc_test_wait = 0;
 // Bounded wait.  Returns false when the limit ran out or another warp already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error,
                                           int code) {
     for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
-        if (g_tc_test_wait ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
     *abort_flag = 1;
     atomicCAS(error, 0, code);
     return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
-        : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
     asm volatile(
@@ -126,14 +111,23 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                           uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
+template <bool TF32>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if constexpr (TF32) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&r)[16]) {
     uint32_t u[16];
@@ -149,26 +143,33 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&r)[16]) {
 }
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4),
-// the fixed field of this architecture, and the swizzle mode (0 none, 2 = 128 B).
+// the fixed field of this architecture, and the swizzle mode (0 none, 1 = 128 B with 32-byte
+// atoms, 2 = 128 B).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t swizzle) {
     return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo >> 4) << 16) |
            (static_cast<uint64_t>(sbo >> 4) << 32) | (1ull << 46) | (static_cast<uint64_t>(swizzle) << 61);
 }
 
-// Instruction descriptor, kind::f16 with bf16 inputs: D = f32, A = B = bf16, A MN-major,
-// B K-major, N = 16, M = 128.
-constexpr uint32_t kIdescBf16 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) | ((16u >> 3) << 17) |
-                                ((128u >> 4) << 24);
+// Instruction descriptors: D = f32, A MN-major, B K-major, N = 16, M = 128;
+// kind::f16 with A = B = bf16 (format 1), kind::tf32 with A = B = tf32 (format 2).
+constexpr uint32_t kIdescBf16 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescTf32 = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
 
-__global__ void __launch_bounds__(kTcThreads, 2)
-bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
+template <bool TF32>
+__global__ void __launch_bounds__(TF32 ? 320 : 192, TF32 ? 1 : 2)
+bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
+    constexpr int kThreads = TF32 ? 320 : 192;
+    constexpr int kBlk = TF32 ? kTcBlkBytesTf32 : kTcBlkBytesBf16;   // bytes of one block in a stage
+    constexpr int kImgOff = TF32 ? 32768 : 8192;                       // block image inside a block's bytes
+    constexpr int kImgBytes = TF32 ? 2048 : 512;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // stage ring first (1024-byte aligned for the 128-byte swizzle), barriers after it
+    // stage ring first (1024-byte aligned for the 128-byte swizzle), barriers and metadata after it
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + a.stages * kTcStageBytes);
-    uint64_t *full = bars, *empty = bars + kTcStages, *acc_full = bars + 2 * kTcStages,
-             *acc_empty = bars + 2 * kTcStages + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kTcStages + 4);
+    const int stage_bytes = a.sb * kBlk;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + a.stages * stage_bytes);
+    uint64_t *full = bars, *empty = bars + kTcMaxStages, *conv = bars + 2 * kTcMaxStages,
+             *acc_full = bars + 3 * kTcMaxStages, *acc_empty = bars + 3 * kTcMaxStages + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * kTcMaxStages + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     int32_t *meta_b0 = reinterpret_cast<int32_t *>(tmem_slot + 2);
     int32_t *meta_nblk = meta_b0 + kTcBatchItems;
@@ -179,6 +180,7 @@ bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
         for (int s = 0; s < a.stages; ++s) {
             mbar_init(smem_u32(full + s), 1);
             mbar_init(smem_u32(empty + s), 1);
+            mbar_init(smem_u32(conv + s), 4);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(acc_full + s), 1);
@@ -200,14 +202,13 @@ bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
     const uint32_t tmem_base = *tmem_slot;
 
     const int nitems = a.Mb * a.nslab;
-
     // Block-row pointers and block columns live in global memory.  A dependent global load
     // between two blocks would serialise the pipeline on memory latency, so the CTA first
     // brings the metadata of a batch of its work items into shared memory (all threads, two
-    // overlapped round trips), then the three roles run through the batch from there.
+    // overlapped round trips), then the roles run through the batch from there.
     const int my_items = (nitems - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
-    uint32_t p_stage = 0, p_phase = 0, p_filled = 0, p_fill_parity = 0;   // producer ring state
-    uint32_t m_stage = 0, m_phase = 0;                                   // MMA ring state
+    uint32_t p_stage = 0, p_phase = 0, p_issued = 0;                     // producer ring state
+    uint32_t m_stage = 0, m_phase = 0;                                   // consumer ring state (MMA, converters)
     uint32_t it = 0;                                                      // items done (accumulator slot / parity)
     bool ok = true;
 
@@ -217,94 +218,146 @@ bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
             __syncthreads();                       // everybody is done with the previous batch's metadata
             if (*abort_flag) break;                // uniform: read after the barrier
         }
-        for (int j = threadIdx.x; j < bn; j += kTcThreads) {
+        for (int j = threadIdx.x; j < bn; j += kThreads) {
             const int I = (blockIdx.x + (batch0 + j) * gridDim.x) / a.nslab;
             const int b0 = __ldg(a.browptr + I);
             meta_b0[j] = b0;
             meta_nblk[j] = __ldg(a.browptr + I + 1) - b0;
         }
         __syncthreads();
-        {
-            int off = 0;
-            for (int j = 0; j < bn; ++j) {
-                const int nb = meta_nblk[j], b0 = meta_b0[j];
-                for (int k = threadIdx.x; k < nb && off + k < kTcBatchBlocks; k += kTcThreads)
-                    meta_col[off + k] = __ldg(a.bcol + b0 + k);
-                off += nb;
-            }
+        int total = 0;   // blocks of the batch (every thread computes it)
+        for (int j = 0; j < bn; ++j) {
+            const int nb = meta_nblk[j], b0 = meta_b0[j];
+            for (int k = threadIdx.x; k < nb && total + k < kTcBatchBlocks; k += kThreads)
+                meta_col[total + k] = __ldg(a.bcol + b0 + k);
+            total += nb;
         }
         __syncthreads();
 
         if (warp == 0) {
             // -------------------------------------------------------------- TMA producer
             if (lane == 0) {
-                int off = 0;
-                for (int j = 0; j < bn && ok; ++j) {
-                    const int item = blockIdx.x + (batch0 + j) * gridDim.x;
-                    const int n0 = (item % a.nslab) * kTcSlabCols;
-                    const int mt_n = min(2, (a.N - n0 + 127) / 128);
-                    const int nb = meta_nblk[j], b0 = meta_b0[j];
-                    for (int k = 0; k < nb; ++k) {
-                        const int krow = ((off + k < kTcBatchBlocks) ? meta_col[off + k] : __ldg(a.bcol + b0 + k)) * 16;
-                        if (!(ok = mbar_wait(smem_u32(empty + p_stage), p_phase ^ 1, abort_flag, a.error, 1))) break;
-                        p_filled |= 1u << p_stage;
-                        p_fill_parity = (p_fill_parity & ~(1u << p_stage)) | (p_phase << p_stage);
-                        const uint32_t sbase = smem_u32(smem + p_stage * kTcStageBytes);
-                        const uint32_t fb = smem_u32(full + p_stage);
-                        const uint32_t slab_bytes = (a.debug & 8) ? 0u : (a.map3d ? a.box_bytes : mt_n * 4096);
-                        mbar_expect_tx(fb, slab_bytes + ((a.debug & 4) ? 0u : 512u));
-                        if (a.debug & 8) {
-                        } else if (a.map3d) {
-                            // one copy brings all 64-column groups of the slab: [group][16 rows][128 B]
-                            tma_load_3d(sbase, &tmapB, 0, krow, n0 / 64, fb);
-                        } else {
-                            for (int h = 0; h < 2 * mt_n; ++h) tma_load_2d(sbase + h * 2048, &tmapB, n0 + h * 64, krow, fb);
+                // This thread runs alone in its warp, so every instruction of the per-block path costs
+                // its full issue latency: per-item values are computed when the item changes, and
+                // addresses advance by addition.
+                int j = -1, k = 0, nbj = 0, zc = 0;
+                const uint8_t *img = nullptr;
+                const uint32_t ring0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
+                const uint32_t tx1 = static_cast<uint32_t>(a.box_bytes + kImgBytes);
+                for (int fb = 0; fb < total && ok; fb += a.sb) {
+                    const int cnt = min(a.sb, total - fb);
+                    if (!(ok = mbar_wait(empty0 + p_stage * 8, p_phase ^ 1, abort_flag, a.error, 1))) break;
+                    ++p_issued;
+                    uint32_t dst = ring0 + p_stage * stage_bytes;
+                    const uint32_t fbar = full0 + p_stage * 8;
+                    mbar_expect_tx(fbar, cnt * tx1);
+                    for (int u = 0; u < cnt; ++u) {
+                        while (k == nbj) {   // next item with blocks
+                            ++j;
+                            k = 0;
+                            nbj = meta_nblk[j];
+                            const int item = blockIdx.x + (batch0 + j) * gridDim.x;
+                            zc = (a.nslab == 1 ? 0 : (item % a.nslab) * kTcSlabCols) / (TF32 ? 32 : 64);
+                            img = static_cast<const uint8_t *>(a.bmma) + static_cast<int64_t>(meta_b0[j]) * kImgBytes;
                         }
-                        if (!(a.debug & 4))
-                            bulk_load(sbase + kTcBlockOff,
-                                      static_cast<const uint8_t *>(a.bmma) + static_cast<int64_t>(b0 + k) * 512, 512, fb);
-                        if (++p_stage == a.stages) {
-                            p_stage = 0;
-                            p_phase ^= 1;
-                        }
+                        const int flat = fb + u;
+                        const int krow = ((flat < kTcBatchBlocks) ? meta_col[flat] : __ldg(a.bcol + meta_b0[j] + k)) * 16;
+                        // one copy brings all column groups of the slab: [group][16 rows][128 B]
+                        tma_load_3d(dst, &tmapB, 0, krow, zc, fbar);
+                        bulk_load(dst + kImgOff, img, kImgBytes, fbar);
+                        img += kImgBytes;
+                        dst += kBlk;
+                        ++k;
                     }
-                    off += nb;
+                    if (++p_stage == static_cast<uint32_t>(a.stages)) {
+                        p_stage = 0;
+                        p_phase ^= 1;
+                    }
                 }
             }
         } else if (warp == 1) {
             // -------------------------------------------------------------- MMA issuer
             if (lane == 0) {
-                uint32_t mit = it;
-                for (int j = 0; j < bn && ok; ++j, ++mit) {
-                    const int item = blockIdx.x + (batch0 + j) * gridDim.x;
-                    const int n0 = (item % a.nslab) * kTcSlabCols;
-                    const int mt_n = min(2, (a.N - n0 + 127) / 128);
-                    const int nb = meta_nblk[j];
-                    const uint32_t as = mit & 1, aphase = (mit >> 1) & 1;
-                    if (!(ok = mbar_wait(smem_u32(acc_empty + as), aphase ^ 1, abort_flag, a.error, 2))) break;
+                int j = 0, k = 0;
+                uint32_t ms = m_stage, mp = m_phase;
+                // items without blocks produce no MMA: their accumulator is simply declared ready
+                auto skip_empty_items = [&]() {
+                    while (ok && j < bn && meta_nblk[j] == 0) {
+                        const uint32_t as = (it + j) & 1, aphase = ((it + j) >> 1) & 1;
+                        if (!(ok = mbar_wait(smem_u32(acc_empty + as), aphase ^ 1, abort_flag, a.error, 2))) break;
+                        mbar_arrive(smem_u32(acc_full + as));
+                        ++j;
+                    }
+                };
+                skip_empty_items();
+                // descriptors differ from block to block only in their start-address field
+                const uint64_t a_hi0 = smem_desc(0, 2048, TF32 ? 512 : 1024, TF32 ? 1 : 2);
+                const uint64_t b_hi0 = smem_desc(0, 256, 128, 0);
+                const uint32_t ring0 = smem_u32(smem), wait0 = smem_u32(TF32 ? conv : full), empty0 = smem_u32(empty);
+                const uint32_t accf0 = smem_u32(acc_full), acce0 = smem_u32(acc_empty);
+                int mt_n = 2, nbj = (j < bn) ? meta_nblk[j] : 0;
+                uint32_t as = 0, d0 = 0;
+                auto enter_item = [&]() {   // per-item values, when the first block of item j comes up
+                    as = (it + j) & 1;
+                    d0 = tmem_base + as * 32;
+                    nbj = meta_nblk[j];
+                    if (a.nslab == 1) {
+                        mt_n = min(2, (a.N + 127) / 128);
+                    } else {
+                        const int item = blockIdx.x + (batch0 + j) * gridDim.x;
+                        mt_n = min(2, (a.N - (item % a.nslab) * kTcSlabCols + 127) / 128);
+                    }
+                    return mbar_wait(acce0 + as * 8, (((it + j) >> 1) & 1) ^ 1, abort_flag, a.error, 2);
+                };
+                for (int fb = 0; fb < total && ok; fb += a.sb) {
+                    const int cnt = min(a.sb, total - fb);
+                    if (!(ok = mbar_wait(wait0 + ms * 8, mp, abort_flag, a.error, 3))) break;
                     tc_fence_after();
-                    for (int b = 0; b < nb; ++b) {
-                        if (!(ok = mbar_wait(smem_u32(full + m_stage), m_phase, abort_flag, a.error, 3))) break;
-                        tc_fence_after();
-                        const uint32_t sbase = smem_u32(smem + m_stage * kTcStageBytes);
-                        const uint64_t bdesc = smem_desc(sbase + kTcBlockOff, a.lbo_b, a.sbo_b, 0);
-                        for (int mt = 0; mt < mt_n; ++mt) {
-                            const uint64_t adesc = smem_desc(sbase + mt * 4096, a.lbo_a, a.sbo_a, 2);
-                            if (!(a.debug & 1)) tc_mma_f16(tmem_base + as * 32 + mt * 16, adesc, bdesc, kIdescBf16, b > 0 ? 1u : 0u);
+                    uint32_t blk = ring0 + ms * stage_bytes;
+                    for (int u = 0; u < cnt && ok; ++u, blk += kBlk) {
+                        if (k == 0) {
+                            if (!(ok = enter_item())) break;
+                            tc_fence_after();
                         }
-                        if (a.debug & 32) mbar_arrive(smem_u32(empty + m_stage));
-                        else tc_commit(smem_u32(empty + m_stage));   // the stage is free once these MMAs retire
-                        if (++m_stage == a.stages) {
-                            m_stage = 0;
-                            m_phase ^= 1;
+                        const uint64_t blk16 = static_cast<uint64_t>((blk & 0x3FFFFu) >> 4);
+                        for (int mt = 0; mt < mt_n; ++mt) {
+                            const uint32_t d = d0 + mt * 16;
+                            if constexpr (TF32) {
+                                // operand "A", MN-major 32-bit elements: the 128-byte swizzle with 32-byte
+                                // atoms (layout type 1; its atom is 4 k rows of 128 bytes); 32-column groups
+                                // 2048 bytes apart, 4-row k groups 512 bytes apart, k step = 8 rows = 1024 bytes
+#pragma unroll
+                                for (int ks = 0; ks < 2; ++ks) {
+                                    const uint64_t a_hi = a_hi0 + blk16 + ((mt * 8192 + ks * 1024) >> 4);
+                                    const uint64_t a_lo = a_hi + (16384 >> 4);
+                                    const uint64_t b_hi = b_hi0 + blk16 + ((kImgOff + ks * 512) >> 4);
+                                    const uint64_t b_lo = b_hi + (1024 >> 4);
+                                    tc_mma<true>(d, a_hi, b_hi, kIdescTf32, (k > 0 || ks > 0) ? 1u : 0u);
+                                    tc_mma<true>(d, a_lo, b_hi, kIdescTf32, 1u);
+                                    tc_mma<true>(d, a_hi, b_lo, kIdescTf32, 1u);
+                                }
+                            } else {
+                                // operand "A": 64-column atoms 2048 bytes apart, 8-row k groups 1024 bytes apart
+                                tc_mma<false>(d, a_hi0 + blk16 + ((mt * 4096) >> 4), b_hi0 + blk16 + (kImgOff >> 4), kIdescBf16,
+                                              k > 0 ? 1u : 0u);
+                            }
+                        }
+                        if (++k == nbj) {
+                            tc_commit(accf0 + as * 8);   // the item's accumulator is complete
+                            ++j;
+                            k = 0;
+                            skip_empty_items();
                         }
                     }
                     if (!ok) break;
-                    if (nb > 0) tc_commit(smem_u32(acc_full + as));
-                    else mbar_arrive(smem_u32(acc_full + as));   // block-row without blocks: nothing to wait for
+                    tc_commit(empty0 + ms * 8);   // the slot is free once these MMAs retire
+                    if (++ms == static_cast<uint32_t>(a.stages)) {
+                        ms = 0;
+                        mp ^= 1;
+                    }
                 }
             }
-        } else {
+        } else if (warp < 6) {
             // -------------------------------------------------------------- epilogue warps
             const int q = warp & 3;   // TMEM lane quarter this warp may read
             uint32_t eit = it;
@@ -352,7 +405,7 @@ bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
 #pragma unroll
                         for (int rr = 0; rr < 16; ++rr) {
                             const int64_t row = static_cast<int64_t>(I) * 16 + rr;
-                            if (row < a.M && !(a.debug & 2)) {
+                            if (row < a.M) {
                                 float v = a.alpha * r[mt][rr];
                                 if (a.beta != 0.f) v = fmaf(a.beta, cold[mt][rr], v);
                                 a.C[row * a.ldc + col] = v;
@@ -361,15 +414,59 @@ bsr_tc_bf16_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                     }
                 }
             }
+        } else if constexpr (TF32) {
+            // -------------------------------------------------------------- converter warps
+            // split the fp32 slab of every block of the slot: hi stays in place, lo goes beside it
+            const int ct = threadIdx.x - 192;   // 0..127
+            uint32_t cs = m_stage, cp = m_phase;
+            for (int fb = 0; fb < total && ok; fb += a.sb) {
+                const int cnt = min(a.sb, total - fb);
+                if (lane == 0) ok = mbar_wait(smem_u32(full + cs), cp, abort_flag, a.error, 5);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                uint8_t *sbp = smem + cs * stage_bytes;
+                for (int u = 0; u < cnt; ++u) {
+                    float4 *hi = reinterpret_cast<float4 *>(sbp + u * kBlk);
+                    float4 *lo = reinterpret_cast<float4 *>(sbp + u * kBlk + 16384);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 x = hi[i * 128 + ct];
+                        float4 h;
+                        h.x = __uint_as_float(__float_as_uint(x.x) & 0xFFFFE000u);
+                        h.y = __uint_as_float(__float_as_uint(x.y) & 0xFFFFE000u);
+                        h.z = __uint_as_float(__float_as_uint(x.z) & 0xFFFFE000u);
+                        h.w = __uint_as_float(__float_as_uint(x.w) & 0xFFFFE000u);
+                        hi[i * 128 + ct] = h;
+                        lo[i * 128 + ct] = make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(conv + cs));
+                if (++cs == static_cast<uint32_t>(a.stages)) {
+                    cs = 0;
+                    cp ^= 1;
+                }
+            }
+        }
+        // every thread advances its copy of the consumer ring position past the batch, so that
+        // the MMA issuer and the converter warps enter the next batch at the same slot
+        {
+            const uint32_t adv = m_stage + static_cast<uint32_t>((total + a.sb - 1) / a.sb);
+            m_phase ^= (adv / static_cast<uint32_t>(a.stages)) & 1;
+            m_stage = adv % static_cast<uint32_t>(a.stages);
         }
         it += bn;
     }
     if (warp == 0 && lane == 0 && *abort_flag) {
-        // give the copies this thread issued a bounded time to land before shared memory is released
-        for (int s2 = 0; s2 < a.stages; ++s2)
-            if (p_filled & (1u << s2))
-                for (uint32_t i = 0; i < 65536 && !mbar_try_wait(smem_u32(full + s2), (p_fill_parity >> s2) & 1); ++i) {
-                }
+        // give the copies this thread issued a bounded time to land before shared memory is released:
+        // slot s was last filled by issue number i = s (mod stages), whose ring pass gives the parity
+        for (uint32_t s2 = 0; s2 < static_cast<uint32_t>(a.stages) && s2 < p_issued; ++s2) {
+            const uint32_t last = p_issued - 1 - ((p_issued - 1 - s2) % static_cast<uint32_t>(a.stages));
+            const uint32_t parity = (last / static_cast<uint32_t>(a.stages)) & 1;
+            for (uint32_t i = 0; i < 65536 && !mbar_try_wait(smem_u32(full + s2), parity); ++i) {
+            }
+        }
     }
 
     // ---- teardown: everybody meets here, also after an expired wait --------------------------
@@ -390,6 +487,21 @@ static __global__ void bsr_mma_image_bf16_kernel(const uint16_t *__restrict__ bv
     const int r = (i >> 4) & 15, c = i & 15;
     const int off = (((c >> 3) * 2 + (r >> 3)) * 8 + (r & 7)) * 8 + (c & 7);
     img[b * 256 + off] = bval[i];
+}
+
+// fp32 blocks: hi / lo split and the K-major image of each half: per k step (8 block columns)
+// four core matrices of 8 rows x 4 floats, ordered [k step][k half][row group]; hi image first
+// (1 KB), lo image after it.
+static __global__ void bsr_mma_image_tf32_kernel(const float *__restrict__ bval, float *__restrict__ img, int64_t nnzb) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= nnzb * 256) return;
+    const int64_t b = i >> 8;
+    const int r = (i >> 4) & 15, c = i & 15;
+    const int off = (c >> 3) * 128 + ((c & 7) >> 2) * 64 + (r >> 3) * 32 + (r & 7) * 4 + (c & 3);
+    const float x = bval[i];
+    const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    img[b * 512 + off] = h;
+    img[b * 512 + 256 + off] = x - h;
 }
 
 }  // namespace sd

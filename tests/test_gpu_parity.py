@@ -314,14 +314,16 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
 
 @pytest.mark.parametrize("N", [64, 128, 192, 256, 320, 512])
 @pytest.mark.parametrize("beta", [0.0, -0.75])
-def test_bsr_tensor_core_path_bf16(N, beta):
-    # bf16 blocks on the tcgen05 path: ragged M and K, empty block-rows, partially filled blocks,
-    # padded leading dimensions (kept multiples of 8 so that the TMA alignment rules hold)
+@pytest.mark.parametrize("dtype", [W.SD_BF16, W.SD_F32])
+def test_bsr_tensor_core_path(N, beta, dtype):
+    # blocks on the tcgen05 path (bf16 directly, fp32 as three tf32 products): ragged M and K,
+    # empty block-rows, partially filled blocks, padded leading dimensions (kept multiples of 8 so
+    # that the TMA alignment rules hold)
     rng = np.random.default_rng(N)
     M, K = 16 * 37 + 5, 16 * 29 + 11
     lengths = np.clip(rng.poisson(30, M), 0, K)
     lengths[32:64] = 0        # two empty block-rows
-    w = W.random_csr(M, K, N, lengths, seed=N + 1, dtype=W.SD_BF16, alpha=1.5, beta=beta)
+    w = W.random_csr(M, K, N, lengths, seed=N + 1, dtype=dtype, alpha=1.5, beta=beta)
     dw = DeviceWorkload(w)
     plan = dw.plan(family=sd.SD_BSR_TC)
     for pad_b, pad_c in [(0, 0), (8, 3)]:
@@ -334,13 +336,16 @@ def test_bsr_tensor_core_path_bf16(N, beta):
     plan.close()
 
 
-def test_bsr_tensor_core_dense_blocks_bf16_exact_products():
-    # fully dense blocks, small integers: every product and partial sum is exact in fp32, so the
-    # tensor-core result must equal the oracle bit for bit
-    w = W.g4_block(Mb=96, Kb=80, N=256, nblocks=700, seed=5, dtype=W.SD_BF16)
+@pytest.mark.parametrize("dtype", [W.SD_BF16, W.SD_F32])
+def test_bsr_tensor_core_dense_blocks_exact_products(dtype):
+    # fully dense blocks, small integers: every product and partial sum is exact in fp32 (and the
+    # lo halves of the fp32 split vanish), so the tensor-core result must equal the oracle bit for bit
+    w = W.g4_block(Mb=96, Kb=80, N=256, nblocks=700, seed=5, dtype=dtype)
     rng = np.random.default_rng(1)
-    w.vals = W.f32_to_bf16_bits(rng.integers(-4, 5, w.vals.shape).astype(np.float32))
-    w.B = W.f32_to_bf16_bits(rng.integers(-4, 5, w.B.shape).astype(np.float32)).reshape(w.B.shape)
+    iv = rng.integers(-4, 5, w.vals.shape).astype(np.float32)
+    ib = rng.integers(-4, 5, w.B.shape).astype(np.float32)
+    w.vals = W.f32_to_bf16_bits(iv) if dtype == W.SD_BF16 else iv
+    w.B = W.f32_to_bf16_bits(ib).reshape(w.B.shape) if dtype == W.SD_BF16 else ib
     dw = DeviceWorkload(w)
     plan = dw.plan()
     assert plan.info().family == sd.SD_BSR_TC
