@@ -1165,6 +1165,10 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         set_error(SD_ERR_INVALID_ARG, "B is null or ldb < N");
         return SD_ERR_INVALID_ARG;
     }
+    if (ldb * (plan->dtype == SD_F32 ? 4 : 2) > static_cast<int64_t>(UINT32_MAX)) {
+        set_error(SD_ERR_UNSUPPORTED, "row pitch of B must be below 4 GiB");
+        return SD_ERR_UNSUPPORTED;
+    }
     const int vw = plan->dtype == SD_F32 ? 4 : 8;
     const bool vec = aligned16(B) && aligned16(C) && N % vw == 0 && ldb % vw == 0 && ldc % 4 == 0;
 
@@ -1177,6 +1181,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     a.C = C;
     a.ldb = ldb;
     a.ldc = ldc;
+    a.ldb_bytes = static_cast<uint32_t>(ldb * (plan->dtype == SD_F32 ? 4 : 2));
     a.S = M;
     a.N = static_cast<int32_t>(N);
     a.alpha = alpha;

@@ -86,6 +86,14 @@ __device__ __forceinline__ void store_cols(float *c, const float (&acc)[VW], flo
     }
 }
 
+// Address of row `col` of B given a per-lane base pointer: one 32 x 32 -> 64 bit multiply-add
+// (column indices are non-negative and the row pitch in bytes is below 2^32, checked on the host).
+template <typename T>
+__device__ __forceinline__ const T *b_row(const T *base, int col, uint32_t ldb_bytes) {
+    return reinterpret_cast<const T *>(reinterpret_cast<const char *>(base) +
+                                       static_cast<uint64_t>(static_cast<uint32_t>(col)) * ldb_bytes);
+}
+
 // Arguments common to the CSR kernels.
 struct SpmmArgs {
     const int32_t *ptr;     // row (or segment) pointer array, [S+1]
@@ -96,6 +104,7 @@ struct SpmmArgs {
     const void *B;
     float *C;
     int64_t ldb, ldc;
+    uint32_t ldb_bytes;     // ldb * sizeof(element of B)
     int64_t S;              // number of rows / segments
     int32_t N;
     float alpha, beta;

@@ -112,7 +112,7 @@ merge_tile_kernel(const MergeArgs m) {
             float b[WB][NV][VW];
 #pragma unroll
             for (int u = 0; u < WB; ++u) {
-                const T *brow = Bl + static_cast<int64_t>(it[u].x) * a.ldb;
+                const T *brow = b_row(Bl, it[u].x, a.ldb_bytes);
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     if (colok[v]) {
@@ -133,7 +133,7 @@ merge_tile_kernel(const MergeArgs m) {
         for (; j < jend; ++j) {
             const int2 it = nz_s[j];
             const float av = __int_as_float(it.y);
-            const T *brow = Bl + static_cast<int64_t>(it.x) * a.ldb;
+            const T *brow = b_row(Bl, it.x, a.ldb_bytes);
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 if (colok[v]) {

@@ -117,6 +117,10 @@ sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, c
         set_error(SD_ERR_INVALID_ARG, "colind, vals or B is null, or ldb < N");
         return SD_ERR_INVALID_ARG;
     }
+    if (ldb * 4 > static_cast<int64_t>(UINT32_MAX)) {
+        set_error(SD_ERR_UNSUPPORTED, "row pitch of B must be below 4 GiB");
+        return SD_ERR_UNSUPPORTED;
+    }
     // layout of the fixed array: [tile table | head rows | tail rows]
     const int64_t ntiles = (M + nnz + kMergeTile - 1) / kMergeTile;
     const size_t table_bytes = ((static_cast<size_t>(ntiles) + 1) * sizeof(int32_t) + 255) & ~static_cast<size_t>(255);
@@ -143,6 +147,7 @@ sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, c
     a.C = C;
     a.ldb = ldb;
     a.ldc = ldc;
+    a.ldb_bytes = static_cast<uint32_t>(ldb * 4);
     a.S = M;
     a.N = static_cast<int32_t>(N);
     a.alpha = alpha;

@@ -86,7 +86,7 @@ rowsplit_kernel(const SpmmArgs a) {
             const int c = (LPR == 1) ? myc : __shfl_sync(FULL, myc, q, LPR);
             const float av = (LPR == 1) ? myv : __shfl_sync(FULL, myv, q, LPR);
             if (base + q < len) {
-                const T *brow = B + static_cast<int64_t>(c) * a.ldb + cbase;
+                const T *brow = b_row(B, c, a.ldb_bytes) + cbase;
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     if (colok[v]) {

@@ -71,7 +71,7 @@ seg_kernel(const SpmmArgs a) {
                     // unconditionally (only a segment's last chunk has such entries); short segments
                     // would waste most of their gathers that way and keep the test
                     const bool valid = SCRATCH || (p + q0 + qq < p1);
-                    const T *brow = Bl + static_cast<int64_t>(cq[qq]) * a.ldb;
+                    const T *brow = b_row(Bl, cq[qq], a.ldb_bytes);
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
                         if (valid && colok[v]) {
@@ -132,7 +132,7 @@ single_kernel(const SpmmArgs a) {
         float b[kSingleBatch][VW], o[kSingleBatch][VW];
 #pragma unroll
         for (int u = 0; u < kSingleBatch; ++u) {
-            RowLoad<T, VW>::ld(static_cast<const T *>(a.B) + static_cast<int64_t>(c[u]) * a.ldb + cbase + col, b[u]);
+            RowLoad<T, VW>::ld(b_row(static_cast<const T *>(a.B), c[u], a.ldb_bytes) + cbase + col, b[u]);
             const bool need_c = (s0 + u < a.S) && (r[u] < 0 || a.beta != 0.f);
             const float *crow = a.C + static_cast<int64_t>(r[u] & 0x7FFFFFFF) * a.ldc + cbase + col;
             if constexpr (VW == 1) {
