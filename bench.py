@@ -331,6 +331,32 @@ def run_gpu(args, rank, local_rank, world):
     e2e_ms = max_over_ranks(e2e_local, dev)
     e2e_value = flops_all / (e2e_ms * 1e-3) / 1e9
 
+    # ---- context only: cuSPARSE CSR SpMM (what the paper compares against), fp32 workloads ------
+    if args.cusparse and rank == 0:
+        for c in cases:
+            w = c["w"]
+            if w.dtype != W.SD_F32:
+                continue
+            try:
+                A = torch.sparse_csr_tensor(to_dev(w.rowptr).long(), to_dev(w.colind).long(), to_dev(w.vals),
+                                            size=(w.M, w.K))
+                ts = []
+                for i in range(8):
+                    flush.fill_(1.0)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    out = torch.sparse.mm(A, c["B"])   # alpha = 1, beta = 0 product only
+                    e1.record(stream)
+                    torch.cuda.synchronize()
+                    if i >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                    del out
+                c["cusparse_ms"] = float(np.mean(ts))
+                del A
+            except Exception as exc:   # context only: never fails the bench
+                c["cusparse_ms"] = None
+                c["cusparse_error"] = str(exc)[:120]
+
     if rank != 0:
         return
 
@@ -347,6 +373,10 @@ def run_gpu(args, rank, local_rank, world):
                     "effective_gbs": gbs, "frac_of_measured_hbm": gbs / peak,
                     "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS, "launches": int(info.launches), "windows": int(info.windows),
                     "plan_ms": c["plan_ms"], "plan_bytes": int(info.plan_bytes)})
+        if "cusparse_ms" in c:
+            per[-1]["context_cusparse_ms"] = c["cusparse_ms"]
+            if c["cusparse_ms"]:
+                per[-1]["context_speedup_over_cusparse"] = c["cusparse_ms"] / ms
     dom = max(per, key=lambda p: p["ms"])
     roofline = {"bound": "hbm", "kernel": dom["family"] + " on " + dom["workload"],
                 "achieved": dom["effective_gbs"], "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
@@ -398,6 +428,9 @@ def main():
     ap.add_argument("--impl", default="sd", choices=["sd", "reference"])
     ap.add_argument("--configs", default="", help="comma list of config indices (1..4) to restrict the step")
     ap.add_argument("--windows", type=int, default=0, help="column windows of the merge family (0 = plan's rule)")
+    ap.add_argument("--cusparse", action="store_true",
+                    help="also time cuSPARSE CSR SpMM through torch.sparse.mm on the fp32 workloads, as context "
+                         "only (the paper's comparison baseline; the library never calls it)")
     ap.add_argument("--small", action="store_true",
                     help="reduced sizes of the same workloads (dense operands still above the L2 size where "
                          "the full-size ones are); for profiler captures, not a bench number")
