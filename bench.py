@@ -209,7 +209,10 @@ SMALL_KW = {1: dict(n=768), 2: dict(scale=18), 3: dict(Mb=2048, Kb=2048), 4: dic
 
 
 def make_workload(args, ci, dt):
-    return W.config(ci, dtype=dt, **(SMALL_KW[ci] if args.small else {}))
+    kw = dict(SMALL_KW[ci]) if args.small else {}
+    if args.width:
+        kw["N"] = args.width
+    return W.config(ci, dtype=dt, **kw)
 
 
 def select_set(args):
@@ -428,6 +431,9 @@ def main():
     ap.add_argument("--impl", default="sd", choices=["sd", "reference"])
     ap.add_argument("--configs", default="", help="comma list of config indices (1..4) to restrict the step")
     ap.add_argument("--windows", type=int, default=0, help="column windows of the merge family (0 = plan's rule)")
+    ap.add_argument("--width", type=int, default=0,
+                    help="override the dense width N of every selected workload (width sweep: 1 = SpMV, 8, 32, "
+                         "128, 256); not the benchmark configuration")
     ap.add_argument("--cusparse", action="store_true",
                     help="also time cuSPARSE CSR SpMM through torch.sparse.mm on the fp32 workloads, as context "
                          "only (the paper's comparison baseline; the library never calls it)")
