@@ -334,6 +334,28 @@ def run_gpu(args, rank, local_rank, world):
     e2e_ms = max_over_ranks(e2e_local, dev)
     e2e_value = flops_all / (e2e_ms * 1e-3) / 1e9
 
+    # ---- gather ceiling: the workload's own index stream as bare row gathers ------------------------
+    if args.probe and rank == 0:
+        sink = torch.zeros(sd.sd_probe_gather(None, 0, None, 128), dtype=torch.float32, device=dev)
+        for c in cases:
+            w = c["w"]
+            row_bytes = w.N * (4 if w.dtype == W.SD_F32 else 2)
+            if row_bytes not in (16, 32, 64, 128, 256, 512):
+                continue
+            colind = to_dev(w.colind)
+            ts = []
+            for i in range(8):
+                flush.fill_(1.0)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                sd.sd_probe_gather(colind, w.nnz, c["B"], row_bytes, sink, stream)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(e0.elapsed_time(e1))
+            c["probe_ms"] = float(np.mean(ts))
+            del colind
+
     # ---- context only: cuSPARSE CSR SpMM (what the paper compares against), fp32 workloads ------
     if args.cusparse and rank == 0:
         for c in cases:
@@ -376,6 +398,10 @@ def run_gpu(args, rank, local_rank, world):
                     "effective_gbs": gbs, "frac_of_measured_hbm": gbs / peak,
                     "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS, "launches": int(info.launches), "windows": int(info.windows),
                     "plan_ms": c["plan_ms"], "plan_bytes": int(info.plan_bytes)})
+        if "probe_ms" in c:
+            per[-1]["gather_probe_ms"] = c["probe_ms"]
+            per[-1]["gather_probe_tbs"] = w.nnz * w.N * (4 if w.dtype == W.SD_F32 else 2) / (c["probe_ms"] * 1e-3) / 1e12
+            per[-1]["spmm_over_gather_probe"] = ms / c["probe_ms"]
         if "cusparse_ms" in c:
             per[-1]["context_cusparse_ms"] = c["cusparse_ms"]
             if c["cusparse_ms"]:
@@ -431,6 +457,9 @@ def main():
     ap.add_argument("--impl", default="sd", choices=["sd", "reference"])
     ap.add_argument("--configs", default="", help="comma list of config indices (1..4) to restrict the step")
     ap.add_argument("--windows", type=int, default=0, help="column windows of the merge family (0 = plan's rule)")
+    ap.add_argument("--probe", action="store_true",
+                    help="also replay every workload's colind stream as bare row gathers (sd_probe_gather) and "
+                         "report its time beside the SpMM time: the gather ceiling of the memory system for that stream")
     ap.add_argument("--width", type=int, default=0,
                     help="override the dense width N of every selected workload (width sweep: 1 = SpMV, 8, 32, "
                          "128, 256); not the benchmark configuration")

@@ -213,6 +213,18 @@ sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, c
                                  int64_t ldb, float *C, int64_t ldc, float alpha, float beta,
                                  void *stream);
 
+/* sd_probe_gather -- measurement aid (no counterpart in the paper).  Replays `count` row
+ * indices idx[] (device, e.g. the colind array of a CSR matrix, in storage order) as bare
+ * gathers of `row_bytes`-byte rows (16, 32, ..., 512; 16-byte aligned table, row pitch =
+ * row_bytes) from `table` (device): the memory access stream of SpMM with the values of A, the
+ * multiply-adds and the output removed.  Its time is the rate at which the memory system
+ * delivers that gather stream, against which bench.py sets the time of the SpMM kernels.
+ * `sink` (device) receives one partial sum per thread so that the loads stay alive; a call with
+ * idx, table and sink all NULL only reports the floats `sink` must hold in *sink_floats_needed.
+ * Asynchronous on `stream`; allocates nothing. */
+sd_status_t sd_probe_gather(const int32_t *idx, int64_t count, const void *table, int32_t row_bytes,
+                            float *sink, int32_t *sink_floats_needed, void *stream);
+
 /* sd_last_error -- copy the calling thread's last error text into buf (NUL-terminated,
  * at most n bytes); returns the last status code. */
 int sd_last_error(char *buf, size_t n);
