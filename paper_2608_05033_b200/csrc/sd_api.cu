@@ -423,6 +423,8 @@ struct sd_plan {
     int32_t *bcol = nullptr;
     void *bval = nullptr;
     void *bval_mma = nullptr;   // tensor-core operand images of the blocks
+    int32_t *bsr_part = nullptr; // block-row ranges of the tensor-core kernel's CTAs
+    int32_t bsr_nparts = 0;
     int32_t *dev_error = nullptr;
     int64_t nnzb = 0;
 
@@ -802,6 +804,13 @@ static sd_status_t build_bsr(sd_plan *p, const unsigned long long *ukeys, int64_
                        "bval (tensor-core image)")))
         return s;
     SD_CUDA_TRY(build_bsr_mma_image(p->bval, p->bval_mma, nnzb, p->dtype, st));
+    // one persistent CTA per SM, each with a contiguous range of block-rows of about equal cost
+    p->bsr_nparts = static_cast<int32_t>(Mb < p->info.sm_count ? Mb : p->info.sm_count);
+    if (p->bsr_nparts > 0) {
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->bsr_part), sizeof(int32_t) * (p->bsr_nparts + 1), "block-row partition")))
+            return s;
+        SD_CUDA_TRY(build_bsr_partition(p->browptr, static_cast<int32_t>(Mb), p->bsr_nparts, p->bsr_part, st));
+    }
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->dev_error), sizeof(int32_t), "error word"))) return s;
     SD_CUDA_TRY(cudaMemsetAsync(p->dev_error, 0, sizeof(int32_t), st));
     SD_CUDA_TRY(cudaStreamSynchronize(st));
@@ -967,6 +976,7 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->bcol);
     cudaFree(p->bval);
     cudaFree(p->bval_mma);
+    cudaFree(p->bsr_part);
     cudaFree(p->dev_error);
     cudaFree(p->stage_B);
     cudaFree(p->stage_C);
@@ -1274,6 +1284,8 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         b.bcol = plan->bcol;
         b.bval = plan->bval;
         b.bval_mma = plan->bval_mma;
+        b.part = plan->bsr_part;
+        b.nparts = plan->bsr_nparts;
         b.B = B;
         b.C = C;
         b.ldb = ldb;

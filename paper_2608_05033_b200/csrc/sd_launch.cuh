@@ -50,6 +50,8 @@ struct BsrArgs {
     const int32_t *bcol;     // [nnzb]
     const void *bval;        // [nnzb][16][16] row-major, plan dtype
     const void *bval_mma;    // [nnzb] tensor-core operand images of the same blocks
+    const int32_t *part;     // [nparts + 1] block-row ranges of the tensor-core kernel's CTAs
+    int32_t nparts;
     const void *B;
     float *C;
     int64_t ldb, ldc;
@@ -62,6 +64,7 @@ cudaError_t run_bsr_simt(const BsrArgs &a, int dtype, bool vec, cudaStream_t st)
 // Tensor-core form.  bsr_tc_usable: dtype, dense width and the TMA alignment rules allow it.
 bool bsr_tc_usable(const BsrArgs &a, int dtype);
 cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_count, cudaStream_t st);
+cudaError_t build_bsr_partition(const int32_t *browptr, int32_t Mb, int32_t nparts, int32_t *part, cudaStream_t st);
 cudaError_t build_bsr_mma_image(const void *bval, void *img, int64_t nnzb, int dtype, cudaStream_t st);
 
 }  // namespace sd

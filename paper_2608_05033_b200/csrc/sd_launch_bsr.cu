@@ -24,6 +24,33 @@ cudaError_t build_bsr_mma_image(const void *bval, void *img, int64_t nnzb, int d
     return cudaGetLastError();
 }
 
+// Block-row ranges of about equal cost for the CTAs of the tensor-core kernel: a block-row costs
+// 8 units per block plus 2 for its accumulator hand-over, so the running cost up to block-row I is
+// F(I) = 8*browptr[I] + 2*I; part[c] is the first I with F(I) >= c*F(Mb)/nparts.
+static __global__ void bsr_partition_kernel(const int32_t *__restrict__ browptr, int32_t Mb, int32_t nparts,
+                                            int32_t *__restrict__ part) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c > nparts) return;
+    if (c == nparts) {
+        part[c] = Mb;
+        return;
+    }
+    const int64_t total = 8ll * browptr[Mb] + 2ll * Mb;
+    const int64_t target = total / nparts * c + total % nparts * c / nparts;
+    int lo = 0, hi = Mb;   // first I in [0, Mb] with F(I) >= target
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (8ll * browptr[mid] + 2ll * mid >= target) hi = mid;
+        else lo = mid + 1;
+    }
+    part[c] = lo;
+}
+
+cudaError_t build_bsr_partition(const int32_t *browptr, int32_t Mb, int32_t nparts, int32_t *part, cudaStream_t st) {
+    bsr_partition_kernel<<<(nparts + 256) / 256, 256, 0, st>>>(browptr, Mb, nparts, part);
+    return cudaGetLastError();
+}
+
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -43,13 +70,15 @@ static EncodeTiledFn encode_tiled() {
 
 // The tensor-core kernel reads B through a 3-D TMA view {one 128-byte column group, K rows,
 // N / group columns}: N must be a multiple of the group (64 bf16 / 32 fp32 columns), the base
-// 16-byte aligned and the row pitch a multiple of 16 bytes.
+// 16-byte aligned and the row pitch a multiple of 16 bytes.  Its epilogue stores 16-byte vectors
+// of C: base 16-byte aligned, ldc a multiple of 4.
 bool bsr_tc_usable(const BsrArgs &a, int dtype) {
-    if (a.bval_mma == nullptr) return false;
+    if (a.bval_mma == nullptr || a.part == nullptr || a.nparts < 1) return false;
     const int group = dtype == SD_BF16 ? 64 : 32;
     const int es = dtype == SD_BF16 ? 2 : 4;
     if (a.N < group || a.N % group != 0 || (a.ldb * es) % 16 != 0) return false;
     if (reinterpret_cast<uintptr_t>(a.B) & 15u) return false;
+    if ((reinterpret_cast<uintptr_t>(a.C) & 15u) || a.ldc % 4 != 0) return false;
     return encode_tiled() != nullptr;
 }
 
@@ -86,20 +115,22 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     t.Mb = a.Mb;
     t.N = a.N;
     t.nslab = (a.N + kTcSlabCols - 1) / kTcSlabCols;
+    t.part = a.part;
     t.alpha = a.alpha;
     t.beta = a.beta;
     t.error = error_word;
     t.box_bytes = box_groups * 2048;
-    // ring geometry (bench-only overrides through the environment).  bf16: two CTAs per SM, each
-    // with 10 slots of 1 block; fp32: one CTA per SM with 2 slots of 3 blocks (34 KB per block).
-    t.sb = env_int(tf32 ? "SD_TC32_SB" : "SD_TC_SB", tf32 ? 3 : 1);
-    t.stages = env_int(tf32 ? "SD_TC32_STAGES" : "SD_TC_STAGES", tf32 ? 2 : 10);
-    const int ctas_per_sm = env_int(tf32 ? "SD_TC32_CTAS" : "SD_TC_CTAS", tf32 ? 1 : 2);
-    const int blk = tf32 ? kTcBlkBytesTf32 : kTcBlkBytesBf16;
+    // ring geometry (bench-only overrides through the environment); one CTA per SM, its ring
+    // takes most of the shared memory: bf16 2 slots of 8 blocks (8.5 KB per block), fp32 3 slots
+    // of 2 blocks (34 KB per block).  A barrier round trip costs far more than a block's work,
+    // so slots hold several blocks.
+    t.sb = env_int(tf32 ? "SD_TC32_SB" : "SD_TC_SB", tf32 ? 2 : 8);
+    t.stages = env_int(tf32 ? "SD_TC32_STAGES" : "SD_TC_STAGES", tf32 ? 3 : 2);
     if (t.sb < 1) t.sb = 1;
+    if (t.sb > 64) t.sb = 64;
     if (t.stages < 1) t.stages = 1;
     if (t.stages > kTcMaxStages) t.stages = kTcMaxStages;
-    const int smem = t.stages * t.sb * blk + 2048 + 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks);
+    const int smem = t.stages * tc_stage_bytes(tf32, t.sb) + 2048 + 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks);
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
     static int attr_set[2] = {0, 0};
     if (attr_set[tf32] < smem) {
@@ -108,10 +139,10 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
         if (e != cudaSuccess) return e;
         attr_set[tf32] = smem;
     }
-    const int items = t.Mb * t.nslab;
-    const int grid = items < sm_count * ctas_per_sm ? items : sm_count * ctas_per_sm;
-    if (tf32) bsr_tc_kernel<true><<<grid, 320, smem, st>>>(map, t);
-    else bsr_tc_kernel<false><<<grid, 192, smem, st>>>(map, t);
+    const int grid = a.nparts;
+    (void)sm_count;
+    if (tf32) bsr_tc_kernel<true><<<grid, kTcThreadsTf32, smem, st>>>(map, t);
+    else bsr_tc_kernel<false><<<grid, kTcThreadsBf16, smem, st>>>(map, t);
     return cudaGetLastError();
 }
 

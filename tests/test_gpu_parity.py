@@ -317,8 +317,9 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
 @pytest.mark.parametrize("dtype", [W.SD_BF16, W.SD_F32])
 def test_bsr_tensor_core_path(N, beta, dtype):
     # blocks on the tcgen05 path (bf16 directly, fp32 as three tf32 products): ragged M and K,
-    # empty block-rows, partially filled blocks, padded leading dimensions (kept multiples of 8 so
-    # that the TMA alignment rules hold)
+    # empty block-rows, partially filled blocks, padded leading dimensions (ldb kept a multiple of 8
+    # so that the TMA alignment rules hold; ldc = N + 4 keeps the 16-byte stores of the epilogue,
+    # ldc = N + 3 breaks them and must be served by the SIMT form with the same result)
     rng = np.random.default_rng(N)
     M, K = 16 * 37 + 5, 16 * 29 + 11
     lengths = np.clip(rng.poisson(30, M), 0, K)
@@ -326,12 +327,35 @@ def test_bsr_tensor_core_path(N, beta, dtype):
     w = W.random_csr(M, K, N, lengths, seed=N + 1, dtype=dtype, alpha=1.5, beta=beta)
     dw = DeviceWorkload(w)
     plan = dw.plan(family=sd.SD_BSR_TC)
-    for pad_b, pad_c in [(0, 0), (8, 3)]:
+    for pad_b, pad_c in [(0, 0), (8, 4), (8, 3)]:
         got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_c)
         assert plan.device_status() == 0
         assert intact
         check(w, got)
     got2, _ = run_spmm(plan, w, pad_b=8, pad_c=3)
+    assert np.array_equal(got, got2)
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", [W.SD_BF16, W.SD_F32])
+def test_bsr_tensor_core_block_row_partition(dtype):
+    # very uneven block-rows: one with 2,500 blocks (more than the kernel stages at once, so it goes
+    # through the oversized-row path), runs of empty block-rows, a ragged tail; 512 dense columns =
+    # two slabs per block-row.  The CTAs' block-row ranges come from the plan-time partition.
+    rng = np.random.default_rng(17)
+    M, K, N = 16 * 400 + 7, 16 * 2500, 512
+    lengths = np.clip(rng.poisson(20, M), 0, K)
+    lengths[16 * 40:16 * 90] = 0
+    lengths[16 * 200] = K            # every block of this block-row is occupied
+    lengths[16 * 399:] = 0
+    w = W.random_csr(M, K, N, lengths, seed=23, dtype=dtype, alpha=-0.5, beta=0.25)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_BSR_TC)
+    got, intact = run_spmm(plan, w)
+    assert plan.device_status() == 0
+    assert intact
+    check(w, got)
+    got2, _ = run_spmm(plan, w)
     assert np.array_equal(got, got2)
     plan.close()
 

@@ -114,6 +114,9 @@ def distinct_sorted_columns(rng: np.random.Generator, lengths: np.ndarray, K: in
         np.cumsum(lengths, out=rp[1:])
         for r in bad_rows:
             lo, hi = int(rp[r]), int(rp[r + 1])
+            if hi - lo == K:   # a full row holds every column: nothing to draw
+                key[lo:hi] = np.arange(K, dtype=np.int64) + r * K
+                continue
             seg = key[lo:hi] - r * K
             while True:
                 u = np.unique(seg)
