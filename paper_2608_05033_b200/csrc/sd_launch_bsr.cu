@@ -127,10 +127,10 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     t.sb = env_int(tf32 ? "SD_TC32_SB" : "SD_TC_SB", tf32 ? 2 : 8);
     t.stages = env_int(tf32 ? "SD_TC32_STAGES" : "SD_TC_STAGES", tf32 ? 3 : 2);
     if (t.sb < 1) t.sb = 1;
-    if (t.sb > 64) t.sb = 64;
+    if (t.sb > 32) t.sb = 32;   // one mask bit per block of a ring slot
     if (t.stages < 1) t.stages = 1;
     if (t.stages > kTcMaxStages) t.stages = kTcMaxStages;
-    const int smem = t.stages * tc_stage_bytes(tf32, t.sb) + 2048 + 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks);
+    const int smem = t.stages * tc_stage_bytes(tf32, t.sb) + 2048 + 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks + 2 * tc_mask_words(t.sb));
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
     static int attr_set[2] = {0, 0};
     if (attr_set[tf32] < smem) {
