@@ -418,6 +418,11 @@ struct sd_plan {
     float *tile_tail = nullptr;
     int64_t ntiles = 0;
 
+    // narrow dense operands (N <= kCooMaxN) of the merge family
+    int32_t *coo_row = nullptr;
+    int32_t *coo_c1_row = nullptr, *coo_c2_row = nullptr;
+    float *coo_c1_val = nullptr, *coo_c2_val = nullptr;
+
     // BSR
     int32_t *browptr = nullptr;
     int32_t *bcol = nullptr;
@@ -775,6 +780,20 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
     p->info.num_segments = p->num_segments;
     p->info.windows = W;
     p->info.launches = launches;
+    // Narrow dense operands take the COO segmented reduction instead of the tile kernel (the tile
+    // table above stays valid and inspectable): one row index per nonzero and two carry lists.
+    if (W == 1 && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !getenv("SD_NO_COO")) {
+        const int64_t chunks1 = (p->nnz + kCooChunk - 1) / kCooChunk, count2 = 2 * chunks1;
+        const int64_t chunks2 = (count2 + kCooChunk - 1) / kCooChunk, count3 = 2 * chunks2;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_row), sizeof(int32_t) * p->nnz, "row index per nonzero"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_row), sizeof(int32_t) * count2, "carry rows"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_val), sizeof(float) * count2 * p->N, "carry sums"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_row), sizeof(int32_t) * count3, "carry rows (level 2)"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_val), sizeof(float) * count3 * p->N, "carry sums (level 2)"))) return s;
+        SD_CUDA_TRY(build_coo_rows(p->rowptr, p->M, p->nnz, p->coo_row, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        p->info.launches = 3 + (count2 > kCooDirectFinal);
+    }
     return SD_OK;
 }
 
@@ -972,6 +991,11 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->fix_long);
     cudaFree(p->tile_head);
     cudaFree(p->tile_tail);
+    cudaFree(p->coo_row);
+    cudaFree(p->coo_c1_row);
+    cudaFree(p->coo_c1_val);
+    cudaFree(p->coo_c2_row);
+    cudaFree(p->coo_c2_val);
     cudaFree(p->browptr);
     cudaFree(p->bcol);
     cudaFree(p->bval);
@@ -1202,6 +1226,21 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         SD_CUDA_TRY(run_rowsplit(a, plan->dtype, vec, st));
         return SD_OK;
     case SD_MERGE: {
+        if (plan->coo_row) {   // narrow dense operand: C = beta * C, then one writer per row adds alpha * (A B)
+            if (beta != 1.f) SD_CUDA_TRY(run_scale_c(C, ldc, M, static_cast<int32_t>(N), beta, st));
+            a.colind = plan->colind;
+            a.vals = plan->vals;
+            CooPlan cp;
+            cp.row = plan->coo_row;
+            cp.nnz = plan->nnz;
+            cp.c1_row = plan->coo_c1_row;
+            cp.c1_val = plan->coo_c1_val;
+            cp.c2_row = plan->coo_c2_row;
+            cp.c2_val = plan->coo_c2_val;
+            const bool bvec = aligned16(B) && (ldb * (plan->dtype == SD_F32 ? 4 : 2)) % 16 == 0;
+            SD_CUDA_TRY(run_coo(cp, a, plan->dtype, bvec, plan->info.sm_count, st));
+            return SD_OK;
+        }
         a.ptr = plan->m_ptr;
         a.colind = plan->m_col;
         a.vals = plan->m_vals;

@@ -44,6 +44,23 @@ cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fi
                       const int32_t *fix_long, int32_t nlong, cudaStream_t st);
 constexpr int kMergeLongChain = 8;   // chains of at least this many tiles go to the per-CTA fix-up
 
+// Family (b) for dense widths up to kCooMaxN (beyond it the shuffles per nonzero outweigh the
+// gain; measured cross-over between 4 and 8 columns): segmented reduction over the nonzeros with an
+// explicit row index per nonzero, carries reduced in two more levels.  C must hold beta * C_in.
+constexpr int kCooMaxN = 4;
+constexpr int kCooChunk = 128;             // nonzeros per warp step
+constexpr int64_t kCooDirectFinal = 4096;  // carry lists up to this length skip the second level
+struct CooPlan {
+    const int32_t *row;   // [nnz] row of every nonzero
+    int64_t nnz;
+    int32_t *c1_row;      // [2 * ceil(nnz / kCooChunk)] first-level carries
+    float *c1_val;        // ... x N
+    int32_t *c2_row;      // [2 * ceil(len(c1) / kCooChunk)] second-level carries
+    float *c2_val;
+};
+cudaError_t run_coo(const CooPlan &cp, const SpmmArgs &s, int dtype, bool vec, int sm_count, cudaStream_t st);
+cudaError_t build_coo_rows(const int32_t *rowptr, int64_t M, int64_t nnz, int32_t *row, cudaStream_t st);
+
 // Family (c).
 struct BsrArgs {
     const int32_t *browptr;  // [Mb + 1]

@@ -1,5 +1,6 @@
 #include "sd_launch.cuh"
 #include "sd_merge.cuh"
+#include "sd_coo.cuh"
 #include "sd_rowsplit.cuh"
 
 namespace sd {
@@ -20,6 +21,78 @@ cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fi
         e = cudaGetLastError();
     }
     return e;
+}
+
+// ---- narrow dense operands: COO segmented reduction --------------------------------------------
+template <typename T, int N>
+static cudaError_t launch_coo_n(const CooPlan &cp, const SpmmArgs &s, bool vec, int sm_count, cudaStream_t st) {
+    const int64_t chunks1 = (cp.nnz + kCooChunk - 1) / kCooChunk;
+    const int64_t count2 = 2 * chunks1;
+    const int64_t chunks2 = (count2 + kCooChunk - 1) / kCooChunk;
+    const int64_t count3 = 2 * chunks2;
+    auto grid_for = [&](int64_t chunks) {
+        const int64_t want = (chunks + 7) / 8;   // 8 warps per CTA, one chunk per warp step
+        const int64_t cap = static_cast<int64_t>(sm_count) * 8;
+        return static_cast<unsigned>(want < cap ? (want > 0 ? want : 1) : cap);
+    };
+    CooArgs a;
+    a.row = cp.row;
+    a.colind = s.colind;
+    a.vals = s.vals;
+    a.B = s.B;
+    a.ldb_bytes = s.ldb_bytes;
+    a.count = cp.nnz;
+    a.C = s.C;
+    a.ldc = s.ldc;
+    a.alpha = s.alpha;
+    a.carry_row = cp.c1_row;
+    a.carry_val = cp.c1_val;
+    if (vec) coo_reduce_kernel<T, N, true, false><<<grid_for(chunks1), 256, 0, st>>>(a);
+    else coo_reduce_kernel<T, N, false, false><<<grid_for(chunks1), 256, 0, st>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int32_t *frow = cp.c1_row;
+    const float *fval = cp.c1_val;
+    int64_t fcount = count2;
+    if (count2 > kCooDirectFinal) {   // level 2: the carry list is reduced the same way
+        CooArgs b = a;
+        b.row = cp.c1_row;
+        b.colind = nullptr;
+        b.vals = cp.c1_val;
+        b.B = nullptr;
+        b.count = count2;
+        b.carry_row = cp.c2_row;
+        b.carry_val = cp.c2_val;
+        coo_reduce_kernel<float, N, false, true><<<grid_for(chunks2), 256, 0, st>>>(b);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        frow = cp.c2_row;
+        fval = cp.c2_val;
+        fcount = count3;
+    }
+    coo_final_kernel<N><<<static_cast<unsigned>((fcount + 255) / 256), 256, 0, st>>>(frow, fval, fcount, s.C, s.ldc, s.alpha);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t launch_coo(const CooPlan &cp, const SpmmArgs &s, bool vec, int sm_count, cudaStream_t st) {
+    switch (s.N) {
+    case 1: return launch_coo_n<T, 1>(cp, s, false, sm_count, st);
+    case 2: return launch_coo_n<T, 2>(cp, s, false, sm_count, st);
+    case 3: return launch_coo_n<T, 3>(cp, s, false, sm_count, st);
+    case 4: return launch_coo_n<T, 4>(cp, s, vec && sizeof(T) == 4, sm_count, st);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+// `vec`: B is 16-byte aligned and its row pitch a multiple of 16 bytes.  C must hold beta * C_in.
+cudaError_t run_coo(const CooPlan &cp, const SpmmArgs &s, int dtype, bool vec, int sm_count, cudaStream_t st) {
+    return dtype == SD_F32 ? launch_coo<float>(cp, s, vec, sm_count, st) : launch_coo<__nv_bfloat16>(cp, s, vec, sm_count, st);
+}
+
+cudaError_t build_coo_rows(const int32_t *rowptr, int64_t M, int64_t nnz, int32_t *row, cudaStream_t st) {
+    if (nnz == 0) return cudaSuccess;
+    coo_rows_kernel<<<static_cast<unsigned>((nnz + 255) / 256), 256, 0, st>>>(rowptr, M, nnz, row);
+    return cudaGetLastError();
 }
 
 }  // namespace sd

@@ -12,7 +12,10 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 CASES = [("tiny_uniform", 0, W.SD_F32, 1), ("stencil", 1, W.SD_F32, 1), ("gcn_rmat", 2, W.SD_F32, 2),
-         ("block16_f32", 3, W.SD_F32, 3), ("block16_bf16", 3, W.SD_BF16, 3), ("skewed", 4, W.SD_F32, 2)]
+         ("block16_f32", 3, W.SD_F32, 3), ("block16_bf16", 3, W.SD_BF16, 3), ("skewed", 4, W.SD_F32, 2),
+         # narrow dense operands of the two merge-family workloads (SpMV and four columns)
+         ("skewed_spmv", 4, W.SD_F32, 2), ("gcn_rmat_n4", 2, W.SD_F32, 2)]
+NARROW = {"skewed_spmv": 1, "gcn_rmat_n4": 4}
 
 
 @pytest.mark.parametrize("name,ci,dtype,family", CASES)
@@ -20,7 +23,7 @@ def test_full_size_config_matches_oracle(name, ci, dtype, family):
     import paper_2608_05033_b200 as sd
     from util import DeviceWorkload, dev
 
-    w = W.config(ci, dtype=dtype)
+    w = W.config(ci, dtype=dtype, **({"N": NARROW[name]} if name in NARROW else {}))
     dw = DeviceWorkload(w)
     plan = dw.plan()
     info = plan.info()

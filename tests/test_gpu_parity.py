@@ -312,6 +312,39 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     plan.close()
 
 
+@pytest.mark.parametrize("N", [1, 2, 3, 4])
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_merge_narrow_operand_all_carry_levels(N, dtype):
+    # dense widths up to 4 take the segmented reduction over (row, column, value) triples: enough
+    # nonzeros that its carry list goes through the second level, one row holding every column (it
+    # spans about two thousand 128-nonzero chunks), runs of empty rows, one-nonzero rows, a padded
+    # and misaligned B
+    rng = np.random.default_rng(N)
+    M, K = 5003, 260_000
+    lengths = np.clip((5000.0 * np.arange(1, M + 1) ** -0.9).astype(np.int64), 1, 5000)
+    lengths = rng.permutation(lengths)
+    lengths[100:140] = 0
+    lengths[M // 2] = K
+    lengths[M - 1] = 0
+    w = W.random_csr(M, K, N, lengths, seed=40 + N, dtype=dtype, alpha=0.75, beta=-1.5)
+    assert 2 * ((w.nnz + 127) // 128) > 4096   # the first carry list is longer than the direct-final limit
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE)
+    assert plan.info().launches == 4
+    for pad_b, offset in [(0, 0), (3, 1)]:
+        got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_b, offset=offset)
+        assert intact
+        check(w, got)
+    got2, _ = run_spmm(plan, w, pad_b=3, pad_c=3, offset=1)
+    assert np.array_equal(got, got2)
+    poison = np.full((M, N), np.nan, np.float32)
+    got3, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got3, beta=0.0)
+    got4, _ = run_spmm(plan, w, beta=1.0)
+    check(w, got4, beta=1.0)
+    plan.close()
+
+
 @pytest.mark.parametrize("N", [64, 128, 192, 256, 320, 512])
 @pytest.mark.parametrize("beta", [0.0, -0.75])
 @pytest.mark.parametrize("dtype", [W.SD_BF16, W.SD_F32])
