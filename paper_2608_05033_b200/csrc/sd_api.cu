@@ -1217,6 +1217,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     a.ldc = ldc;
     a.ldb_bytes = static_cast<uint32_t>(ldb * (plan->dtype == SD_F32 ? 4 : 2));
     a.S = M;
+    a.max_len = plan->info.max_r;
     a.N = static_cast<int32_t>(N);
     a.alpha = alpha;
     a.beta = beta;

@@ -108,6 +108,7 @@ struct SpmmArgs {
     int64_t S;              // number of rows / segments
     int32_t N;
     float alpha, beta;
+    int64_t max_len;        // longest row / segment if known (0: unknown); lets the row-split kernel drop its second accumulator
 };
 
 inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
