@@ -81,7 +81,7 @@ __device__ __forceinline__ void store_cols(float *c, const float (&acc)[VW], flo
                 const float4 o = *p;
                 r.x += beta * o.x; r.y += beta * o.y; r.z += beta * o.z; r.w += beta * o.w;
             }
-            *p = r;
+            __stcs(p, r);   // C is written once and not read again: streaming store, first to leave L2
         }
     }
 }

@@ -63,7 +63,7 @@ merge_tile_kernel(const MergeArgs m) {
     for (int i = tid; i <= ends + 1; i += kMergeThreads)
         ptr_s[i] = __ldg(a.ptr + min(seg0 + i, m.seg_end));
     for (int k = tid; k < nnz_t; k += kMergeThreads)
-        nz_s[k] = make_int2(__ldg(a.colind + nz0 + k), __float_as_int(to_float(vals[nz0 + k])));
+        nz_s[k] = make_int2(__ldcs(a.colind + nz0 + k), __float_as_int(to_float(__ldcs(vals + nz0 + k))));   // A streams through
     if (tid == 0) first_end_s = G;
     __syncthreads();
 
