@@ -22,8 +22,10 @@ constexpr int kMergeEnd = -1;  // column value that marks a segment end in the s
 
 // FULL: every lane's columns are inside N (N is a multiple of the slab width), so the
 // per-vector column tests disappear from the inner loop.
+// One vector per lane: eight CTAs per SM (32 registers; the few spilled bytes cost less than the lost
+// occupancy).  Two vectors per lane need more registers: four CTAs.
 template <typename T, int VW, int LPR, int NV, bool FULL>
-__global__ void __launch_bounds__(kMergeThreads)
+__global__ void __launch_bounds__(kMergeThreads, NV == 1 ? 8 : 4)
 merge_tile_kernel(const MergeArgs m) {
     constexpr unsigned FULLMASK = 0xffffffffu;
     constexpr int G = kMergeThreads / LPR;   // groups per tile
@@ -100,6 +102,7 @@ merge_tile_kernel(const MergeArgs m) {
 #pragma unroll
         for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
 
+    const uint64_t keep = l2_keep_policy();
     int j = j0;
     for (int s = s0;; ++s) {
         const int jend = (s < s1) ? (ptr_s[s + 1] - nz0) : j1;
@@ -116,7 +119,7 @@ merge_tile_kernel(const MergeArgs m) {
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     if (colok[v]) {
-                        RowLoad<T, VW>::ld(brow + v * LPR * VW, b[u][v]);
+                        RowLoadKeep<T, VW>::ld(brow + v * LPR * VW, b[u][v], keep);
                     } else {
 #pragma unroll
                         for (int e = 0; e < VW; ++e) b[u][v][e] = 0.f;
@@ -138,7 +141,7 @@ merge_tile_kernel(const MergeArgs m) {
             for (int v = 0; v < NV; ++v) {
                 if (colok[v]) {
                     float b[VW];
-                    RowLoad<T, VW>::ld(brow + v * LPR * VW, b);
+                    RowLoadKeep<T, VW>::ld(brow + v * LPR * VW, b, keep);
 #pragma unroll
                     for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(av, b[e], acc[v][e]);
                 }
