@@ -8,7 +8,7 @@ One *step* is one pass of the whole hot path: one sd_spmm call on each benchmark
 fp32 and bf16 -> family (c)), inputs resident in HBM, L2 flushed before every call.  The JSON
 line's `value` is sum(2*nnz*N) / sum(device time) over the step; `per_config` carries each
 workload's own GFLOP/s, effective GB/s on the compulsory-traffic model and fraction of the
-measured HBM peak.  `e2e` runs the same step through sd_spmm_host with pinned host buffers
+measured HBM peak.  `e2e` runs the same step through sd_spmm_host_async / sd_plan_sync with pinned host buffers
 (B copied in, C copied out, every call).  `--impl reference` times the CPU oracle instead.
 
 With N > 1 ranks (torchrun), every rank runs the step on its own dense operands (independent
@@ -319,8 +319,12 @@ def run_gpu(args, rank, local_rank, world):
         d2h += Ch.numel() * 4
 
     def e2e_step():
+        # every call queues its copies and kernels on its plan's own stream: one workload's result
+        # travels to the host while the next one's operand travels to the device
         for c, (Bh, Ch) in zip(cases, hosts):
-            c["plan"].spmm_host(Bh, Ch, c["w"].alpha, c["w"].beta)
+            c["plan"].spmm_host_async(Bh, Ch, c["w"].alpha, c["w"].beta)
+        for c in cases:
+            c["plan"].sync()
 
     if e2e_steps:
         e2e_step()

@@ -143,6 +143,17 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
 sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host,
                          int64_t ldc, float alpha, float beta);
 
+/* sd_spmm_host_async / sd_plan_sync -- sd_spmm_host in two halves.  The first queues the
+ * copies and the kernels on the plan's own stream and returns; B_host and C_host must stay
+ * valid and untouched until sd_plan_sync(plan) has returned, which waits for everything
+ * queued on that stream.  Calls on DIFFERENT plans overlap on the GPU and on the bus: one
+ * plan's result travels to the host while the next plan's operand travels to the device
+ * (pinned host memory is needed for that).  Several calls on the same plan run one after the
+ * other; they share its staging buffers. */
+sd_status_t sd_spmm_host_async(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host,
+                               int64_t ldc, float alpha, float beta);
+sd_status_t sd_plan_sync(sd_plan_t *plan);
+
 /* sd_plan_destroy -- the `cleanup` entry.  Frees everything the plan owns.  NULL is a no-op. */
 void sd_plan_destroy(sd_plan_t *plan);
 

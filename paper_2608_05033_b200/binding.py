@@ -21,7 +21,7 @@ SD_F32, SD_BF16 = 0, 1
 SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
-EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_plan_destroy",
+EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_destroy",
            "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_probe_gather", "sd_last_error",
            "sd_version"]
 
@@ -74,6 +74,10 @@ def load():
                             C.c_void_p]
     lib.sd_spmm_host.restype = C.c_int
     lib.sd_spmm_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_float]
+    lib.sd_spmm_host_async.restype = C.c_int
+    lib.sd_spmm_host_async.argtypes = lib.sd_spmm_host.argtypes
+    lib.sd_plan_sync.restype = C.c_int
+    lib.sd_plan_sync.argtypes = [C.c_void_p]
     lib.sd_plan_destroy.restype = None
     lib.sd_plan_destroy.argtypes = [C.c_void_p]
     lib.sd_plan_get_info.restype = C.c_int
@@ -156,6 +160,18 @@ def sd_plan_create_ex(rowptr, colind, vals, M: int, K: int, N: int, dtype: int =
 
 def sd_spmm(plan, B, ldb: int, Cmat, ldc: int, alpha: float, beta: float, stream=None):
     rc = load().sd_spmm(plan, _ptr(B), ldb, _ptr(Cmat), ldc, alpha, beta, _stream_handle(stream))
+    if rc != SD_OK:
+        _raise(rc)
+
+
+def sd_spmm_host_async(plan, B_host, ldb: int, C_host, ldc: int, alpha: float, beta: float):
+    rc = load().sd_spmm_host_async(plan, _ptr(B_host), ldb, _ptr(C_host), ldc, alpha, beta)
+    if rc != SD_OK:
+        _raise(rc)
+
+
+def sd_plan_sync(plan):
+    rc = load().sd_plan_sync(plan)
     if rc != SD_OK:
         _raise(rc)
 
@@ -269,6 +285,16 @@ class Plan:
         ldc = C_host.strides[0] // C_host.itemsize if isinstance(C_host, np.ndarray) else C_host.stride(0)
         sd_spmm_host(self.handle, B_host, ldb, C_host, ldc, alpha, beta)
         return C_host
+
+    def spmm_host_async(self, B_host, C_host, alpha: float = 1.0, beta: float = 0.0):
+        """Queues the copies and the kernels on the plan's own stream; `sync()` waits for them."""
+        ldb = B_host.strides[0] // B_host.itemsize if isinstance(B_host, np.ndarray) else B_host.stride(0)
+        ldc = C_host.strides[0] // C_host.itemsize if isinstance(C_host, np.ndarray) else C_host.stride(0)
+        sd_spmm_host_async(self.handle, B_host, ldb, C_host, ldc, alpha, beta)
+        return C_host
+
+    def sync(self):
+        sd_plan_sync(self.handle)
 
     def device_status(self) -> int:
         return sd_plan_device_status(self.handle)

@@ -1350,7 +1350,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     }
 }
 
-sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host, int64_t ldc, float alpha,
+sd_status_t sd_spmm_host_async(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host, int64_t ldc, float alpha,
                          float beta) {
     if (!plan) {
         set_error(SD_ERR_INVALID_ARG, "plan is null");
@@ -1375,8 +1375,22 @@ sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float
         SD_CUDA_TRY(cudaMemcpy2DAsync(plan->stage_C, 4 * N, C_host, 4 * ldc, 4 * N, M, cudaMemcpyHostToDevice, st));
     if ((s = sd_spmm(plan, plan->stage_B, N, plan->stage_C, N, alpha, beta, st))) return s;
     SD_CUDA_TRY(cudaMemcpy2DAsync(C_host, 4 * ldc, plan->stage_C, 4 * N, 4 * N, M, cudaMemcpyDeviceToHost, st));
-    SD_CUDA_TRY(cudaStreamSynchronize(st));
     return SD_OK;
+}
+
+sd_status_t sd_plan_sync(sd_plan_t *plan) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->host_stream) SD_CUDA_TRY(cudaStreamSynchronize(plan->host_stream));
+    return SD_OK;
+}
+
+sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host, int64_t ldc, float alpha,
+                         float beta) {
+    const sd_status_t s = sd_spmm_host_async(plan, B_host, ldb, C_host, ldc, alpha, beta);
+    return s ? s : sd_plan_sync(plan);
 }
 
 #pragma GCC visibility pop

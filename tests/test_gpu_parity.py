@@ -309,6 +309,13 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     Ch = torch.from_numpy(Cin.copy()).pin_memory()
     plan.spmm_host(Bh, Ch, 0.5, 2.0)
     check(w2, Ch.numpy(), c_in=Cin, alpha=0.5, beta=2.0)
+    # the two-part form: two calls queued back to back on the plan's stream, one wait
+    Ca = torch.full((w.M, w.N), float("nan")).pin_memory()
+    Cb = torch.from_numpy(Cin.copy()).pin_memory()
+    plan.spmm_host_async(Bh, Ca, 1.0, 0.0)
+    plan.spmm_host_async(Bh, Cb, 0.5, 2.0)
+    plan.sync()
+    assert np.array_equal(Ca.numpy(), got2) and np.array_equal(Cb.numpy(), Ch.numpy())
     plan.close()
 
 
