@@ -136,6 +136,18 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
 sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc,
                     float alpha, float beta, void *stream);
 
+/* sd_plan_update_values -- new values for the SAME sparsity pattern (paper, Appendix "A Generated
+ * SpMM Implementation": the structure-only part of the preprocessing is reusable; e.g. edge weights
+ * that change between the epochs of a graph network).
+ *   vals   device [nnz], dtype of the plan, in the order of the colind array given at creation;
+ *          borrowed from now on in place of the previous array (which may be freed once the
+ *          work queued on `stream` has run)
+ * Row-split and row-ordered merge plans only swap the pointer; window-major plans refresh
+ * their re-bucketed copy, block plans refill the 16x16 blocks and the tensor-core images, both
+ * with kernels on `stream`: order the call before the next sd_spmm (same stream, or an event).
+ * The family, the windows and every structural decision stay as they are. */
+sd_status_t sd_plan_update_values(sd_plan_t *plan, const void *vals, void *stream);
+
 /* sd_spmm_host -- same operation with HOST buffers: B (and C when beta != 0) are
  * copied to plan-owned device staging buffers, sd_spmm runs, C is copied back, and
  * the call returns after the copy completed.  The staging buffers are allocated by

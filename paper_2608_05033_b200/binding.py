@@ -21,7 +21,7 @@ SD_F32, SD_BF16 = 0, 1
 SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
-EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_destroy",
+EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_destroy",
            "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_probe_gather", "sd_last_error",
            "sd_version"]
 
@@ -76,6 +76,8 @@ def load():
     lib.sd_spmm_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_float]
     lib.sd_spmm_host_async.restype = C.c_int
     lib.sd_spmm_host_async.argtypes = lib.sd_spmm_host.argtypes
+    lib.sd_plan_update_values.restype = C.c_int
+    lib.sd_plan_update_values.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_sync.restype = C.c_int
     lib.sd_plan_sync.argtypes = [C.c_void_p]
     lib.sd_plan_destroy.restype = None
@@ -166,6 +168,12 @@ def sd_spmm(plan, B, ldb: int, Cmat, ldc: int, alpha: float, beta: float, stream
 
 def sd_spmm_host_async(plan, B_host, ldb: int, C_host, ldc: int, alpha: float, beta: float):
     rc = load().sd_spmm_host_async(plan, _ptr(B_host), ldb, _ptr(C_host), ldc, alpha, beta)
+    if rc != SD_OK:
+        _raise(rc)
+
+
+def sd_plan_update_values(plan, vals, stream=None):
+    rc = load().sd_plan_update_values(plan, _ptr(vals), _stream_handle(stream))
     if rc != SD_OK:
         _raise(rc)
 
@@ -295,6 +303,11 @@ class Plan:
 
     def sync(self):
         sd_plan_sync(self.handle)
+
+    def update_values(self, vals, stream=None):
+        """New values for the same pattern; `vals` is borrowed from now on."""
+        sd_plan_update_values(self.handle, vals, stream)
+        self._keep = (self._keep[0], self._keep[1], vals)
 
     def device_status(self) -> int:
         return sd_plan_device_status(self.handle)

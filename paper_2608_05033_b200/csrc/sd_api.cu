@@ -323,7 +323,7 @@ template <typename T>
 __global__ void window_gather_kernel(const int32_t *__restrict__ seg_ptr2, const int32_t *__restrict__ order,
                                      const int32_t *__restrict__ seg_start, const int32_t *__restrict__ perm,
                                      const int32_t *__restrict__ colind, const T *__restrict__ vals, int64_t S, int64_t nnz,
-                                     int32_t *__restrict__ w_col, T *__restrict__ w_val) {
+                                     int32_t *__restrict__ w_col, T *__restrict__ w_val, int32_t *__restrict__ w_src) {
     const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (q >= nnz) return;
     int64_t lo = 0, hi = S;   // last segment with seg_ptr2[s] <= q and a non-zero length covers q
@@ -335,6 +335,15 @@ __global__ void window_gather_kernel(const int32_t *__restrict__ seg_ptr2, const
     const int32_t p = perm[seg_start[order[lo]] + (q - seg_ptr2[lo])];
     w_col[q] = colind[p];
     w_val[q] = vals[p];
+    w_src[q] = p;
+}
+
+// New values for an unchanged pattern: the re-bucketed copy is refreshed from the caller's array.
+template <typename T>
+__global__ void window_revalue_kernel(const int32_t *__restrict__ w_src, const T *__restrict__ vals, int64_t nnz,
+                                      T *__restrict__ w_val) {
+    const int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (q < nnz) w_val[q] = vals[w_src[q]];
 }
 
 // Chunks of the long segments: segment s (class 0) is cut into ceil(len / chunk) pieces.
@@ -392,6 +401,7 @@ struct sd_plan {
     int32_t *w_ptr = nullptr;      // plan-owned when windows > 1
     int32_t *w_col = nullptr;
     void *w_vals = nullptr;
+    int32_t *w_src = nullptr;   // position in the caller's arrays of every re-bucketed nonzero
     int32_t *w_seg_row = nullptr;
     int64_t num_segments = 0;
     int32_t *seg_chunk = nullptr;   // [S + 1] first chunk of every segment (long segments own chunks)
@@ -517,6 +527,7 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     if ((s = perm.get(4 * nnz, "permutation"))) return s;
     if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_col), 4 * nnz, "window-major colind"))) return s;
     if ((s = dev_alloc(p, &p->w_vals, es * nnz, "window-major values"))) return s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->w_src), 4 * nnz, "window-major source positions"))) return s;
 
     window_keys_kernel<<<148 * 8, 256, 0, st>>>(p->rowptr, p->colind, M, wcols, static_cast<uint32_t *>(wkey.p),
                                                static_cast<int32_t *>(rowid.p));
@@ -614,11 +625,11 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     if (p->dtype == SD_F32)
         window_gather_kernel<float><<<ceil_div(nnz, 256), 256, 0, st>>>(
             p->w_ptr, static_cast<int32_t *>(order.p), static_cast<int32_t *>(seg_start.p), static_cast<int32_t *>(perm.p),
-            p->colind, static_cast<const float *>(p->vals), S, nnz, p->w_col, static_cast<float *>(p->w_vals));
+            p->colind, static_cast<const float *>(p->vals), S, nnz, p->w_col, static_cast<float *>(p->w_vals), p->w_src);
     else
         window_gather_kernel<uint16_t><<<ceil_div(nnz, 256), 256, 0, st>>>(
             p->w_ptr, static_cast<int32_t *>(order.p), static_cast<int32_t *>(seg_start.p), static_cast<int32_t *>(perm.p),
-            p->colind, static_cast<const uint16_t *>(p->vals), S, nnz, p->w_col, static_cast<uint16_t *>(p->w_vals));
+            p->colind, static_cast<const uint16_t *>(p->vals), S, nnz, p->w_col, static_cast<uint16_t *>(p->w_vals), p->w_src);
     SD_CUDA_TRY(cudaGetLastError());
     if ((s = dbounds.get(sizeof(int64_t) * (3 * W + 1), "window bounds"))) return s;
     window_bounds_kernel<<<1, 256, 0, st>>>(static_cast<uint32_t *>(seg_key_sorted.p), S, 3 * W,
@@ -982,6 +993,7 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->w_ptr);
     cudaFree(p->w_col);
     cudaFree(p->w_vals);
+    cudaFree(p->w_src);
     cudaFree(p->w_seg_row);
     cudaFree(p->seg_chunk);
     cudaFree(p->chunk_ptr);
@@ -1347,6 +1359,46 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     default:
         set_error(SD_ERR_INTERNAL, "plan has no family");
         return SD_ERR_INTERNAL;
+    }
+}
+
+sd_status_t sd_plan_update_values(sd_plan_t *plan, const void *vals, void *stream) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->nnz == 0) return SD_OK;
+    if (!vals) {
+        set_error(SD_ERR_INVALID_ARG, "vals is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool same_copy = plan->m_vals == plan->vals;   // the kernels read the caller's array directly
+    plan->vals = vals;
+    switch (plan->info.family) {
+    case SD_MERGE:
+        if (same_copy) {
+            plan->m_vals = vals;
+        } else if (plan->w_src) {
+            const unsigned blocks = static_cast<unsigned>(ceil_div(plan->nnz, 256));
+            if (plan->dtype == SD_F32)
+                window_revalue_kernel<float><<<blocks, 256, 0, st>>>(plan->w_src, static_cast<const float *>(vals), plan->nnz,
+                                                                     static_cast<float *>(plan->w_vals));
+            else
+                window_revalue_kernel<uint16_t><<<blocks, 256, 0, st>>>(plan->w_src, static_cast<const uint16_t *>(vals),
+                                                                        plan->nnz, static_cast<uint16_t *>(plan->w_vals));
+            SD_CUDA_TRY(cudaGetLastError());
+        }
+        return SD_OK;
+    case SD_BSR_TC: {
+        const size_t es = plan->dtype == SD_F32 ? 4 : 2;
+        SD_CUDA_TRY(cudaMemsetAsync(plan->bval, 0, es * 256 * plan->nnzb, st));
+        SD_CUDA_TRY(plan->dtype == SD_F32 ? fill_bsr<float>(plan, st) : fill_bsr<__nv_bfloat16>(plan, st));
+        SD_CUDA_TRY(build_bsr_mma_image(plan->bval, plan->bval_mma, plan->nnzb, plan->dtype, st));
+        return SD_OK;
+    }
+    default:
+        return SD_OK;   // row-split reads the caller's array
     }
 }
 

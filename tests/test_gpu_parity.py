@@ -319,6 +319,49 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     plan.close()
 
 
+@pytest.mark.parametrize("case", ["rowsplit", "merge", "merge_narrow", "merge_windows", "bsr_bf16", "bsr_f32"])
+def test_update_values_same_pattern(case):
+    # new values for an unchanged pattern: every representation that holds its own copy of the values
+    # (window-major lists, 16x16 blocks and their tensor-core images) must follow
+    rng = np.random.default_rng(11)
+    dtype = W.SD_BF16 if case == "bsr_bf16" else W.SD_F32
+    if case.startswith("bsr"):
+        M, K, N = 16 * 21 + 3, 16 * 17, 128
+        lengths = np.clip(rng.poisson(40, M), 0, K)
+        family, windows = sd.SD_BSR_TC, 0
+    else:
+        M, K = 2100, 4000
+        N = 3 if case == "merge_narrow" else 32
+        lengths = shape_lengths("skewed", M, K, rng)
+        family = sd.SD_ROWSPLIT if case == "rowsplit" else sd.SD_MERGE
+        windows = 4 if case == "merge_windows" else 0
+    w = W.random_csr(M, K, N, lengths, seed=77, dtype=dtype, alpha=1.0, beta=0.0)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=family, windows=windows)
+    got, _ = run_spmm(plan, w)
+    check(w, got)
+    # second set of values, same pattern
+    v2 = np.random.default_rng(12).standard_normal(w.nnz).astype(np.float32)
+    w2 = W.Workload(w.name, w.M, w.K, w.N, w.rowptr, w.colind, W.f32_to_bf16_bits(v2) if dtype == W.SD_BF16 else v2,
+                    w.B, None, 1.0, 0.0, dtype, {})
+    from util import dev
+    vals2 = dev(w2.vals)
+    plan.update_values(vals2)
+    got2, _ = run_spmm(plan, w2)
+    assert plan.device_status() == 0
+    check(w2, got2)
+    assert not np.array_equal(got, got2)
+    if case.startswith("bsr"):
+        browptr, bcol, bval = sd.sd_plan_get_bsr(plan.handle)
+        rb, rc, rv = oracle.bsr16(w2.rowptr, w2.colind, w2.vals, M, K)
+        assert np.array_equal(browptr, rb) and np.array_equal(bcol, rc) and bval.tobytes() == rv.tobytes()
+    if case == "merge_windows":
+        seg_ptr, seg_row, colind, vals, win_seg = sd.sd_plan_get_segments(plan.handle)
+        rp, rr, perm, rw = oracle.window_segments(w2.rowptr, w2.colind, M, K, 4)
+        assert np.array_equal(colind, w2.colind[perm]) and vals.tobytes() == w2.vals[perm].tobytes()
+    plan.close()
+
+
 @pytest.mark.parametrize("N", [1, 2, 3, 4])
 @pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
 def test_merge_narrow_operand_all_carry_levels(N, dtype):
