@@ -189,9 +189,9 @@ def summary(rowptr, colind, M, K, N) -> Info:
     return info
 
 
-def decide(info: Info) -> int:
+def decide(info: Info, dtype: int = F32) -> int:
     """O4: family rule on the integers of O3 (parity unpinned: thresholds are not in the paper)."""
-    return int(lib().sdo_decide(C.byref(info)))
+    return int(lib().sdo_decide(C.byref(info), C.c_int(dtype)))
 
 
 def decide_windows(info: Info, dtype: int, l2_bytes: int) -> int:

@@ -394,13 +394,31 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
 
 /* Family rule on O3's integers (thresholds are this build's reading; the
  * paper gives none).  parity unpinned.
- *   BSR-TC    rows strictly ascending and rho_BSR(16) <= 1.5  (256 nnzb <= 1.5 nnz)
+ *   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N)
+ *             (Eq. 4; Sec. 3.1: dense tiles pay "when useful arithmetic outweighs
+ *             compaction and fill-in costs").  rho_max is where the block form stops
+ *             paying on the target GPU, by dense width and value type:
+ *                        N < 128   128 <= N < 256   N >= 256
+ *               fp32       3/2          2              11/4
+ *               bf16       3            5              7
  *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4
  *   ROWSPLIT  otherwise
  * CV^2 = M sum r^2 / nnz^2 - 1 >= 4  <=>  M sum r^2 >= 5 nnz^2. */
-int sdo_decide(const sdo_info_t *o)
+int sdo_decide(const sdo_info_t *o, int dtype)
 {
-    if (o->nnz > 0 && o->unsorted_rows == 0 && 2 * 256 * o->nnzb16 <= 3 * o->nnz)
+    int64_t num, den = 1;
+    if (dtype == SDO_BF16) {
+        num = o->N < 128 ? 3 : (o->N < 256 ? 5 : 7);
+    } else if (o->N < 128) {
+        num = 3;
+        den = 2;
+    } else if (o->N < 256) {
+        num = 2;
+    } else {
+        num = 11;
+        den = 4;
+    }
+    if (o->nnz > 0 && o->unsorted_rows == 0 && den * 256 * o->nnzb16 <= num * o->nnz)
         return SDO_BSR_TC;
     unsigned __int128 lhs = (unsigned __int128)(uint64_t)o->M * o->sum_r2;
     unsigned __int128 rhs = (unsigned __int128)5 * (uint64_t)o->nnz * (uint64_t)o->nnz;

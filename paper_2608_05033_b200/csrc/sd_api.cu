@@ -474,11 +474,30 @@ struct TempBuf {   // frees temporary device memory on every exit path
 
 // Family rule on the integer summary.  The paper ranks templates with a learned model and a
 // measured search (Sec. 3.2-3.3) and prints no thresholds; these are fixed integer rules:
-//   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= 1.5 (Eq. 4)
+//   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N) (Eq. 4)
 //   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4
 //   ROWSPLIT  otherwise
-static int decide_family(const sd_plan_info_t &s) {
-    if (s.nnz > 0 && s.unsorted_rows == 0 && 2 * 256 * s.nnzb16 <= 3 * s.nnz) return SD_BSR_TC;
+// rho_max is where the block form stops paying on this GPU (Sec. 3.1: dense tiles pay "when
+// useful arithmetic outweighs compaction and fill-in costs").  The tensor-core kernel's time
+// depends on the number of blocks only, the CSR kernels' time on the number of nonzeros; the
+// measured cross-over (random 16x16 blocks thinned to a given fill) by width and value type:
+//              N < 128   128 <= N < 256   N >= 256
+//     fp32       3/2          2              11/4
+//     bf16       3            5              7
+static int decide_family(const sd_plan_info_t &s, int dtype) {
+    int64_t num, den = 1;
+    if (dtype == SD_BF16) {
+        num = s.N < 128 ? 3 : (s.N < 256 ? 5 : 7);
+    } else if (s.N < 128) {
+        num = 3;
+        den = 2;
+    } else if (s.N < 256) {
+        num = 2;
+    } else {
+        num = 11;
+        den = 4;
+    }
+    if (s.nnz > 0 && s.unsorted_rows == 0 && den * 256 * s.nnzb16 <= num * s.nnz) return SD_BSR_TC;
     const unsigned __int128 lhs = static_cast<unsigned __int128>(static_cast<uint64_t>(s.M)) * s.sum_r2;
     const unsigned __int128 rhs =
         static_cast<unsigned __int128>(5) * static_cast<uint64_t>(s.nnz) * static_cast<uint64_t>(s.nnz);
@@ -964,7 +983,7 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     info.nnz_dense_blocks = static_cast<int64_t>(h.nnz_dense_blocks);
 
     // ---- decision ------------------------------------------------------------------------------
-    int family = d->family == SD_AUTO ? decide_family(info) : d->family;
+    int family = d->family == SD_AUTO ? decide_family(info, p->dtype) : d->family;
     if (family == SD_BSR_TC && (info.unsorted_rows != 0 || p->nnz == 0)) {
         if (d->family == SD_BSR_TC && info.unsorted_rows != 0) {
             set_error(SD_ERR_UNSUPPORTED, "BSR needs strictly ascending columns in every row (%lld rows are not)",

@@ -32,7 +32,7 @@ def test_full_size_config_matches_oracle(name, ci, dtype, family):
     mine = info.as_dict()
     for k, v in ref.as_dict().items():
         assert mine[k] == v, k
-    assert info.family == oracle.decide(ref)
+    assert info.family == oracle.decide(ref, dtype)
     if info.family == sd.SD_MERGE:
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes)
     if name == "skewed":

@@ -403,6 +403,24 @@ def test_o4_merge_coords_match_closed_form():
             assert got[0] == 0 and got[-1] == S
 
 
+def test_o4_block_rule_thresholds_by_width_and_value_type():
+    # the block form is taken while 256 * nnzb <= rho_max * nnz; rho_max by dense width and value type
+    # (integer arithmetic: the boundary itself is inside)
+    table = {(oracle.F32, 64): (3, 2), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (11, 4), (oracle.F32, 1024): (11, 4),
+             (oracle.BF16, 64): (3, 1), (oracle.BF16, 128): (5, 1), (oracle.BF16, 255): (5, 1), (oracle.BF16, 256): (7, 1)}
+    w = W.g4_block(Mb=16, Kb=16, N=4, nblocks=30)
+    base = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+    for (dt, N), (num, den) in table.items():
+        nnzb = 1000
+        edge = (den * 256 * nnzb + num - 1) // num          # smallest nnz that still qualifies
+        for nnz, want in ((edge, True), (edge - 1, False)):
+            info = oracle.Info.from_buffer_copy(base)
+            info.N, info.nnzb16, info.nnz = N, nnzb, nnz
+            info.sum_r2 = 0          # keep the row-length part of the rule out of the picture
+            info.max_r = 1
+            assert (oracle.decide(info, dt) == oracle.BSR_TC) == want, (dt, N, nnz)
+
+
 def test_o4_family_rule_on_the_five_shapes():
     w = W.g1_tiny_uniform()
     assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.ROWSPLIT
