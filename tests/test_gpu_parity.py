@@ -362,6 +362,24 @@ def test_update_values_same_pattern(case):
     plan.close()
 
 
+@pytest.mark.parametrize("lengths", [[1], [128], [129], [0, 0, 1, 0], [1000], [0, 127, 1, 0, 128, 0], [5] * 257,
+                                     [0] * 40 + [300] + [0] * 40, [1] * 128 + [2] * 64])
+def test_merge_narrow_operand_chunk_edges(lengths):
+    # the 128-nonzero chunks of the narrow-width path: lists that end exactly on a chunk, one nonzero
+    # past it, a single row over several chunks, rows that end exactly on chunk and 32-lane
+    # boundaries, empty rows at both ends
+    lengths = np.asarray(lengths, np.int64)
+    M, K = len(lengths), 1200
+    for N in (1, 4):
+        w = W.random_csr(M, K, N, lengths, seed=int(lengths.sum()) + N, alpha=2.0, beta=0.5)
+        dw = DeviceWorkload(w)
+        plan = dw.plan(family=sd.SD_MERGE)
+        got, intact = run_spmm(plan, w)
+        assert intact
+        check(w, got)
+        plan.close()
+
+
 @pytest.mark.parametrize("N", [1, 2, 3, 4])
 @pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
 def test_merge_narrow_operand_all_carry_levels(N, dtype):
