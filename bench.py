@@ -65,7 +65,7 @@ def ncu_traffic():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) during the timed region."""
 
-    def __init__(self, index: int, period: float = 0.02):
+    def __init__(self, index: int, period: float = 0.002):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
