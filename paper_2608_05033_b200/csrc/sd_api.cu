@@ -411,6 +411,8 @@ struct sd_plan {
     // window-major plans run the three independent segment classes of a window side by side
     cudaStream_t aux[2] = {nullptr, nullptr};
     cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr};
+    cudaStream_t chunk_stream = nullptr;     // the chunk kernels of all windows run ahead on a stream of their own
+    std::vector<cudaEvent_t> ev_chunk;       // one per window: its chunk sums are complete
     struct Window {
         int64_t seg_begin, seg_end;     // segments of the merge-path kernel (all of them without windows)
         int64_t short_begin, short_end; // segments of the group-per-segment kernel (windows only)
@@ -767,6 +769,9 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
             SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
         }
         SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+        SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
+        p->ev_chunk.assign(W, nullptr);
+        for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
     }
     if (W > 1) {   // chunk ranges of the long segments
         std::vector<int32_t> cb(2 * W, 0);
@@ -1041,6 +1046,9 @@ static void free_plan(sd_plan *p) {
         if (p->ev_join[i]) cudaEventDestroy(p->ev_join[i]);
     }
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->chunk_stream) cudaStreamDestroy(p->chunk_stream);
+    for (cudaEvent_t e : p->ev_chunk)
+        if (e) cudaEventDestroy(e);
     delete p;
 }
 
@@ -1279,6 +1287,43 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         a.seg_row = plan->m_seg_row;
         a.S = plan->num_segments;
         const bool side = plan->wins.size() > 1 && plan->aux[0] && !getenv("SD_NO_SIDE_STREAMS");
+        // The chunk kernels only read A and B and write their own scratch rows: they run on a stream of
+        // their own, up to `depth` windows ahead of the kernels that update C, which wait for their
+        // window's event.
+        const bool ahead = side && plan->chunk_stream && !getenv("SD_NO_CHUNK_AHEAD");
+        auto launch_chunks = [&](size_t w, cudaStream_t cs) -> sd_status_t {
+            const sd_plan::Window &win = plan->wins[w];
+            SpmmArgs ca = a;
+            ca.ptr = plan->chunk_ptr + win.chunk_begin + w;
+            ca.seg_row = nullptr;
+            ca.S = win.chunk_end - win.chunk_begin;
+            ca.C = plan->chunk_out + win.chunk_begin * N;
+            ca.ldc = N;
+            ca.alpha = 1.f;
+            ca.beta = 0.f;
+            SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, cs));
+            return SD_OK;
+        };
+        const size_t depth = 2;   // windows the chunk stream may be ahead (measured: 2 is as good as all of them, and keeps
+                                  // fewer slabs of B competing for L2)
+        size_t chunks_issued = 0;
+        auto issue_chunks_upto = [&](size_t upto) -> sd_status_t {   // windows [chunks_issued, upto)
+            for (; chunks_issued < upto && chunks_issued < plan->wins.size(); ++chunks_issued) {
+                const size_t w = chunks_issued;
+                if (plan->wins[w].chunk_end > plan->wins[w].chunk_begin) {
+                    sd_status_t cs = launch_chunks(w, plan->chunk_stream);
+                    if (cs) return cs;
+                }
+                SD_CUDA_TRY(cudaEventRecord(plan->ev_chunk[w], plan->chunk_stream));
+            }
+            return SD_OK;
+        };
+        if (ahead) {
+            SD_CUDA_TRY(cudaEventRecord(plan->ev_fork, st));
+            SD_CUDA_TRY(cudaStreamWaitEvent(plan->chunk_stream, plan->ev_fork, 0));
+            sd_status_t cs = issue_chunks_upto(depth);
+            if (cs) return cs;
+        }
         for (size_t w = 0; w < plan->wins.size(); ++w) {   // windows run in order
             const sd_plan::Window &win = plan->wins[w];
             // Inside a window every row belongs to one segment, so the three classes touch disjoint
@@ -1300,15 +1345,12 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
             if (win.chunk_end > win.chunk_begin) {
                 // long segments: every chunk is summed by one lane group into its own scratch row,
                 // then each segment adds its chunks in order and updates its row of C
-                SpmmArgs ca = a;
-                ca.ptr = plan->chunk_ptr + win.chunk_begin + w;
-                ca.seg_row = nullptr;
-                ca.S = win.chunk_end - win.chunk_begin;
-                ca.C = plan->chunk_out + win.chunk_begin * N;
-                ca.ldc = N;
-                ca.alpha = 1.f;
-                ca.beta = 0.f;
-                SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, st));
+                if (ahead) {
+                    SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_chunk[w], 0));
+                } else {
+                    sd_status_t cs = launch_chunks(w, st);
+                    if (cs) return cs;
+                }
                 SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->seg_chunk, a.seg_row, win.seg_begin, win.seg_end, C,
                                              ldc, static_cast<int32_t>(N), alpha, beta, st));
             }
@@ -1335,6 +1377,12 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
                 SD_CUDA_TRY(cudaEventRecord(plan->ev_join[1], s_single));
                 SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[1], 0));
             }
+            if (ahead && chunks_issued < plan->wins.size()) {   // window w is done: the chunk stream may go one further
+                SD_CUDA_TRY(cudaEventRecord(plan->ev_join[0], st));
+                SD_CUDA_TRY(cudaStreamWaitEvent(plan->chunk_stream, plan->ev_join[0], 0));
+                sd_status_t cs = issue_chunks_upto(chunks_issued + 1);
+                if (cs) return cs;
+            }
             if (win.ntiles == 0) continue;
             MergeArgs m;
             m.s = a;
@@ -1347,6 +1395,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
             SD_CUDA_TRY(run_merge(m, plan->dtype, vec, plan->fix_short + win.tile_base, win.nshort,
                                   plan->fix_long + win.tile_base, win.nlong, st));
         }
+        if (ahead) SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_chunk.back(), 0));   // the caller's stream covers everything
         return SD_OK;
     }
     case SD_BSR_TC: {
