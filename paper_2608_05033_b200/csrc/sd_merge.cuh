@@ -43,6 +43,10 @@ merge_tile_kernel(const MergeArgs m) {
     __shared__ uint8_t has_end_s[G], open_s[G];
     __shared__ int32_t first_end_s;
 
+    // head_s / tail_s rows are stored element-major, slot(v, e) = e * (LPR * NV) + v * LPR + lg: for a
+    // fixed element the lanes of a group touch consecutive words (no bank conflicts); slot k holds
+    // column (k % (LPR * NV)) * VW + k / (LPR * NV) of the slab
+    constexpr int LN = LPR * NV;
     const SpmmArgs &a = m.s;
     const T *__restrict__ vals = static_cast<const T *>(a.vals);
     const int tid = threadIdx.x;
@@ -153,7 +157,7 @@ merge_tile_kernel(const MergeArgs m) {
 #pragma unroll
             for (int v = 0; v < NV; ++v)
 #pragma unroll
-                for (int e = 0; e < VW; ++e) head_s[g * CP + (v * LPR + lg) * VW + e] = acc[v][e];
+                for (int e = 0; e < VW; ++e) head_s[g * CP + e * LN + v * LPR + lg] = acc[v][e];
         } else {
             // the group saw this segment from its first nonzero: finished here
             const int64_t sg = seg0 + s;
@@ -177,7 +181,7 @@ merge_tile_kernel(const MergeArgs m) {
 #pragma unroll
     for (int v = 0; v < NV; ++v)
 #pragma unroll
-        for (int e = 0; e < VW; ++e) tail_s[g * CP + (v * LPR + lg) * VW + e] = acc[v][e];
+        for (int e = 0; e < VW; ++e) tail_s[g * CP + e * LN + v * LPR + lg] = acc[v][e];
     if (lg == 0) {
         has_end_s[g] = seen_end;
         open_s[g] = open;
@@ -197,7 +201,8 @@ merge_tile_kernel(const MergeArgs m) {
                 tail_s[gg * CP + tid] = run;
                 run = has_end_s[gg] ? tv : run + tv;
             }
-            if (cbase + tid < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + tid] = run;
+            const int col = (tid % LN) * VW + tid / LN;   // the column this slot holds
+            if (cbase + col < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + col] = run;
         }
     } else {
         // few columns, many groups: segmented scan across groups with warp shuffles
@@ -223,7 +228,8 @@ merge_tile_kernel(const MergeArgs m) {
                 run = __shfl_sync(FULLMASK, v, 31);
                 tail_s[gg * CP + c] = ex;   // now the carry-in of group gg
             }
-            if (lane == 0 && cbase + c < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + c] = run;
+            const int col = (c % LN) * VW + c / LN;   // the column this slot holds
+            if (lane == 0 && cbase + col < a.N) m.tile_tail[static_cast<int64_t>(t) * a.N + cbase + col] = run;
         }
     }
     __syncthreads();
@@ -238,7 +244,7 @@ merge_tile_kernel(const MergeArgs m) {
         for (int v = 0; v < NV; ++v)
 #pragma unroll
             for (int e = 0; e < VW; ++e) {
-                const int c = (v * LPR + lg) * VW + e;
+                const int c = e * LN + v * LPR + lg;
                 r[v][e] = tail_s[g * CP + c] + head_s[g * CP + c];
             }
         if (g == first_end && tile_open) {
