@@ -818,8 +818,9 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
     // Narrow dense operands take the COO segmented reduction instead of the tile kernel (the tile
     // table above stays valid and inspectable): one row index per nonzero and two carry lists.
     if (W == 1 && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !getenv("SD_NO_COO")) {
-        const int64_t chunks1 = (p->nnz + kCooChunk - 1) / kCooChunk, count2 = 2 * chunks1;
-        const int64_t chunks2 = (count2 + kCooChunk - 1) / kCooChunk, count3 = 2 * chunks2;
+        const int cchunk = coo_chunk(static_cast<int>(p->N));
+        const int64_t chunks1 = (p->nnz + cchunk - 1) / cchunk, count2 = 2 * chunks1;
+        const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk, count3 = 2 * chunks2;
         if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_row), sizeof(int32_t) * p->nnz, "row index per nonzero"))) return s;
         if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_row), sizeof(int32_t) * count2, "carry rows"))) return s;
         if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_val), sizeof(float) * count2 * p->N, "carry sums"))) return s;

@@ -4,7 +4,8 @@
 //
 // With one to eight columns a lane group per row has nothing to share: the generic merge kernel
 // spends its time on per-lane searches and block-wide phases.  Here a warp owns 128 consecutive
-// nonzeros (four coalesced loads of row, column and value per lane, four gathers of B in flight),
+// nonzeros (256 at one or two columns: four or eight coalesced loads of row, column and value per lane, as many
+// gathers of B in flight),
 // multiplies, and reduces equal-row runs with warp shuffles; no shared memory, no block barrier.
 //
 // Rows are ascending in storage order, so a row is one run.  A run that lies strictly inside a
@@ -68,6 +69,8 @@ coo_reduce_kernel(const CooArgs a) {
     constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    constexpr int kCooChunk = LEVEL2 ? kCooCarryChunk : coo_chunk(N);
+    constexpr int kCooU = kCooChunk / 32;   // items per lane and warp step
     const int64_t chunks = (a.count + kCooChunk - 1) / kCooChunk;
     const T *__restrict__ vals = static_cast<const T *>(a.vals);
     const float *__restrict__ pvals = static_cast<const float *>(a.vals);
@@ -76,11 +79,11 @@ coo_reduce_kernel(const CooArgs a) {
         const int64_t k0 = c * kCooChunk + lane;
         const bool whole = (c + 1) * kCooChunk <= a.count;   // warp-uniform: no item of the chunk is past the end
         // ---- four items per lane: loads first, all gathers in flight together ------------------
-        int r[4];
-        float p[4][N];
+        int r[kCooU];
+        float p[kCooU][N];
         if constexpr (LEVEL2) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kCooU; ++u) {
                 const int64_t k = k0 + u * 32;
                 const bool ok = whole || k < a.count;
                 r[u] = ok ? __ldg(a.row + k) : -1;
@@ -88,10 +91,10 @@ coo_reduce_kernel(const CooArgs a) {
                 for (int e = 0; e < N; ++e) p[u][e] = ok ? __ldg(pvals + k * N + e) : 0.f;
             }
         } else {
-            int col[4];
-            float av[4];
+            int col[kCooU];
+            float av[kCooU];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kCooU; ++u) {
                 const int64_t k = k0 + u * 32;
                 const bool ok = whole || k < a.count;
                 r[u] = ok ? __ldg(a.row + k) : -1;
@@ -99,9 +102,9 @@ coo_reduce_kernel(const CooArgs a) {
                 av[u] = ok ? to_float(vals[k]) : 0.f;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) coo_gather<T, N, VEC>(a.B, col[u], a.ldb_bytes, p[u]);
+            for (int u = 0; u < kCooU; ++u) coo_gather<T, N, VEC>(a.B, col[u], a.ldb_bytes, p[u]);
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < kCooU; ++u)
 #pragma unroll
                 for (int e = 0; e < N; ++e) p[u][e] *= av[u];
         }
@@ -110,12 +113,12 @@ coo_reduce_kernel(const CooArgs a) {
             const int last_u = static_cast<int>((last - c * kCooChunk) >> 5), last_l = static_cast<int>(last & 31);
             int pad_row = 0;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kCooU; ++u) {
                 const int t = __shfl_sync(FULL, r[u], last_l);
                 if (u == last_u) pad_row = t;
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < kCooU; ++u)
                 if (r[u] < 0) r[u] = pad_row;
         }
 
@@ -138,7 +141,7 @@ coo_reduce_kernel(const CooArgs a) {
         for (int e = 0; e < N; ++e) cval[e] = 0.f;
 
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kCooU; ++u) {
             // where runs start among these 32 items: one ballot replaces a row exchange per scan step
             const int rp = __shfl_up_sync(FULL, r[u], 1);
             const unsigned starts = __ballot_sync(FULL, lane == 0 || rp != r[u]);

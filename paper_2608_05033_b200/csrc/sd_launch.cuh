@@ -48,14 +48,17 @@ constexpr int kMergeLongChain = 8;   // chains of at least this many tiles go to
 // gain; measured cross-over between 4 and 8 columns): segmented reduction over the nonzeros with an
 // explicit row index per nonzero, carries reduced in two more levels.  C must hold beta * C_in.
 constexpr int kCooMaxN = 4;
-constexpr int kCooChunk = 128;             // nonzeros per warp step
+// nonzeros per warp step: 8 per lane at one or two columns (the gathers are 4 or 8 bytes: more of them
+// must be in flight; measured), 4 per lane at three or four; carry lists are always cut into 128-entry chunks
+constexpr int coo_chunk(int N) { return N <= 2 ? 256 : 128; }
+constexpr int kCooCarryChunk = 128;
 constexpr int64_t kCooDirectFinal = 4096;  // carry lists up to this length skip the second level
 struct CooPlan {
     const int32_t *row;   // [nnz] row of every nonzero
     int64_t nnz;
-    int32_t *c1_row;      // [2 * ceil(nnz / kCooChunk)] first-level carries
+    int32_t *c1_row;      // [2 * ceil(nnz / coo_chunk(N))] first-level carries
     float *c1_val;        // ... x N
-    int32_t *c2_row;      // [2 * ceil(len(c1) / kCooChunk)] second-level carries
+    int32_t *c2_row;      // [2 * ceil(len(c1) / kCooCarryChunk)] second-level carries
     float *c2_val;
 };
 cudaError_t run_coo(const CooPlan &cp, const SpmmArgs &s, int dtype, bool vec, int sm_count, cudaStream_t st);

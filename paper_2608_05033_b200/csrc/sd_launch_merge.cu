@@ -26,9 +26,9 @@ cudaError_t run_merge(const MergeArgs &m, int dtype, bool vec, const int32_t *fi
 // ---- narrow dense operands: COO segmented reduction --------------------------------------------
 template <typename T, int N>
 static cudaError_t launch_coo_n(const CooPlan &cp, const SpmmArgs &s, bool vec, int sm_count, cudaStream_t st) {
-    const int64_t chunks1 = (cp.nnz + kCooChunk - 1) / kCooChunk;
+    const int64_t chunks1 = (cp.nnz + coo_chunk(N) - 1) / coo_chunk(N);
     const int64_t count2 = 2 * chunks1;
-    const int64_t chunks2 = (count2 + kCooChunk - 1) / kCooChunk;
+    const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk;
     const int64_t count3 = 2 * chunks2;
     auto grid_for = [&](int64_t chunks) {
         const int64_t want = (chunks + 7) / 8;   // 8 warps per CTA, one chunk per warp step

@@ -385,17 +385,18 @@ def test_merge_narrow_operand_chunk_edges(lengths):
 def test_merge_narrow_operand_all_carry_levels(N, dtype):
     # dense widths up to 4 take the segmented reduction over (row, column, value) triples: enough
     # nonzeros that its carry list goes through the second level, one row holding every column (it
-    # spans about two thousand 128-nonzero chunks), runs of empty rows, one-nonzero rows, a padded
+    # spans one to two thousand chunks), runs of empty rows, one-nonzero rows, a padded
     # and misaligned B
     rng = np.random.default_rng(N)
     M, K = 5003, 260_000
-    lengths = np.clip((5000.0 * np.arange(1, M + 1) ** -0.9).astype(np.int64), 1, 5000)
+    lengths = np.clip((40000.0 * np.arange(1, M + 1) ** -0.9).astype(np.int64), 1, 30000)
     lengths = rng.permutation(lengths)
     lengths[100:140] = 0
     lengths[M // 2] = K
     lengths[M - 1] = 0
     w = W.random_csr(M, K, N, lengths, seed=40 + N, dtype=dtype, alpha=0.75, beta=-1.5)
-    assert 2 * ((w.nnz + 127) // 128) > 4096   # the first carry list is longer than the direct-final limit
+    chunk = 256 if N <= 2 else 128
+    assert 2 * ((w.nnz + chunk - 1) // chunk) > 4096   # the first carry list is longer than the direct-final limit
     dw = DeviceWorkload(w)
     plan = dw.plan(family=sd.SD_MERGE)
     assert plan.info().launches == 4
