@@ -828,7 +828,7 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
         if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_val), sizeof(float) * count3 * p->N, "carry sums (level 2)"))) return s;
         SD_CUDA_TRY(build_coo_rows(p->rowptr, p->M, p->nnz, p->coo_row, st));
         SD_CUDA_TRY(cudaStreamSynchronize(st));
-        p->info.launches = 3 + (count2 > kCooDirectFinal);
+        p->info.launches = 2 + (count2 > kCooDirectFinal);
     }
     return SD_OK;
 }
@@ -1267,12 +1267,13 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         SD_CUDA_TRY(run_rowsplit(a, plan->dtype, vec, st));
         return SD_OK;
     case SD_MERGE: {
-        if (plan->coo_row) {   // narrow dense operand: C = beta * C, then one writer per row adds alpha * (A B)
-            if (beta != 1.f) SD_CUDA_TRY(run_scale_c(C, ldc, M, static_cast<int32_t>(N), beta, st));
+        if (plan->coo_row) {   // narrow dense operand: one writer per row
             a.colind = plan->colind;
             a.vals = plan->vals;
             CooPlan cp;
             cp.row = plan->coo_row;
+            cp.rowptr = plan->rowptr;
+            cp.M = plan->info.empty_rows > 0 ? M : 0;   // no search for rows without nonzeros when the scan found none
             cp.nnz = plan->nnz;
             cp.c1_row = plan->coo_c1_row;
             cp.c1_val = plan->coo_c1_val;

@@ -9,12 +9,13 @@
 // multiplies, and reduces equal-row runs with warp shuffles; no shared memory, no block barrier.
 //
 // Rows are ascending in storage order, so a row is one run.  A run that lies strictly inside a
-// warp's 128 nonzeros is complete: its lane adds alpha * sum to C (C was scaled by beta before).
+// warp's 128 nonzeros is complete: its lane writes alpha * sum + beta * C.
 // The first and the last run of a chunk may continue in the neighbours: their sums go to a carry
 // list, two entries per chunk in chunk order, (first row, sum) and (last row, sum) -- a chunk
 // that is one single run writes (row, sum) and (row, 0), so that entries of one row stay
 // adjacent.  The carry list is itself a row-sorted list of values: the same kernel reduces it
 // (level 2), and the few entries that level leaves over are added one run per thread (level 3).
+// Rows without nonzeros are found from the row pointers by the first level and get beta * C.
 // Every row is written by exactly one thread and every sum has a fixed order: results are
 // reproducible bit for bit, no float atomics.
 #pragma once
@@ -33,7 +34,9 @@ struct CooArgs {
     int64_t count;           // items
     float *C;
     int64_t ldc;
-    float alpha;
+    float alpha, beta;
+    const int32_t *rowptr;   // level 1: [M + 1], to find the rows without nonzeros (they get beta * C)
+    int64_t M;
     int32_t *carry_row;      // [2 * chunks] out
     float *carry_val;        // [2 * chunks][N] out
 };
@@ -76,6 +79,19 @@ coo_reduce_kernel(const CooArgs a) {
     const float *__restrict__ pvals = static_cast<const float *>(a.vals);
 
     for (int64_t c = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; c < chunks; c += warps) {
+        if constexpr (!LEVEL2) {
+            // rows without nonzeros have no writer among the runs: this chunk looks after its share of them
+            const int64_t rpc = (a.M + chunks - 1) / chunks;
+            for (int64_t rr = c * rpc + lane; rr < min(a.M, (c + 1) * rpc); rr += 32) {
+                if (__ldg(a.rowptr + rr) == __ldg(a.rowptr + rr + 1)) {
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        float *pc = a.C + rr * a.ldc + e;
+                        *pc = (a.beta != 0.f) ? a.beta * *pc : 0.f;
+                    }
+                }
+            }
+        }
         const int64_t k0 = c * kCooChunk + lane;
         const bool whole = (c + 1) * kCooChunk <= a.count;   // warp-uniform: no item of the chunk is past the end
         // ---- four items per lane: loads first, all gathers in flight together ------------------
@@ -132,7 +148,10 @@ coo_reduce_kernel(const CooArgs a) {
                 for (int e = 0; e < N; ++e) a.carry_val[(2 * c) * N + e] = v[e];
             } else {
 #pragma unroll
-                for (int e = 0; e < N; ++e) a.C[static_cast<int64_t>(row) * a.ldc + e] += a.alpha * v[e];
+                for (int e = 0; e < N; ++e) {
+                    float *pc = a.C + static_cast<int64_t>(row) * a.ldc + e;
+                    *pc = (a.beta != 0.f) ? fmaf(a.beta, *pc, a.alpha * v[e]) : a.alpha * v[e];
+                }
             }
         };
         int crow = first_row;   // the run that reached the end of the previous 32 items ...
@@ -191,7 +210,7 @@ coo_reduce_kernel(const CooArgs a) {
 // Level 3: one thread per run of equal rows in a short carry list.
 template <int N>
 __global__ void coo_final_kernel(const int32_t *__restrict__ row, const float *__restrict__ val, int64_t count, float *C,
-                                 int64_t ldc, float alpha) {
+                                 int64_t ldc, float alpha, float beta) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= count) return;
     const int r = row[i];
@@ -203,7 +222,10 @@ __global__ void coo_final_kernel(const int32_t *__restrict__ row, const float *_
 #pragma unroll
         for (int e = 0; e < N; ++e) s[e] += val[j * N + e];
 #pragma unroll
-    for (int e = 0; e < N; ++e) C[static_cast<int64_t>(r) * ldc + e] += alpha * s[e];
+    for (int e = 0; e < N; ++e) {
+        float *pc = C + static_cast<int64_t>(r) * ldc + e;
+        *pc = (beta != 0.f) ? fmaf(beta, *pc, alpha * s[e]) : alpha * s[e];
+    }
 }
 
 // Row index of every nonzero (plan time).

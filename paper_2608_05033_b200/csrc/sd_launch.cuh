@@ -46,7 +46,7 @@ constexpr int kMergeLongChain = 8;   // chains of at least this many tiles go to
 
 // Family (b) for dense widths up to kCooMaxN (beyond it the shuffles per nonzero outweigh the
 // gain; measured cross-over between 4 and 8 columns): segmented reduction over the nonzeros with an
-// explicit row index per nonzero, carries reduced in two more levels.  C must hold beta * C_in.
+// explicit row index per nonzero, carries reduced in two more levels.
 constexpr int kCooMaxN = 4;
 // nonzeros per warp step: 8 per lane at one or two columns (the gathers are 4 or 8 bytes: more of them
 // must be in flight; measured), 4 per lane at three or four; carry lists are always cut into 128-entry chunks
@@ -55,6 +55,8 @@ constexpr int kCooCarryChunk = 128;
 constexpr int64_t kCooDirectFinal = 4096;  // carry lists up to this length skip the second level
 struct CooPlan {
     const int32_t *row;   // [nnz] row of every nonzero
+    const int32_t *rowptr; // [M + 1]
+    int64_t M;             // rows to search for empty ones (0: the matrix has none)
     int64_t nnz;
     int32_t *c1_row;      // [2 * ceil(nnz / coo_chunk(N))] first-level carries
     float *c1_val;        // ... x N

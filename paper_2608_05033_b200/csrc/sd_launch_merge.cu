@@ -45,6 +45,9 @@ static cudaError_t launch_coo_n(const CooPlan &cp, const SpmmArgs &s, bool vec, 
     a.C = s.C;
     a.ldc = s.ldc;
     a.alpha = s.alpha;
+    a.beta = s.beta;
+    a.rowptr = cp.rowptr;
+    a.M = cp.M;
     a.carry_row = cp.c1_row;
     a.carry_val = cp.c1_val;
     if (vec) coo_reduce_kernel<T, N, true, false><<<grid_for(chunks1), 256, 0, st>>>(a);
@@ -69,7 +72,7 @@ static cudaError_t launch_coo_n(const CooPlan &cp, const SpmmArgs &s, bool vec, 
         fval = cp.c2_val;
         fcount = count3;
     }
-    coo_final_kernel<N><<<static_cast<unsigned>((fcount + 255) / 256), 256, 0, st>>>(frow, fval, fcount, s.C, s.ldc, s.alpha);
+    coo_final_kernel<N><<<static_cast<unsigned>((fcount + 255) / 256), 256, 0, st>>>(frow, fval, fcount, s.C, s.ldc, s.alpha, s.beta);
     return cudaGetLastError();
 }
 
@@ -84,7 +87,7 @@ static cudaError_t launch_coo(const CooPlan &cp, const SpmmArgs &s, bool vec, in
     }
 }
 
-// `vec`: B is 16-byte aligned and its row pitch a multiple of 16 bytes.  C must hold beta * C_in.
+// `vec`: B is 16-byte aligned and its row pitch a multiple of 16 bytes.
 cudaError_t run_coo(const CooPlan &cp, const SpmmArgs &s, int dtype, bool vec, int sm_count, cudaStream_t st) {
     return dtype == SD_F32 ? launch_coo<float>(cp, s, vec, sm_count, st) : launch_coo<__nv_bfloat16>(cp, s, vec, sm_count, st);
 }
