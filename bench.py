@@ -454,6 +454,96 @@ def run_gpu(args, rank, local_rank, world):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- GCN epoch mode
+def run_gcn_epoch(args, local_rank):
+    """Sparse aggregations of a two-layer full-batch GCN (paper, Sec. 5 "End-to-End Application
+    Evaluation"): four products with the normalised adjacency per epoch, two forward (features,
+    hidden activations) and two backward (their gradients); the adjacency is symmetric, so the
+    backward products reuse the forward plan.  One plan per dense width, made once; the dense
+    layers and activations of the training loop are not this library's work and are not run.
+    Prints one JSON line of its own (not the benchmark line)."""
+    import torch
+    import paper_2608_05033_b200 as sd
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    sd.load()
+    stream = torch.cuda.current_stream()
+    kw = dict(SMALL_KW[2]) if args.small else {}
+    base = W.config(2, dtype=W.SD_F32, N=8, **kw)
+    rowptr = torch.from_numpy(base.rowptr).to(dev)
+    colind = torch.from_numpy(base.colind).to(dev)
+    vals = torch.from_numpy(base.vals).to(dev)
+    warm, epochs = max(args.warmup, 3), args.steps
+    rows = []
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for width in (8, 32, 128, 256):
+        t0 = time.time()
+        plan = sd.Plan(rowptr, colind, vals, base.M, base.K, width, dtype=W.SD_F32)
+        torch.cuda.synchronize()
+        plan_ms = (time.time() - t0) * 1e3
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(W.SEED_BASE + width)
+        # features, hidden activations and the two gradients: four different operands per epoch
+        ops = [torch.randn((base.K, width), dtype=torch.float32, device=dev, generator=gen) for _ in range(4)]
+        outs = [torch.empty((base.M, width), dtype=torch.float32, device=dev) for _ in range(2)]
+
+        def epoch():
+            for i, X in enumerate(ops):
+                plan.spmm(X, outs[i & 1], 1.0, 0.0, stream)
+
+        for _ in range(warm):
+            epoch()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(epochs):
+            epoch()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / epochs
+        info = plan.info()
+        row = {"width": width, "aggregation_ms_per_epoch": ms, "ms_per_product": ms / 4,
+               "gflops": 4 * 2.0 * base.nnz * width / (ms * 1e-3) / 1e9, "family": sd.FAMILY_NAMES[info.family],
+               "launches_per_product": int(info.launches), "plan_ms": plan_ms,
+               "operand_mb": base.K * width * 4 / 1e6}
+        if args.cusparse:
+            try:
+                A = torch.sparse_csr_tensor(rowptr.long(), colind.long(), vals, size=(base.M, base.K))
+                for _ in range(3):
+                    for X in ops:
+                        torch.sparse.mm(A, X)
+                torch.cuda.synchronize()
+                n_ctx = max(3, epochs // 10)
+                e0.record(stream)
+                for _ in range(n_ctx):
+                    for X in ops:
+                        torch.sparse.mm(A, X)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                row["context_cusparse_ms_per_epoch"] = e0.elapsed_time(e1) / n_ctx
+                row["context_speedup_over_cusparse"] = row["context_cusparse_ms_per_epoch"] / ms
+                del A
+            except Exception as exc:   # context only
+                row["context_cusparse_error"] = str(exc)[:120]
+        rows.append(row)
+        plan.close()
+        del ops, outs
+    clocks = sampler.stop()
+    print(json.dumps({
+        "mode": "gcn-epoch", "metric": "gcn_sparse_aggregation_ms_per_epoch", "unit": "ms", "higher_is_better": False,
+        "n_gpus": 1, "epochs": epochs, "warmup_epochs": warm, "data": "synthetic", "dtype": "f32",
+        "config": {"workload": f"{base.name}: symmetrised R-MAT + I, D^-1/2 (A+I) D^-1/2, M = {base.M}, nnz = {base.nnz}; "
+                               "four products per epoch on four different dense operands, one plan per width reused "
+                               "for the forward and the backward products (symmetric adjacency)",
+                   "l2": "no flush inside an epoch; the four operands and two results of a width together exceed the "
+                         "126 MB L2 from width 8 on (6 x 33.5 MB at width 8)"},
+        "clocks": clocks, "per_width": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -475,10 +565,18 @@ def main():
                     help="reduced sizes of the same workloads (dense operands still above the L2 size where "
                          "the full-size ones are); for profiler captures, not a bench number")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer and CPU-baseline legs")
+    ap.add_argument("--gcn-epoch", action="store_true",
+                    help="time the four sparse aggregations of a two-layer GCN epoch on the R-MAT adjacency at dense "
+                         "widths 8, 32, 128, 256 (--steps epochs after --warmup epochs; the paper averages 100 after "
+                         "10); one GPU, prints its own JSON line")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.gcn_epoch:
+        if rank == 0:
+            run_gcn_epoch(args, local_rank)
         return
     run_gpu(args, rank, local_rank, world)
     if world > 1:

@@ -319,6 +319,31 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     plan.close()
 
 
+@pytest.mark.parametrize("N", [8, 32, 128])
+def test_symmetric_adjacency_forward_plan_serves_the_backward_product(N):
+    """Sec. 5, GCN evaluation: the backward aggregation is a product with the transposed adjacency;
+    the normalised adjacency is symmetric, so the forward plan serves it.  The oracle gets the
+    explicitly transposed CSR (a counting-sort transpose written here), the library the forward plan."""
+    w = W.config(2, scale=12, N=N)
+    M, nnz = w.M, w.nnz
+    rows = np.repeat(np.arange(M, dtype=np.int64), np.diff(w.rowptr))
+    order = np.lexsort((rows, w.colind))                      # transpose: sort by (column, row)
+    t_rowptr = np.zeros(M + 1, np.int32)
+    np.cumsum(np.bincount(w.colind, minlength=M), out=t_rowptr[1:])
+    t_colind = rows[order].astype(np.int32)
+    t_vals = w.vals[order]
+    assert np.array_equal(t_rowptr, w.rowptr) and np.array_equal(t_colind, w.colind)   # pattern symmetric
+    assert np.array_equal(t_vals, w.vals)                                               # values symmetric, bit for bit
+    G = np.random.default_rng(N).standard_normal((M, N)).astype(np.float32)            # an upstream gradient
+    dw = DeviceWorkload(w)
+    plan = dw.plan()
+    w.B = G
+    got, _ = run_spmm(plan, w)
+    r = oracle.check(t_rowptr, t_colind, t_vals, G, N, got, None, 1.0, 0.0)
+    assert r["ok"], r
+    plan.close()
+
+
 @pytest.mark.parametrize("case", ["rowsplit", "merge", "merge_narrow", "merge_windows", "bsr_bf16", "bsr_f32"])
 def test_update_values_same_pattern(case):
     # new values for an unchanged pattern: every representation that holds its own copy of the values
