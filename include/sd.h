@@ -172,6 +172,56 @@ void sd_plan_destroy(sd_plan_t *plan);
 /* sd_plan_get_info -- structure summary and decision (host struct out). */
 sd_status_t sd_plan_get_info(const sd_plan_t *plan, sd_plan_info_t *out);
 
+/* Extended structure analysis (Sec. 3.1: row-length quartiles, column-degree statistics,
+ * the value-slot expansion of padded and blocked layouts of Eq. 4 with their storage
+ * estimates; Sec. 3.3, Eq. 10-13: footprint, working sets, work units).  Exact integers;
+ * ratios (rho = slots / nnz, q_R = m_r / l2_bytes, ...) are left to the caller.
+ * Quartiles are nearest-rank: the ceil(q*n/4)-th smallest of n values, q = 1, 2, 3
+ * (0 when n == 0).  SELL slices are c consecutive rows in storage order (no sorting
+ * window); the last slice may be shorter and counts its own rows only. */
+typedef enum {
+    SD_SHAPE_UNIFORM = 0,  /* CV^2 <= 1/16 */
+    SD_SHAPE_MODERATE = 1, /* none of the others */
+    SD_SHAPE_SKEWED = 2,   /* CV^2 >= 1 */
+    SD_SHAPE_POWERLAW = 3, /* CV^2 >= 4 and max r >= 64 x mean r */
+    SD_SHAPE_BIMODAL = 4   /* two row_hist bins at least 3 apart hold >= 1/4 of the non-empty rows each */
+} sd_shape_t;              /* tested in the order UNIFORM, BIMODAL, POWERLAW, SKEWED, MODERATE */
+
+typedef struct {
+    int64_t row_q[3];      /* quartiles of the row length r_i over the M rows */
+    int64_t col_q[3];      /* quartiles of the column degree d_j over the K columns */
+    int64_t col_max;       /* max_j d_j */
+    int64_t col_empty;     /* columns without a stored entry */
+    uint64_t sum_d2;       /* sum of d_j^2 */
+    int64_t ell_slots;     /* M * max_i r_i                          (rho_ELL numerator) */
+    int64_t sell_slots[3]; /* sum over slices |s| max_{i in s} r_i,  c = 16, 32, 512 */
+    int64_t nnzb[3];       /* occupied b x b blocks,                 b = 4, 8, 16 */
+    /* storage estimates, value type of the plan, 32-bit indices:
+     * [0] CSR (vb+4) nnz + 4 (M+1);  [1] ELL (vb+4) slots;
+     * [2..4] SELL-16/32/512 (vb+4) slots + 4 (slices+1);
+     * [5..7] BSR-4/8/16 (vb b^2 + 4) nnzb + 4 (ceil(M/b)+1) */
+    int64_t rep_bytes[8];
+    int32_t shape_class;   /* sd_shape_t */
+    int32_t value_bytes;   /* vb: 4 or 2 */
+    /* the plan as built (Eq. 10-13) */
+    int64_t borrowed_bytes; /* caller's CSR arrays that sd_spmm reads: all three for SD_ROWSPLIT and for
+                               SD_MERGE without windows, none otherwise */
+    int64_t plan_bytes;     /* device memory owned by the plan: representation, tables, scratch */
+    int64_t d_r, d_s;       /* dense B: K N vb;  dense C: 4 M N */
+    int64_t m_r, m_t;       /* m_r = borrowed + plan + d_r;  m_t = m_r + d_s */
+    int64_t work_units;     /* rows (SD_ROWSPLIT), tiles (SD_MERGE), (row, window) segments (SD_MERGE with
+                               windows), block-rows (SD_BSR_TC) */
+    int32_t sm_count;
+    int32_t reserved;
+    int64_t l2_bytes;
+} sd_features_t;
+
+/* sd_plan_get_features -- computes the analysis above on the device at the first call
+ * (a few sorts over M, K and nnz keys: temporary device memory of about 40 bytes per nonzero,
+ * freed before returning; synchronous) and keeps it in the plan.  Needs the CSR arrays given
+ * at creation to be still valid.  Not thread-safe against other calls on the same plan. */
+sd_status_t sd_plan_get_features(sd_plan_t *plan, sd_features_t *out);
+
 /* sd_plan_get_bsr -- copy the BSR-16 representation (Sec. 3.1, Eq. 4) to HOST arrays:
  * browptr int32 [ceil(M/16)+1], bcol int32 [nnzb16] ascending inside a block-row,
  * bval [nnzb16][16][16] row-major in the plan dtype, absent slots +0.  Any pointer may

@@ -263,3 +263,58 @@ def working_set_bytes(rep_bytes: int, info: Info, value_bytes: int = 4, workspac
     dense B; total adds dense C (fp32)."""
     m_r = rep_bytes + workspace + info.K * info.N * value_bytes
     return m_r, m_r + info.M * info.N * 4
+
+
+# ---- O5: extended structure analysis (Sec. 3.1, Eq. 4, Eq. 10) ----
+SHAPE_NAMES = {0: "uniform", 1: "moderate", 2: "skewed", 3: "power-law", 4: "bimodal"}
+
+
+class Features(C.Structure):
+    _fields_ = [("row_q", C.c_int64 * 3), ("col_q", C.c_int64 * 3), ("col_max", C.c_int64), ("col_empty", C.c_int64),
+                ("sum_d2", C.c_uint64), ("ell_slots", C.c_int64), ("sell_slots", C.c_int64 * 3),
+                ("nnzb", C.c_int64 * 3), ("rep_bytes", C.c_int64 * 8), ("shape_class", C.c_int32),
+                ("value_bytes", C.c_int32)]
+
+    def as_dict(self) -> dict:
+        d = {}
+        for name, _ in self._fields_:
+            v = getattr(self, name)
+            d[name] = list(v) if hasattr(v, "__len__") else int(v)
+        return d
+
+
+def quartile(values, q: int) -> int:
+    """Nearest-rank quartile: the ceil(q n / 4)-th smallest (0 for no values)."""
+    v = np.ascontiguousarray(values, dtype=np.int32)
+    lib().sdo_quartile.restype = C.c_int64
+    return int(lib().sdo_quartile(_p(v), C.c_int64(v.size), C.c_int(q)))
+
+
+def sell_slots(rowptr, c: int) -> int:
+    """Numerator of rho_SELL(c) (Eq. 4), slices of c consecutive rows in storage order."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    lib().sdo_sell_slots.restype = C.c_int64
+    return int(lib().sdo_sell_slots(C.c_int64(rowptr.size - 1), _p(rowptr), C.c_int64(c)))
+
+
+def block_count(rowptr, colind, b: int) -> int:
+    """nnzb_b of Eq. 4: occupied b x b blocks."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    colind = np.ascontiguousarray(colind, dtype=np.int32)
+    lib().sdo_block_count.restype = C.c_int64
+    return int(lib().sdo_block_count(C.c_int64(rowptr.size - 1), _p(rowptr), _p(colind), C.c_int64(b)))
+
+
+def shape_class(info: Info) -> int:
+    """Row-length shape class (parity unpinned: the paper names the classes, not the cut-offs)."""
+    return int(lib().sdo_shape_class(C.byref(info)))
+
+
+def features(rowptr, colind, M, K, info: Info, value_bytes: int = 4) -> Features:
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    colind = np.ascontiguousarray(colind, dtype=np.int32)
+    f = Features()
+    rc = lib().sdo_features(C.c_int64(M), C.c_int64(K), _p(rowptr), _p(colind), C.c_int(value_bytes),
+                            C.byref(info), C.byref(f))
+    assert rc == 0
+    return f

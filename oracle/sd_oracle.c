@@ -539,3 +539,161 @@ int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const i
     free(key);
     return S;
 }
+
+/* ------------------------------------------------------------------ O5 */
+/* Extended structure analysis: Sec. 3.1 (row-length quartiles, column-degree statistics,
+ * shape class), Eq. 4 (value-slot expansion of ELL, SELL(c), BSR(b)) and the storage
+ * estimates of the candidate layouts (Eq. 10).  Every function is the definition written out. */
+
+/* Nearest-rank quartile: the ceil(q n / 4)-th smallest of n values (q = 1, 2, 3); 0 for n = 0. */
+int64_t sdo_quartile(const int32_t *v, int64_t n, int q)
+{
+    if (n <= 0)
+        return 0;
+    int32_t *t = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+    memcpy(t, v, sizeof(int32_t) * (size_t)n);
+    qsort(t, (size_t)n, sizeof(int32_t), cmp_i32);
+    int64_t rank = (q * n + 3) / 4;
+    int64_t r = t[rank - 1];
+    free(t);
+    return r;
+}
+
+/* Eq. 4, rho_SELL(c) numerator: slices of c consecutive rows in storage order (the formula
+ * names no sorting window), sum over slices of |s| * max_{i in s} r_i; |s| of the last slice
+ * is the number of rows it really holds. */
+int64_t sdo_sell_slots(int64_t M, const int32_t *rowptr, int64_t c)
+{
+    int64_t total = 0;
+    for (int64_t r0 = 0; r0 < M; r0 += c) {
+        int64_t r1 = r0 + c < M ? r0 + c : M, mx = 0;
+        for (int64_t i = r0; i < r1; ++i) {
+            int64_t r = (int64_t)rowptr[i + 1] - rowptr[i];
+            if (r > mx)
+                mx = r;
+        }
+        total += (r1 - r0) * mx;
+    }
+    return total;
+}
+
+/* Eq. 4, nnzb_b: number of b x b blocks (I, J) for which some stored entry has
+ * row / b == I and col / b == J.  Any b >= 1. */
+int64_t sdo_block_count(int64_t M, const int32_t *rowptr, const int32_t *colind, int64_t b)
+{
+    int64_t total = 0, cap = 0;
+    int32_t *t = NULL;
+    for (int64_t r0 = 0; r0 < M; r0 += b) {
+        int64_t r1 = r0 + b < M ? r0 + b : M;
+        int64_t n = (int64_t)rowptr[r1] - rowptr[r0];
+        if (n > cap) {
+            free(t);
+            cap = n + n / 2 + 16;
+            t = (int32_t *)malloc(sizeof(int32_t) * (size_t)cap);
+        }
+        for (int64_t p = rowptr[r0], k = 0; p < rowptr[r1]; ++p, ++k)
+            t[k] = (int32_t)(colind[p] / b);
+        qsort(t, (size_t)n, sizeof(int32_t), cmp_i32);
+        for (int64_t k = 0; k < n; ++k)
+            if (k == 0 || t[k] != t[k - 1])
+                ++total;
+    }
+    free(t);
+    return total;
+}
+
+#define SDO_SHAPE_UNIFORM 0
+#define SDO_SHAPE_MODERATE 1
+#define SDO_SHAPE_SKEWED 2
+#define SDO_SHAPE_POWERLAW 3
+#define SDO_SHAPE_BIMODAL 4
+
+/* Shape class of the row-length distribution (Sec. 3.1 names the five classes and prints no
+ * cut-offs: this build's reading, parity unpinned).  With CV^2 = M sum r^2 / nnz^2 - 1, tested
+ * in this order:
+ *   uniform    CV^2 <= 1/16
+ *   bimodal    two bins of the power-of-two row-length histogram, at least 3 bins apart,
+ *              each hold at least a quarter of the non-empty rows
+ *   power-law  CV^2 >= 4 and max r >= 64 * mean r
+ *   skewed     CV^2 >= 1
+ *   moderate   otherwise                                                               */
+int sdo_shape_class(const sdo_info_t *o)
+{
+    if (o->nnz <= 0 || o->M <= 0)
+        return SDO_SHAPE_UNIFORM;
+    unsigned __int128 m_r2 = (unsigned __int128)(uint64_t)o->M * o->sum_r2;
+    unsigned __int128 nnz2 = (unsigned __int128)(uint64_t)o->nnz * (uint64_t)o->nnz;
+    /* CV^2 <= 1/16  <=>  16 (M sum r^2 - nnz^2) <= nnz^2 */
+    if (16 * m_r2 <= 17 * nnz2)
+        return SDO_SHAPE_UNIFORM;
+    int64_t nonempty = o->M - o->empty_rows;
+    for (int b1 = 1; b1 < 32; ++b1)
+        for (int b2 = b1 + 3; b2 < 32; ++b2)
+            if (4 * o->row_hist[b1] >= nonempty && 4 * o->row_hist[b2] >= nonempty)
+                return SDO_SHAPE_BIMODAL;
+    unsigned __int128 max_m = (unsigned __int128)(uint64_t)o->max_r * (uint64_t)o->M;
+    if (m_r2 >= 5 * nnz2 && max_m >= (unsigned __int128)64 * (uint64_t)o->nnz)
+        return SDO_SHAPE_POWERLAW;
+    if (m_r2 >= 2 * nnz2)
+        return SDO_SHAPE_SKEWED;
+    return SDO_SHAPE_MODERATE;
+}
+
+typedef struct {
+    int64_t row_q[3];      /* quartiles of r_i */
+    int64_t col_q[3];      /* quartiles of the column degree d_j */
+    int64_t col_max, col_empty;
+    uint64_t sum_d2;
+    int64_t ell_slots;     /* M max r */
+    int64_t sell_slots[3]; /* c = 16, 32, 512 */
+    int64_t nnzb[3];       /* b = 4, 8, 16 */
+    int64_t rep_bytes[8];  /* CSR, ELL, SELL-16/32/512, BSR-4/8/16 */
+    int32_t shape_class, value_bytes;
+} sdo_features_t;
+
+/* Storage estimates (Eq. 10: value slots x bytes per value + metadata fields x their width,
+ * 32-bit indices): CSR values + column indices + row pointers; ELL one value and one column
+ * index per slot; SELL the same per slot plus slice offsets; BSR b^2 values and one
+ * block-column index per occupied block plus block-row pointers. */
+int sdo_features(int64_t M, int64_t K, const int32_t *rowptr, const int32_t *colind,
+                 int value_bytes, const sdo_info_t *info, sdo_features_t *o)
+{
+    memset(o, 0, sizeof *o);
+    int64_t nnz = M > 0 ? rowptr[M] : 0, vb = value_bytes;
+    int32_t *len = (int32_t *)malloc(sizeof(int32_t) * (size_t)(M > 0 ? M : 1));
+    int64_t max_r = 0;
+    for (int64_t i = 0; i < M; ++i) {
+        len[i] = rowptr[i + 1] - rowptr[i];
+        if (len[i] > max_r)
+            max_r = len[i];
+    }
+    int32_t *deg = (int32_t *)calloc((size_t)(K > 0 ? K : 1), sizeof(int32_t));
+    for (int64_t p = 0; p < nnz; ++p)
+        deg[colind[p]] += 1;
+    for (int q = 1; q <= 3; ++q) {
+        o->row_q[q - 1] = sdo_quartile(len, M, q);
+        o->col_q[q - 1] = sdo_quartile(deg, K, q);
+    }
+    for (int64_t j = 0; j < K; ++j) {
+        if (deg[j] > o->col_max)
+            o->col_max = deg[j];
+        if (deg[j] == 0)
+            o->col_empty += 1;
+        o->sum_d2 += (uint64_t)deg[j] * (uint64_t)deg[j];
+    }
+    free(len);
+    free(deg);
+    o->ell_slots = M * max_r;
+    const int64_t heights[3] = {16, 32, 512}, bs[3] = {4, 8, 16};
+    o->value_bytes = value_bytes;
+    o->rep_bytes[0] = (vb + 4) * nnz + 4 * (M + 1);
+    o->rep_bytes[1] = (vb + 4) * o->ell_slots;
+    for (int k = 0; k < 3; ++k) {
+        o->sell_slots[k] = sdo_sell_slots(M, rowptr, heights[k]);
+        o->rep_bytes[2 + k] = (vb + 4) * o->sell_slots[k] + 4 * ((M + heights[k] - 1) / heights[k] + 1);
+        o->nnzb[k] = sdo_block_count(M, rowptr, colind, bs[k]);
+        o->rep_bytes[5 + k] = (vb * bs[k] * bs[k] + 4) * o->nnzb[k] + 4 * ((M + bs[k] - 1) / bs[k] + 1);
+    }
+    o->shape_class = sdo_shape_class(info);
+    return 0;
+}

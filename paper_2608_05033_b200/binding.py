@@ -22,7 +22,7 @@ SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_probe_gather", "sd_last_error",
+           "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_probe_gather", "sd_last_error",
            "sd_version"]
 
 
@@ -51,6 +51,18 @@ class sd_plan_info_t(C.Structure):
             v = getattr(self, name)
             d[name] = list(v) if hasattr(v, "__len__") else int(v)
         return d
+
+
+SHAPE_NAMES = {0: "uniform", 1: "moderate", 2: "skewed", 3: "power-law", 4: "bimodal"}
+
+
+class sd_features_t(C.Structure):
+    _fields_ = [("row_q", C.c_int64 * 3), ("col_q", C.c_int64 * 3), ("col_max", C.c_int64), ("col_empty", C.c_int64),
+                ("sum_d2", C.c_uint64), ("ell_slots", C.c_int64), ("sell_slots", C.c_int64 * 3), ("nnzb", C.c_int64 * 3),
+                ("rep_bytes", C.c_int64 * 8), ("shape_class", C.c_int32), ("value_bytes", C.c_int32),
+                ("borrowed_bytes", C.c_int64), ("plan_bytes", C.c_int64), ("d_r", C.c_int64), ("d_s", C.c_int64),
+                ("m_r", C.c_int64), ("m_t", C.c_int64), ("work_units", C.c_int64), ("sm_count", C.c_int32),
+                ("reserved", C.c_int32), ("l2_bytes", C.c_int64)]
 
 
 _lib = None
@@ -84,6 +96,8 @@ def load():
     lib.sd_plan_destroy.argtypes = [C.c_void_p]
     lib.sd_plan_get_info.restype = C.c_int
     lib.sd_plan_get_info.argtypes = [C.c_void_p, C.POINTER(sd_plan_info_t)]
+    lib.sd_plan_get_features.restype = C.c_int
+    lib.sd_plan_get_features.argtypes = [C.c_void_p, C.POINTER(sd_features_t)]
     lib.sd_plan_get_bsr.restype = C.c_int
     lib.sd_plan_get_bsr.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_get_tiles.restype = C.c_int
@@ -223,6 +237,14 @@ def sd_plan_get_info(plan) -> sd_plan_info_t:
     return info
 
 
+def sd_plan_get_features(plan) -> sd_features_t:
+    f = sd_features_t()
+    rc = load().sd_plan_get_features(plan, C.byref(f))
+    if rc != SD_OK:
+        _raise(rc)
+    return f
+
+
 def sd_plan_get_bsr(plan):
     info = sd_plan_get_info(plan)
     Mb = (info.M + 15) // 16
@@ -314,6 +336,9 @@ class Plan:
 
     def info(self) -> sd_plan_info_t:
         return sd_plan_get_info(self.handle)
+
+    def features(self) -> sd_features_t:
+        return sd_plan_get_features(self.handle)
 
     def close(self):
         if self.handle:

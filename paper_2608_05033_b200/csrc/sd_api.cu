@@ -451,6 +451,9 @@ struct sd_plan {
     cudaStream_t host_stream = nullptr;
 
     int64_t owned = 0;
+
+    sd_features_t feat{};       // extended analysis, computed at the first sd_plan_get_features
+    bool have_feat = false;
 };
 
 namespace sd {
@@ -1140,6 +1143,86 @@ sd_status_t sd_plan_get_info(const sd_plan_t *plan, sd_plan_info_t *out) {
         return SD_ERR_INVALID_ARG;
     }
     *out = plan->info;
+    return SD_OK;
+}
+
+// Row-length shape class on the integers of the summary (Sec. 3.1 names five classes and gives no
+// cut-offs; the rule is stated beside sd_shape_t).  CV^2 = M sum r^2 / nnz^2 - 1.
+static int shape_class_of(const sd_plan_info_t &s) {
+    if (s.nnz <= 0 || s.M <= 0) return SD_SHAPE_UNIFORM;
+    using u128 = unsigned __int128;
+    const u128 m_r2 = static_cast<u128>(static_cast<uint64_t>(s.M)) * s.sum_r2;
+    const u128 nnz2 = static_cast<u128>(static_cast<uint64_t>(s.nnz)) * static_cast<uint64_t>(s.nnz);
+    if (16 * m_r2 <= 17 * nnz2) return SD_SHAPE_UNIFORM;
+    const int64_t nonempty = s.M - s.empty_rows;
+    int first = -1, last = -1;
+    for (int b = 1; b < 32; ++b) {
+        if (4 * s.row_hist[b] >= nonempty) {
+            if (first < 0) first = b;
+            last = b;
+        }
+    }
+    if (first >= 0 && last - first >= 3) return SD_SHAPE_BIMODAL;
+    if (m_r2 >= 5 * nnz2 && static_cast<u128>(static_cast<uint64_t>(s.max_r)) * static_cast<uint64_t>(s.M) >=
+                                static_cast<u128>(64) * static_cast<uint64_t>(s.nnz))
+        return SD_SHAPE_POWERLAW;
+    if (m_r2 >= 2 * nnz2) return SD_SHAPE_SKEWED;
+    return SD_SHAPE_MODERATE;
+}
+
+sd_status_t sd_plan_get_features(sd_plan_t *plan, sd_features_t *out) {
+    if (!plan || !out) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_get_features: null argument");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (!plan->have_feat) {
+        int prev = 0;
+        SD_CUDA_TRY(cudaGetDevice(&prev));
+        SD_CUDA_TRY(cudaSetDevice(plan->device));
+        FeatureCounts fc;
+        const sd_status_t s = compute_feature_counts(plan->rowptr, plan->colind, plan->M, plan->K, plan->nnz, nullptr, &fc);
+        cudaSetDevice(prev);
+        if (s) return s;
+        const sd_plan_info_t &info = plan->info;
+        sd_features_t f{};
+        for (int k = 0; k < 3; ++k) {
+            f.row_q[k] = fc.row_q[k];
+            f.col_q[k] = fc.col_q[k];
+            f.sell_slots[k] = fc.sell_slots[k];
+        }
+        f.col_max = fc.col_max;
+        f.col_empty = fc.col_empty;
+        f.sum_d2 = fc.sum_d2;
+        f.ell_slots = info.M * info.max_r;
+        f.nnzb[0] = fc.nnzb4;
+        f.nnzb[1] = fc.nnzb8;
+        f.nnzb[2] = info.nnzb16;
+        const int64_t vb = plan->dtype == SD_BF16 ? 2 : 4;
+        f.value_bytes = static_cast<int32_t>(vb);
+        f.rep_bytes[0] = (vb + 4) * info.nnz + 4 * (info.M + 1);
+        f.rep_bytes[1] = (vb + 4) * f.ell_slots;
+        const int64_t heights[3] = {16, 32, 512};
+        for (int k = 0; k < 3; ++k)
+            f.rep_bytes[2 + k] = (vb + 4) * f.sell_slots[k] + 4 * ((info.M + heights[k] - 1) / heights[k] + 1);
+        const int64_t bs[3] = {4, 8, 16};
+        for (int k = 0; k < 3; ++k)
+            f.rep_bytes[5 + k] = (vb * bs[k] * bs[k] + 4) * f.nnzb[k] + 4 * ((info.M + bs[k] - 1) / bs[k] + 1);
+        f.shape_class = shape_class_of(info);
+        const bool reads_csr = info.family == SD_ROWSPLIT || (info.family == SD_MERGE && info.windows <= 1);
+        f.borrowed_bytes = reads_csr ? f.rep_bytes[0] : 0;
+        f.plan_bytes = info.plan_bytes;
+        f.d_r = info.K * info.N * vb;
+        f.d_s = 4 * info.M * info.N;
+        f.m_r = f.borrowed_bytes + f.plan_bytes + f.d_r;
+        f.m_t = f.m_r + f.d_s;
+        f.work_units = info.family == SD_MERGE ? (info.windows > 1 ? info.num_segments : info.num_tiles)
+                                               : (info.family == SD_BSR_TC ? (info.M + 15) / 16 : info.M);
+        f.sm_count = info.sm_count;
+        f.l2_bytes = info.l2_bytes;
+        plan->feat = f;
+        plan->have_feat = true;
+    }
+    *out = plan->feat;
     return SD_OK;
 }
 

@@ -86,6 +86,17 @@ cudaError_t run_bsr_simt(const BsrArgs &a, int dtype, bool vec, cudaStream_t st)
 // Tensor-core form.  bsr_tc_usable: dtype, dense width and the TMA alignment rules allow it.
 bool bsr_tc_usable(const BsrArgs &a, int dtype);
 cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_count, cudaStream_t st);
+// Counts behind sd_plan_get_features (row-length / column-degree quartiles, column-degree moments,
+// SELL slots for slice heights 16 / 32 / 512, occupied 4x4 and 8x8 blocks).  Synchronous.
+struct FeatureCounts {
+    int64_t row_q[3], col_q[3], col_max, col_empty;
+    uint64_t sum_d2;
+    int64_t sell_slots[3];
+    int64_t nnzb4, nnzb8;
+};
+sd_status_t compute_feature_counts(const int32_t *rowptr, const int32_t *colind, int64_t M, int64_t K, int64_t nnz,
+                                   cudaStream_t st, FeatureCounts *out);
+
 cudaError_t build_bsr_partition(const int32_t *browptr, int32_t Mb, int32_t nparts, int32_t *part, cudaStream_t st);
 cudaError_t build_bsr_mma_image(const void *bval, void *img, int64_t nnzb, int dtype, cudaStream_t st);
 

@@ -35,6 +35,12 @@ def test_full_size_config_matches_oracle(name, ci, dtype, family):
     assert info.family == oracle.decide(ref, dtype)
     if info.family == sd.SD_MERGE:
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes)
+    if name not in NARROW:   # extended analysis (quartiles, column degrees, SELL / BSR slots), every count exact
+        fo = oracle.features(w.rowptr, w.colind, w.M, w.K, ref, 4 if dtype == W.SD_F32 else 2)
+        fm = plan.features()
+        for k, v in fo.as_dict().items():
+            g = getattr(fm, k)
+            assert (list(g) if hasattr(g, "__len__") else int(g)) == v, k
     if name == "skewed":
         assert w.nnz == 59_839_586 and info.windows == 8
     if name == "stencil":

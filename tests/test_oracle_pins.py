@@ -509,3 +509,115 @@ def test_o4_window_rule():
     info.unsorted_rows = 0
     info.K = 100_000
     assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 1     # B fits
+
+
+# ------------------------------------------------------------------ O5
+def _features_of(w, value_bytes=4):
+    info = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+    return info, oracle.features(w.rowptr, w.colind, w.M, w.K, info, value_bytes)
+
+
+def test_o5_quartiles_are_nearest_rank():
+    # hand case: 1..8 -> the 2nd, 4th and 6th smallest
+    assert [oracle.quartile(np.arange(8, 0, -1), q) for q in (1, 2, 3)] == [2, 4, 6]
+    assert [oracle.quartile([7], q) for q in (1, 2, 3)] == [7, 7, 7]
+    assert oracle.quartile([], 2) == 0
+    # the library's inverted-CDF percentile is the same definition
+    rng = np.random.default_rng(5)
+    for n in (2, 3, 4, 5, 7, 100, 1001):
+        v = rng.integers(0, 50, n).astype(np.int32)
+        for q in (1, 2, 3):
+            assert oracle.quartile(v, q) == int(np.percentile(v, 25 * q, method="inverted_cdf")), (n, q)
+
+
+def test_o5_sell_slots_special_cases_and_hand_example():
+    lengths = np.array([3, 1, 0, 5, 2], np.int64)
+    rowptr = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    # slices {3,1}, {0,5}, {2}: 2*3 + 2*5 + 1*2
+    assert oracle.sell_slots(rowptr, 2) == 18
+    assert oracle.sell_slots(rowptr, 1) == lengths.sum()              # no padding with one row per slice
+    assert oracle.sell_slots(rowptr, 5) == 5 * 5                      # one slice = ELL
+    assert oracle.sell_slots(rowptr, 512) == 5 * 5                    # a short last slice counts its own rows only
+    rng = np.random.default_rng(6)
+    lengths = rng.poisson(9, 3000)
+    rowptr = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    chain = [oracle.sell_slots(rowptr, c) for c in (1, 2, 4, 8, 16, 32, 512, 4096)]
+    assert chain[0] == lengths.sum() and chain[-1] == 3000 * lengths.max()
+    assert all(a <= b for a, b in zip(chain, chain[1:]))              # merging slices never removes padding
+    uniform = np.arange(0, 7 * 1000 + 1, 7, dtype=np.int32)
+    assert all(oracle.sell_slots(uniform, c) == 7000 for c in (16, 32, 512))
+
+
+def test_o5_block_count_brute_force_and_closed_forms():
+    rng = np.random.default_rng(7)
+    for M, K, dens in ((37, 53, 0.08), (64, 64, 0.3), (100, 9, 0.2)):
+        D = rng.random((M, K)) < dens
+        rowptr = np.concatenate([[0], np.cumsum(D.sum(1))]).astype(np.int32)
+        colind = np.nonzero(D)[1].astype(np.int32)
+        assert oracle.block_count(rowptr, colind, 1) == D.sum()
+        assert oracle.block_count(rowptr, colind, 1000) == 1
+        for b in (4, 8, 16, 5):
+            P = np.zeros(((M + b - 1) // b * b, (K + b - 1) // b * b), bool)
+            P[:M, :K] = D
+            want = int(P.reshape(P.shape[0] // b, b, P.shape[1] // b, b).any(axis=(1, 3)).sum())
+            assert oracle.block_count(rowptr, colind, b) == want, (M, K, b)
+        info = oracle.summary(rowptr, colind, M, K, 1)
+        assert oracle.block_count(rowptr, colind, 16) == info.nnzb16
+    # 5-point stencil on an n x n grid, natural ordering, b | n: a block-row is b consecutive points of
+    # one grid line: its own block, the left / right neighbour blocks, one block in the line above / below
+    for n, b in ((32, 4), (32, 8), (48, 16)):
+        w = W.g2_stencil(n=n, N=1)
+        nb = n // b
+        assert oracle.block_count(w.rowptr, w.colind, b) == n * nb + 2 * n * (nb - 1) + 2 * (n - 1) * nb
+
+
+def test_o5_column_degrees_are_the_row_lengths_of_the_transpose():
+    sp = pytest.importorskip("scipy.sparse")
+    w = W.g5_skewed(M=3000, N=1, scale_c=2.4e7 / 1024, cap=400)
+    _, f = _features_of(w)
+    At = sp.csr_matrix((np.ones(w.nnz, np.float32), w.colind, w.rowptr), shape=(w.M, w.K)).T.tocsr()
+    At.sort_indices()
+    t = oracle.summary(At.indptr.astype(np.int32), At.indices.astype(np.int32), w.K, w.M, 1)
+    assert (f.col_max, f.col_empty, f.sum_d2) == (t.max_r, t.empty_rows, t.sum_r2)
+    deg = np.bincount(w.colind, minlength=w.K)
+    assert list(f.col_q) == [int(np.percentile(deg, 25 * q, method="inverted_cdf")) for q in (1, 2, 3)]
+    lengths = np.diff(w.rowptr)
+    assert list(f.row_q) == [int(np.percentile(lengths, 25 * q, method="inverted_cdf")) for q in (1, 2, 3)]
+
+
+def test_o5_storage_estimates_paper_example_and_hand_case():
+    # Sec. 3.3 worked example: m = 17,281, nnz = 553,562, longest row 62 -> CSR 4,497,624 B, rho_ELL ~ 1.9
+    g = read_golden("sec3_3_shen_e40r0100.txt")
+    m, nnz, mx = int(g["m"]), int(g["nnz"]), int(g["max_row_length"])
+    lengths = np.full(m, 32, np.int64)
+    lengths[:19] = mx
+    assert lengths.sum() == nnz
+    w = W.random_csr(m, m, 1, lengths, seed=3)
+    _, f = _features_of(w, 4)
+    assert f.rep_bytes[0] == int(g["csr_bytes_fp32_int32"])
+    assert round(f.ell_slots / nnz, 1) == g["rho_ell_approx"]
+    assert f.rep_bytes[1] == 8 * m * mx
+    # hand case: 6 x 8, entries (0,0) (0,5) (3,4) (5,7): b = 4 -> blocks (0,0) (0,1) (1,1); b = 8 and 16 -> one block
+    rowptr = np.array([0, 2, 2, 2, 3, 3, 4], np.int32)
+    colind = np.array([0, 5, 4, 7], np.int32)
+    info = oracle.summary(rowptr, colind, 6, 8, 1)
+    f = oracle.features(rowptr, colind, 6, 8, info, 2)
+    assert list(f.nnzb) == [3, 1, 1]
+    assert f.rep_bytes[5] == (2 * 16 + 4) * 3 + 4 * 3      # BSR-4: two block-rows
+    assert f.rep_bytes[6] == (2 * 64 + 4) * 1 + 4 * 2
+    assert f.rep_bytes[7] == (2 * 256 + 4) * 1 + 4 * 2
+    assert f.ell_slots == 12 and list(f.sell_slots) == [12, 12, 12]
+    assert f.rep_bytes[2] == 6 * 12 + 4 * 2                # SELL-16: one slice, two offsets
+    assert f.rep_bytes[0] == 6 * 4 + 4 * 7
+
+
+def test_o5_shape_class_on_designed_distributions():
+    cls = lambda w: oracle.SHAPE_NAMES[oracle.shape_class(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N))]
+    assert cls(W.g2_stencil(n=64, N=1)) == "uniform"
+    assert cls(W.g1_tiny_uniform()) == "moderate"                                   # Poisson(8): CV^2 = 1/8
+    assert cls(W.g5_skewed(M=1 << 14, N=1, scale_c=2.4e7 / 256, cap=800)) == "power-law"
+    rng = np.random.default_rng(9)
+    two = np.where(rng.random(4000) < 0.5, 2, 64)                                   # two populations, 32x apart
+    assert cls(W.random_csr(4000, 5000, 1, two, seed=1)) == "bimodal"
+    geo = np.minimum(rng.geometric(1 / 9.0, 4000) - 1, 4000)                        # CV^2 = 1 / (1 - p) > 1, no heavy tail
+    assert cls(W.random_csr(4000, 5000, 1, geo, seed=2)) == "skewed"
