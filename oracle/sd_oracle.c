@@ -394,14 +394,19 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
 
 /* Family rule on O3's integers (thresholds are this build's reading; the
  * paper gives none).  parity unpinned.
- *   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N)
+ *   BSR-TC    rows strictly ascending, N a whole number of 128-byte column groups (a
+ *             multiple of 32 for fp32, of 64 for bf16: the widths the tensor-core kernel
+ *             serves), and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N)
  *             (Eq. 4; Sec. 3.1: dense tiles pay "when useful arithmetic outweighs
  *             compaction and fill-in costs").  rho_max is where the block form stops
  *             paying on the target GPU, by dense width and value type:
  *                        N < 128   128 <= N < 256   N >= 256
  *               fp32       3/2          2              11/4
  *               bf16       3            5              7
- *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4
+ *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4, or a narrow
+ *             dense operand with long rows: N <= 4 and nnz >= 32 M (Sec. 3.1 lists the
+ *             nonzero-parallel COO form for SpMV-like widths; it pays once rows are longer
+ *             than a thread-per-row kernel can stream)
  *   ROWSPLIT  otherwise
  * CV^2 = M sum r^2 / nnz^2 - 1 >= 4  <=>  M sum r^2 >= 5 nnz^2. */
 int sdo_decide(const sdo_info_t *o, int dtype)
@@ -418,12 +423,15 @@ int sdo_decide(const sdo_info_t *o, int dtype)
         num = 11;
         den = 4;
     }
-    if (o->nnz > 0 && o->unsorted_rows == 0 && den * 256 * o->nnzb16 <= num * o->nnz)
+    int64_t group = dtype == SDO_BF16 ? 64 : 32;
+    if (o->N >= group && o->N % group == 0 && o->nnz > 0 && o->unsorted_rows == 0 &&
+        den * 256 * o->nnzb16 <= num * o->nnz)
         return SDO_BSR_TC;
     unsigned __int128 lhs = (unsigned __int128)(uint64_t)o->M * o->sum_r2;
     unsigned __int128 rhs = (unsigned __int128)5 * (uint64_t)o->nnz * (uint64_t)o->nnz;
     int skew = (o->max_r >= 256 && 10 * o->nnz_long_rows >= o->nnz) || (o->nnz > 0 && lhs >= rhs);
-    return skew ? SDO_MERGE : SDO_ROWSPLIT;
+    int narrow_long = o->N >= 1 && o->N <= 4 && o->nnz >= 32 * o->M;
+    return (skew || narrow_long) ? SDO_MERGE : SDO_ROWSPLIT;
 }
 
 /* Merge-path coordinates by the sequential definition.  The merged list

@@ -479,8 +479,10 @@ struct TempBuf {   // frees temporary device memory on every exit path
 
 // Family rule on the integer summary.  The paper ranks templates with a learned model and a
 // measured search (Sec. 3.2-3.3) and prints no thresholds; these are fixed integer rules:
-//   BSR-TC    rows strictly ascending and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N) (Eq. 4)
-//   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4
+//   BSR-TC    rows strictly ascending, N a multiple of 32 (fp32) / 64 (bf16) columns, and
+//             rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N) (Eq. 4)
+//   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4,
+//             or N <= 4 and a mean row length of at least 32
 //   ROWSPLIT  otherwise
 // rho_max is where the block form stops paying on this GPU (Sec. 3.1: dense tiles pay "when
 // useful arithmetic outweighs compaction and fill-in costs").  The tensor-core kernel's time
@@ -502,12 +504,20 @@ static int decide_family(const sd_plan_info_t &s, int dtype) {
         num = 11;
         den = 4;
     }
-    if (s.nnz > 0 && s.unsorted_rows == 0 && den * 256 * s.nnzb16 <= num * s.nnz) return SD_BSR_TC;
+    // the tensor-core kernel serves dense widths that are whole 128-byte groups of columns; at any other
+    // width the block form would run its SIMT kernel, which is slower than the CSR kernels at every width
+    const int64_t group = dtype == SD_BF16 ? 64 : 32;
+    const bool tc_width = s.N >= group && s.N % group == 0;
+    if (tc_width && s.nnz > 0 && s.unsorted_rows == 0 && den * 256 * s.nnzb16 <= num * s.nnz) return SD_BSR_TC;
     const unsigned __int128 lhs = static_cast<unsigned __int128>(static_cast<uint64_t>(s.M)) * s.sum_r2;
     const unsigned __int128 rhs =
         static_cast<unsigned __int128>(5) * static_cast<uint64_t>(s.nnz) * static_cast<uint64_t>(s.nnz);
     const bool skew = (s.max_r >= 256 && 10 * s.nnz_long_rows >= s.nnz) || (s.nnz > 0 && lhs >= rhs);
-    return skew ? SD_MERGE : SD_ROWSPLIT;
+    // up to four columns a lane group per row has nothing to share: the row-split kernel works one thread
+    // (or a few) per row, which pays only while rows are short; from a mean of 32 nonzeros per row the
+    // nonzero-parallel segmented reduction of the merge family is faster (measured cross-over: 24..32)
+    const bool narrow_long = s.N >= 1 && s.N <= 4 && s.nnz >= 32 * s.M;
+    return (skew || narrow_long) ? SD_MERGE : SD_ROWSPLIT;
 }
 
 // Number of column windows: none unless the rows are short on average (nnz < 16 M, so the

@@ -258,6 +258,8 @@ def test_block_workload_strip_gemm_and_bsr(dtype):
     info = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
     assert info.nnzb16 == 60 and oracle.rho_bsr16(info) == 1.0
     assert info.blk_hist[8] == 60 and info.nnz_dense_blocks == w.nnz
+    assert oracle.decide(info) != oracle.BSR_TC     # 8 columns: not a width of the tensor-core kernel
+    info.N = 64
     assert oracle.decide(info) == oracle.BSR_TC
 
 
@@ -407,7 +409,7 @@ def test_o4_block_rule_thresholds_by_width_and_value_type():
     # the block form is taken while 256 * nnzb <= rho_max * nnz; rho_max by dense width and value type
     # (integer arithmetic: the boundary itself is inside)
     table = {(oracle.F32, 64): (3, 2), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (11, 4), (oracle.F32, 1024): (11, 4),
-             (oracle.BF16, 64): (3, 1), (oracle.BF16, 128): (5, 1), (oracle.BF16, 255): (5, 1), (oracle.BF16, 256): (7, 1)}
+             (oracle.BF16, 64): (3, 1), (oracle.BF16, 128): (5, 1), (oracle.BF16, 192): (5, 1), (oracle.BF16, 256): (7, 1)}
     w = W.g4_block(Mb=16, Kb=16, N=4, nblocks=30)
     base = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
     for (dt, N), (num, den) in table.items():
@@ -419,6 +421,22 @@ def test_o4_block_rule_thresholds_by_width_and_value_type():
             info.sum_r2 = 0          # keep the row-length part of the rule out of the picture
             info.max_r = 1
             assert (oracle.decide(info, dt) == oracle.BSR_TC) == want, (dt, N, nnz)
+    # widths that are not whole 128-byte column groups never take the block form, however dense the blocks
+    for dt, N in ((oracle.F32, 1), (oracle.F32, 4), (oracle.F32, 16), (oracle.F32, 48), (oracle.F32, 100),
+                  (oracle.BF16, 32), (oracle.BF16, 96), (oracle.BF16, 255)):
+        info = oracle.Info.from_buffer_copy(base)
+        info.N = N
+        assert info.nnz == 256 * info.nnzb16 and oracle.decide(info, dt) != oracle.BSR_TC, (dt, N)
+
+
+def test_o4_narrow_operands_take_the_nonzero_parallel_form_from_32_per_row():
+    for L, N, want in ((31, 1, oracle.ROWSPLIT), (32, 1, oracle.MERGE), (32, 4, oracle.MERGE), (32, 5, oracle.ROWSPLIT),
+                       (200, 8, oracle.ROWSPLIT), (8, 2, oracle.ROWSPLIT)):
+        M = 64
+        rowptr = np.arange(0, M * L + 1, L, dtype=np.int32)
+        colind = np.tile(np.arange(L, dtype=np.int32) * 3, M)    # uniform rows: no skew, blocks sparse
+        info = oracle.summary(rowptr, colind, M, 3 * L + 8, N)
+        assert oracle.decide(info) == want, (L, N)
 
 
 def test_o4_family_rule_on_the_five_shapes():
@@ -428,7 +446,7 @@ def test_o4_family_rule_on_the_five_shapes():
     assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.ROWSPLIT
     w = W.g3_gcn_rmat(scale=12, N=4)
     assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.MERGE
-    w = W.g4_block(Mb=32, Kb=32, N=4, nblocks=40)
+    w = W.g4_block(Mb=32, Kb=32, N=64, nblocks=40)
     assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.BSR_TC
     w = W.g5_skewed(M=1 << 14, N=4, scale_c=2.4e7 / 256, cap=800)
     assert oracle.decide(oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)) == oracle.MERGE
