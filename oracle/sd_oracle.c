@@ -403,10 +403,7 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
  *                        N < 128   128 <= N < 256   N >= 256
  *               fp32       3/2          2              11/4
  *               bf16       3            5              7
- *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4, or a narrow
- *             dense operand with long rows: N <= 4 and nnz >= 32 M (Sec. 3.1 lists the
- *             nonzero-parallel COO form for SpMV-like widths; it pays once rows are longer
- *             than a thread-per-row kernel can stream)
+ *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4
  *   ROWSPLIT  otherwise
  * CV^2 = M sum r^2 / nnz^2 - 1 >= 4  <=>  M sum r^2 >= 5 nnz^2. */
 int sdo_decide(const sdo_info_t *o, int dtype)
@@ -430,8 +427,7 @@ int sdo_decide(const sdo_info_t *o, int dtype)
     unsigned __int128 lhs = (unsigned __int128)(uint64_t)o->M * o->sum_r2;
     unsigned __int128 rhs = (unsigned __int128)5 * (uint64_t)o->nnz * (uint64_t)o->nnz;
     int skew = (o->max_r >= 256 && 10 * o->nnz_long_rows >= o->nnz) || (o->nnz > 0 && lhs >= rhs);
-    int narrow_long = o->N >= 1 && o->N <= 4 && o->nnz >= 32 * o->M;
-    return (skew || narrow_long) ? SDO_MERGE : SDO_ROWSPLIT;
+    return skew ? SDO_MERGE : SDO_ROWSPLIT;
 }
 
 /* Merge-path coordinates by the sequential definition.  The merged list

@@ -481,8 +481,7 @@ struct TempBuf {   // frees temporary device memory on every exit path
 // measured search (Sec. 3.2-3.3) and prints no thresholds; these are fixed integer rules:
 //   BSR-TC    rows strictly ascending, N a multiple of 32 (fp32) / 64 (bf16) columns, and
 //             rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N) (Eq. 4)
-//   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4,
-//             or N <= 4 and a mean row length of at least 32
+//   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4
 //   ROWSPLIT  otherwise
 // rho_max is where the block form stops paying on this GPU (Sec. 3.1: dense tiles pay "when
 // useful arithmetic outweighs compaction and fill-in costs").  The tensor-core kernel's time
@@ -513,11 +512,7 @@ static int decide_family(const sd_plan_info_t &s, int dtype) {
     const unsigned __int128 rhs =
         static_cast<unsigned __int128>(5) * static_cast<uint64_t>(s.nnz) * static_cast<uint64_t>(s.nnz);
     const bool skew = (s.max_r >= 256 && 10 * s.nnz_long_rows >= s.nnz) || (s.nnz > 0 && lhs >= rhs);
-    // up to four columns a lane group per row has nothing to share: the row-split kernel works one thread
-    // (or a few) per row, which pays only while rows are short; from a mean of 32 nonzeros per row the
-    // nonzero-parallel segmented reduction of the merge family is faster (measured cross-over: 24..32)
-    const bool narrow_long = s.N >= 1 && s.N <= 4 && s.nnz >= 32 * s.M;
-    return (skew || narrow_long) ? SD_MERGE : SD_ROWSPLIT;
+    return skew ? SD_MERGE : SD_ROWSPLIT;
 }
 
 // Number of column windows: none unless the rows are short on average (nnz < 16 M, so the
@@ -1351,6 +1346,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     a.ldb_bytes = static_cast<uint32_t>(ldb * (plan->dtype == SD_F32 ? 4 : 2));
     a.S = M;
     a.max_len = plan->info.max_r;
+    a.mean_len = M > 0 ? (plan->nnz + M - 1) / M : 0;
     a.N = static_cast<int32_t>(N);
     a.alpha = alpha;
     a.beta = beta;

@@ -151,6 +151,7 @@ struct SpmmArgs {
     int32_t N;
     float alpha, beta;
     int64_t max_len;        // longest row / segment if known (0: unknown); lets the row-split kernel drop its second accumulator
+    int64_t mean_len;       // mean row length rounded up if known (0: unknown): lanes per row of the narrow row-split kernel
 };
 
 inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }

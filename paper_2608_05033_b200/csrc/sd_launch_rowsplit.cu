@@ -1,10 +1,15 @@
 #include "sd_launch.cuh"
 #include "sd_rowsplit.cuh"
+#include "sd_rowsplit_narrow.cuh"
 #include "sd_segment.cuh"
 
 namespace sd {
 
 cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
+    if (a.N >= 1 && a.N <= 4 && !getenv("SD_NO_NARROW")) {   // one to four columns: lanes share a row, not its columns
+        if (dtype == SD_F32) return launch_rowsplit_narrow<float>(a, vec, st);
+        return launch_rowsplit_narrow<__nv_bfloat16>(a, vec, st);
+    }
     if (dtype == SD_F32) return launch_rowsplit<float>(a, vec, st);
     return launch_rowsplit<__nv_bfloat16>(a, vec, st);
 }

@@ -153,6 +153,7 @@ sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, c
     a.alpha = alpha;
     a.beta = beta;
     a.max_len = 0;
+    a.mean_len = 0;
     MergeArgs m;
     m.s = a;
     m.tile_seg = reinterpret_cast<int32_t *>(p);

@@ -319,6 +319,35 @@ def test_plan_reuse_with_second_dense_operand_and_host_entry():
     plan.close()
 
 
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+@pytest.mark.parametrize("N", [1, 2, 3, 4])
+@pytest.mark.parametrize("mean", [3, 9, 20, 40, 70, 300])
+def test_rowsplit_narrow_widths_every_lane_group(mean, N, dtype):
+    """Row-split family at one to four columns: 1, 2, 4, 8 or 16 lanes share a row according to the mean
+    row length; empty rows, rows far longer than the mean (the two-level sum), ragged row count, padded and
+    misaligned operands."""
+    rng = np.random.default_rng(mean * 10 + N)
+    M, K = 1031, 2500
+    lengths = np.clip(rng.poisson(mean, M), 0, K)
+    lengths[::17] = 0
+    lengths[5] = K            # one row holds every column
+    lengths[M - 1] = 1
+    w = W.random_csr(M, K, N, lengths, seed=mean + N, dtype=dtype, alpha=-0.75, beta=0.5)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_ROWSPLIT)
+    for kw in (dict(), dict(pad_b=3, pad_c=5), dict(offset=1), dict(offset=2, pad_b=1)):
+        got, intact = run_spmm(plan, w, **kw)
+        assert intact
+        check(w, got)
+    got2, _ = run_spmm(plan, w)
+    got3, _ = run_spmm(plan, w)
+    assert np.array_equal(got2, got3)
+    poison = np.full((M, N), np.nan, np.float32)
+    got4, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got4, beta=0.0)
+    plan.close()
+
+
 @pytest.mark.parametrize("N", [8, 32, 128])
 def test_symmetric_adjacency_forward_plan_serves_the_backward_product(N):
     """Sec. 5, GCN evaluation: the backward aggregation is a product with the transposed adjacency;

@@ -429,14 +429,13 @@ def test_o4_block_rule_thresholds_by_width_and_value_type():
         assert info.nnz == 256 * info.nnzb16 and oracle.decide(info, dt) != oracle.BSR_TC, (dt, N)
 
 
-def test_o4_narrow_operands_take_the_nonzero_parallel_form_from_32_per_row():
-    for L, N, want in ((31, 1, oracle.ROWSPLIT), (32, 1, oracle.MERGE), (32, 4, oracle.MERGE), (32, 5, oracle.ROWSPLIT),
-                       (200, 8, oracle.ROWSPLIT), (8, 2, oracle.ROWSPLIT)):
+def test_o4_uniform_rows_stay_row_split_at_every_width_and_length():
+    for L, N in ((5, 1), (31, 1), (32, 1), (32, 4), (200, 1), (200, 8), (8, 2)):
         M = 64
         rowptr = np.arange(0, M * L + 1, L, dtype=np.int32)
         colind = np.tile(np.arange(L, dtype=np.int32) * 3, M)    # uniform rows: no skew, blocks sparse
         info = oracle.summary(rowptr, colind, M, 3 * L + 8, N)
-        assert oracle.decide(info) == want, (L, N)
+        assert oracle.decide(info) == oracle.ROWSPLIT, (L, N)
 
 
 def test_o4_family_rule_on_the_five_shapes():
