@@ -54,3 +54,79 @@ def test_single_process_reductions_are_identity():
     import bench
     assert bench.max_over_ranks(1.5) == 1.5 and bench.sum_over_ranks(2.5) == 2.5
     bench.barrier()
+
+
+# ---- splitting one product over ranks without a collective (host arithmetic + oracle, CPU only) ----
+def test_column_shards_partition_the_width():
+    sys.path.insert(0, ROOT)
+    from paper_2608_05033_b200.shard import column_shard
+    for N, world, align in ((256, 8, 4), (100, 3, 4), (7, 4, 1), (3, 8, 4), (0, 2, 4), (128, 1, 8)):
+        got = [column_shard(N, world, r, align) for r in range(world)]
+        assert got[0][0] == 0 and sum(n for _, n in got) == N
+        for (c0, n), (c1, _) in zip(got, got[1:]):
+            assert c0 + n == c1
+        assert all(c0 % align == 0 for c0, n in got if n)
+        sizes = [(-(-n // align)) for _, n in got]
+        assert max(sizes) - min(sizes) <= 1
+
+
+def test_row_shards_balance_rows_plus_nonzeros():
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import workloads as W
+    from paper_2608_05033_b200.shard import row_shard_bounds
+    w = W.g5_skewed(M=1 << 13, N=4, scale_c=2.4e7 / 512, cap=2000)
+    for world in (1, 2, 3, 8):
+        b = row_shard_bounds(w.rowptr, world)
+        assert b[0] == 0 and b[-1] == w.M and np.all(np.diff(b) >= 0)
+        work = np.array([(b[k + 1] - b[k]) + (w.rowptr[b[k + 1]] - w.rowptr[b[k]]) for k in range(world)])
+        ideal = (w.M + w.nnz) / world
+        longest = int(np.diff(w.rowptr).max()) + 1
+        assert np.all(np.abs(work - ideal) <= longest + 1)      # off by at most one row's weight
+    assert list(row_shard_bounds(np.zeros(6, np.int32), 5)) == [0, 1, 2, 3, 4, 5]
+
+
+def _shard_worker(rank, world, port, out):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import oracle
+    import workloads as W
+    from paper_2608_05033_b200.shard import column_shard, row_shard_bounds, row_shard_csr
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    w = W.g3_gcn_rmat(scale=10, N=12)
+    # rows: this rank's range with rebased pointers, all of B
+    b = row_shard_bounds(w.rowptr, world)
+    r0, r1 = int(b[rank]), int(b[rank + 1])
+    rp, cj, v = row_shard_csr(w.rowptr, w.colind, w.vals, r0, r1)
+    mine, _ = oracle.spmm(rp, cj, v, w.B, w.N)
+    rows_full = torch.zeros((w.M, w.N), dtype=torch.float64)
+    rows_full[r0:r1] = torch.from_numpy(mine)
+    dist.all_reduce(rows_full)                      # test-side assembly only: disjoint rows, zeros elsewhere
+    # columns: all of A, this rank's columns of B
+    c0, n = column_shard(w.N, world, rank, 4)
+    cols_full = torch.zeros((w.M, w.N), dtype=torch.float64)
+    if n:
+        part, _ = oracle.spmm(w.rowptr, w.colind, w.vals, np.ascontiguousarray(w.B[:, c0:c0 + n]), n)
+        cols_full[:, c0:c0 + n] = torch.from_numpy(part)
+    dist.all_reduce(cols_full)
+    if rank == 0:
+        ref, _ = oracle.spmm(w.rowptr, w.colind, w.vals, w.B, w.N)
+        out.put((bool(np.array_equal(rows_full.numpy(), ref)), bool(np.array_equal(cols_full.numpy(), ref))))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_row_and_column_shards_reassemble_the_product():
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = out.get(timeout=180)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == (True, True)

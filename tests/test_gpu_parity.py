@@ -348,6 +348,39 @@ def test_rowsplit_narrow_widths_every_lane_group(mean, N, dtype):
     plan.close()
 
 
+@pytest.mark.parametrize("world", [2, 3])
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_row_and_column_shards_of_one_product(world, dtype):
+    """The two collective-free splits of one product, every rank's share run in turn on this GPU
+    (the shares do not wait on one another): row ranges with rebased pointers and all of B; column
+    ranges through offset base pointers with the full leading dimensions."""
+    from paper_2608_05033_b200.shard import column_shard, row_shard_bounds, row_shard_csr
+    from util import dev
+    w = W.config(2, scale=12, N=96, dtype=dtype)
+    Bd = dev(w.B)
+    # rows
+    Cd = torch.full((w.M, w.N), float("nan"), device="cuda")
+    b = row_shard_bounds(w.rowptr, world)
+    for rank in range(world):
+        r0, r1 = int(b[rank]), int(b[rank + 1])
+        rp, cj, v = row_shard_csr(w.rowptr, w.colind, w.vals, r0, r1)
+        plan = sd.Plan(dev(rp), dev(cj), dev(v), r1 - r0, w.K, w.N, dtype=dtype)
+        plan.spmm(Bd, Cd[r0:r1], 1.0, 0.0)
+        torch.cuda.synchronize()
+        plan.close()
+    check(w, Cd.cpu().numpy())
+    # columns
+    Cd = torch.full((w.M, w.N), float("nan"), device="cuda")
+    dw = DeviceWorkload(w)
+    for rank in range(world):
+        c0, n = column_shard(w.N, world, rank, 8)
+        plan = dw.plan(N=n)
+        plan.spmm(Bd[:, c0:c0 + n], Cd[:, c0:c0 + n], 1.0, 0.0)
+        torch.cuda.synchronize()
+        plan.close()
+    check(w, Cd.cpu().numpy())
+
+
 @pytest.mark.parametrize("N", [8, 32, 128])
 def test_symmetric_adjacency_forward_plan_serves_the_backward_product(N):
     """Sec. 5, GCN evaluation: the backward aggregation is a product with the transposed adjacency;
