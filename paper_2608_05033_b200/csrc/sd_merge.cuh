@@ -35,7 +35,14 @@ merge_tile_kernel(const MergeArgs m) {
     constexpr int COLS = LPR * CPL;          // columns per CTA slab
     constexpr int CP = COLS + 1;             // padded row pitch of head_s / tail_s
 
-    __shared__ int2 nz_s[TILE];               // (column, value bits) of the tile's nonzeros
+    // (column, value bits) of the tile's nonzeros.  Eight or more groups share a warp when LPR <= 4 and read
+    // their own nonzeros in lock step, IPG items apart: one pad slot per IPG items moves neighbouring
+    // groups to different banks.
+    constexpr bool SKEW = LPR <= 4;   // measured: -7 to -9 % at 8 and 16 columns; with 8 or 16 lanes per row the extra index arithmetic costs more than the conflicts
+    constexpr int IPG_SHIFT = (IPG == 4) ? 2 : (IPG == 8) ? 3 : (IPG == 16) ? 4 : (IPG == 32) ? 5 : (IPG == 64) ? 6 : 7;
+    static_assert((1 << IPG_SHIFT) == IPG, "items per group must be a power of two");
+    auto phys = [](int k) { return SKEW ? k + (k >> IPG_SHIFT) : k; };
+    __shared__ int2 nz_s[TILE + (SKEW ? G : 0)];
     __shared__ int32_t ptr_s[TILE + 2];       // ptr[seg0 .. seg0 + ends + 1]
     __shared__ float head_s[G * CP];
     __shared__ float tail_s[G * CP];
@@ -69,7 +76,7 @@ merge_tile_kernel(const MergeArgs m) {
     for (int i = tid; i <= ends + 1; i += kMergeThreads)
         ptr_s[i] = __ldg(a.ptr + min(seg0 + i, m.seg_end));
     for (int k = tid; k < nnz_t; k += kMergeThreads)
-        nz_s[k] = make_int2(__ldcs(a.colind + nz0 + k), __float_as_int(to_float(__ldcs(vals + nz0 + k))));   // A streams through
+        nz_s[phys(k)] = make_int2(__ldcs(a.colind + nz0 + k), __float_as_int(to_float(__ldcs(vals + nz0 + k))));   // A streams through
     if (tid == 0) first_end_s = G;
     __syncthreads();
 
@@ -115,7 +122,7 @@ merge_tile_kernel(const MergeArgs m) {
         for (; j + WB <= jend; j += WB) {
             int2 it[WB];
 #pragma unroll
-            for (int u = 0; u < WB; ++u) it[u] = nz_s[j + u];
+            for (int u = 0; u < WB; ++u) it[u] = nz_s[phys(j + u)];
             float b[WB][NV][VW];
 #pragma unroll
             for (int u = 0; u < WB; ++u) {
@@ -138,7 +145,7 @@ merge_tile_kernel(const MergeArgs m) {
                     for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(__int_as_float(it[u].y), b[u][v][e], acc[v][e]);
         }
         for (; j < jend; ++j) {
-            const int2 it = nz_s[j];
+            const int2 it = nz_s[phys(j)];
             const float av = __int_as_float(it.y);
             const T *brow = b_row(Bl, it.x, a.ldb_bytes);
 #pragma unroll
