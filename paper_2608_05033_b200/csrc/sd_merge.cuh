@@ -219,17 +219,16 @@ merge_tile_kernel(const MergeArgs m) {
             for (int ch = 0; ch < G; ch += 32) {
                 const int gg = ch + lane;
                 float v = tail_s[gg * CP + c];
-                int f = has_end_s[gg];
+                // the groups that saw a segment end restart the sum: one ballot gives every lane the
+                // start of its run, so only the values travel through the shuffles
+                const unsigned restarts = __ballot_sync(FULLMASK, has_end_s[gg] != 0) & (FULLMASK >> (31 - lane));
+                const int reach = restarts ? lane - (31 - __clz(restarts)) : lane;   // lanes below that belong to this lane's run
 #pragma unroll
                 for (int off = 1; off < 32; off <<= 1) {
                     const float v2 = __shfl_up_sync(FULLMASK, v, off);
-                    const int f2 = __shfl_up_sync(FULLMASK, f, off);
-                    if (lane >= off && !f) {
-                        v += v2;
-                        f = f2;
-                    }
+                    if (off <= reach) v += v2;
                 }
-                if (!f) v += run;
+                if (!restarts) v += run;
                 float ex = __shfl_up_sync(FULLMASK, v, 1);
                 if (lane == 0) ex = run;
                 run = __shfl_sync(FULLMASK, v, 31);
