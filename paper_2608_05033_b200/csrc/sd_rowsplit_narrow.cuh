@@ -36,7 +36,34 @@ rowsplit_narrow_kernel(const SpmmArgs a) {
     }
     int p = p0 + g;
     [[maybe_unused]] int folded = 0;
-    // two nonzeros per step: both index loads, then both gathers, in flight together
+    // four nonzeros per step while the row lasts: the index loads first, then the gathers, all in flight together
+    for (; p + 3 * G < p1; p += 4 * G) {
+        int c[4];
+        float v[4], b[4][N];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            c[u] = __ldg(a.colind + p + u * G);
+            v[u] = to_float(vals[p + u * G]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) coo_gather<T, N, VEC>(a.B, c[u], a.ldb_bytes, b[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int e = 0; e < N; ++e) acc[e] = fmaf(v[u], b[u][e], acc[e]);
+        if constexpr (LONG) {
+            folded += 2;
+            if (folded >= kNarrowFold / 2) {
+                folded = 0;
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    tot[e] += acc[e];
+                    acc[e] = 0.f;
+                }
+            }
+        }
+    }
+    // then two per step
     for (; p + G < p1; p += 2 * G) {
         const int c0 = __ldg(a.colind + p), c1 = __ldg(a.colind + p + G);
         const float v0 = to_float(vals[p]), v1 = to_float(vals[p + G]);
