@@ -394,9 +394,10 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
 
 /* Family rule on O3's integers (thresholds are this build's reading; the
  * paper gives none).  parity unpinned.
- *   BSR-TC    rows strictly ascending, N a whole number of 128-byte column groups (a
- *             multiple of 32 for fp32, of 64 for bf16: the widths the tensor-core kernel
- *             serves), and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N)
+ *   BSR-TC    rows strictly ascending, N at least 64 and a whole number of 128-byte column
+ *             groups (a multiple of 32 for fp32, of 64 for bf16: the widths the tensor-core
+ *             kernel serves; at 32 fp32 columns the CSR kernels are ahead even on full
+ *             blocks), and rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N)
  *             (Eq. 4; Sec. 3.1: dense tiles pay "when useful arithmetic outweighs
  *             compaction and fill-in costs").  rho_max is where the block form stops
  *             paying on the target GPU, by dense width and value type:
@@ -421,7 +422,7 @@ int sdo_decide(const sdo_info_t *o, int dtype)
         den = 4;
     }
     int64_t group = dtype == SDO_BF16 ? 64 : 32;
-    if (o->N >= group && o->N % group == 0 && o->nnz > 0 && o->unsorted_rows == 0 &&
+    if (o->N >= 64 && o->N % group == 0 && o->nnz > 0 && o->unsorted_rows == 0 &&
         den * 256 * o->nnzb16 <= num * o->nnz)
         return SDO_BSR_TC;
     unsigned __int128 lhs = (unsigned __int128)(uint64_t)o->M * o->sum_r2;

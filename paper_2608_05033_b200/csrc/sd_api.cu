@@ -479,7 +479,7 @@ struct TempBuf {   // frees temporary device memory on every exit path
 
 // Family rule on the integer summary.  The paper ranks templates with a learned model and a
 // measured search (Sec. 3.2-3.3) and prints no thresholds; these are fixed integer rules:
-//   BSR-TC    rows strictly ascending, N a multiple of 32 (fp32) / 64 (bf16) columns, and
+//   BSR-TC    rows strictly ascending, N >= 64 and a multiple of 32 (fp32) / 64 (bf16) columns, and
 //             rho_BSR(16) = 256 nnzb / nnz <= rho_max(dtype, N) (Eq. 4)
 //   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV(r)^2 >= 4
 //   ROWSPLIT  otherwise
@@ -506,7 +506,7 @@ static int decide_family(const sd_plan_info_t &s, int dtype) {
     // the tensor-core kernel serves dense widths that are whole 128-byte groups of columns; at any other
     // width the block form would run its SIMT kernel, which is slower than the CSR kernels at every width
     const int64_t group = dtype == SD_BF16 ? 64 : 32;
-    const bool tc_width = s.N >= group && s.N % group == 0;
+    const bool tc_width = s.N >= 64 && s.N % group == 0;   // 32 fp32 columns: the row-split kernel is ahead even on full blocks
     if (tc_width && s.nnz > 0 && s.unsorted_rows == 0 && den * 256 * s.nnzb16 <= num * s.nnz) return SD_BSR_TC;
     const unsigned __int128 lhs = static_cast<unsigned __int128>(static_cast<uint64_t>(s.M)) * s.sum_r2;
     const unsigned __int128 rhs =

@@ -118,6 +118,123 @@ rowsplit_narrow_kernel(const SpmmArgs a) {
     }
 }
 
+// The same scheme at 8 to 32 columns (one 16-byte vector per lane, LPR = 2..8 lanes across the columns):
+// G such lane sets share a row, set k takes the nonzeros p0 + k, p0 + k + G, ...; the G partial rows meet by
+// xor shuffles over the set index.  Pays when rows are long enough to keep G sets busy (the paper's
+// af_shell10 case: a few threads per row, each holding several outputs); short rows keep the plain kernel.
+template <typename T, int VW, int LPR, int G, bool LONG>
+__global__ void __launch_bounds__(kNarrowThreads)
+rowsplit_ksplit_kernel(const SpmmArgs a) {
+    constexpr unsigned FULL = 0xffffffffu;
+    constexpr int LANES = LPR * G;                 // lanes per row
+    const int lc = threadIdx.x % LPR;              // column vector of this lane
+    const int gk = (threadIdx.x / LPR) % G;        // which share of the row's nonzeros
+    const int64_t row = (static_cast<int64_t>(blockIdx.x) * kNarrowThreads + threadIdx.x) / LANES;
+    const T *__restrict__ vals = static_cast<const T *>(a.vals);
+    const T *__restrict__ Bl = static_cast<const T *>(a.B) + lc * VW;
+    int p0 = 0, p1 = 0;
+    if (row < a.S) {
+        p0 = __ldg(a.ptr + row);
+        p1 = __ldg(a.ptr + row + 1);
+    }
+    float acc[VW], tot[LONG ? VW : 1];
+#pragma unroll
+    for (int e = 0; e < VW; ++e) {
+        acc[e] = 0.f;
+        if constexpr (LONG) tot[e] = 0.f;
+    }
+    int p = p0 + gk;
+    [[maybe_unused]] int folded = 0;
+    for (; p + 3 * G < p1; p += 4 * G) {
+        int c[4];
+        float v[4], b[4][VW];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            c[u] = __ldg(a.colind + p + u * G);
+            v[u] = to_float(vals[p + u * G]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) RowLoad<T, VW>::ld(b_row(Bl, c[u], a.ldb_bytes), b[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int e = 0; e < VW; ++e) acc[e] = fmaf(v[u], b[u][e], acc[e]);
+        if constexpr (LONG) {
+            if (++folded == kNarrowFold / 4) {
+                folded = 0;
+#pragma unroll
+                for (int e = 0; e < VW; ++e) {
+                    tot[e] += acc[e];
+                    acc[e] = 0.f;
+                }
+            }
+        }
+    }
+    for (; p < p1; p += G) {
+        const int c0 = __ldg(a.colind + p);
+        const float v0 = to_float(vals[p]);
+        float b0[VW];
+        RowLoad<T, VW>::ld(b_row(Bl, c0, a.ldb_bytes), b0);
+#pragma unroll
+        for (int e = 0; e < VW; ++e) acc[e] = fmaf(v0, b0[e], acc[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < VW; ++e) {
+        if constexpr (LONG) acc[e] += tot[e];
+#pragma unroll
+        for (int d = LANES / 2; d >= LPR; d >>= 1) acc[e] += __shfl_xor_sync(FULL, acc[e], d);
+    }
+    if (gk == 0 && row < a.S) store_cols<VW>(a.C + row * a.ldc + lc * VW, acc, a.alpha, a.beta, 0);
+}
+
+inline int ksplit_override() {
+    static const int v = [] {
+        const char *e = getenv("SD_KSPLIT_G");   // measurement switch: lane sets per row (0: rule, 1: off)
+        return e ? atoi(e) : 0;
+    }();
+    return v;
+}
+
+// Lane sets per row for the kernel above: 1 (= use the plain row-split kernel) unless rows are long.
+// Swept on uniform rows of 16 to 131 nonzeros at 8, 16 and 32 columns: about one set per eight nonzeros of
+// the mean row, at most 16 lanes per row below a mean of 128 nonzeros and a whole warp from there.
+inline int ksplit_group(int64_t mean_len, int lpr) {
+    int g = 1;
+    const int lanes = mean_len >= 128 ? 32 : 16;
+    if (const int o = ksplit_override()) g = o;
+    else while (2 * g * lpr <= lanes && 2 * g <= mean_len / 8) g <<= 1;
+    while (g > 1 && g * lpr > 32) g >>= 1;
+    return g;
+}
+
+template <typename T, int VW, int LPR, int G>
+cudaError_t launch_ksplit_g(const SpmmArgs &a, cudaStream_t st) {
+    if constexpr (LPR * G > 32) {
+        return cudaErrorInvalidValue;
+    } else {
+        const int rows_per_cta = kNarrowThreads / (LPR * G);
+        const unsigned grid = static_cast<unsigned>((a.S + rows_per_cta - 1) / rows_per_cta);
+        const bool is_long = !(a.max_len > 0 && a.max_len <= static_cast<int64_t>(kNarrowFold) * G);
+        if (is_long) rowsplit_ksplit_kernel<T, VW, LPR, G, true><<<grid, kNarrowThreads, 0, st>>>(a);
+        else rowsplit_ksplit_kernel<T, VW, LPR, G, false><<<grid, kNarrowThreads, 0, st>>>(a);
+        return cudaGetLastError();
+    }
+}
+
+// N * sizeof(T) = 16 * LPR bytes exactly, LPR in {2, 4, 8}; g from ksplit_group (> 1).
+template <typename T>
+cudaError_t launch_rowsplit_ksplit(const SpmmArgs &a, int lpr, int g, cudaStream_t st) {
+    constexpr int VWV = vec_width<T>::value;
+#define SD_KS_CASE(L, GG) \
+    if (lpr == L && g == GG) return launch_ksplit_g<T, VWV, L, GG>(a, st);
+    SD_KS_CASE(1, 2) SD_KS_CASE(1, 4) SD_KS_CASE(1, 8) SD_KS_CASE(1, 16) SD_KS_CASE(1, 32)
+    SD_KS_CASE(2, 2) SD_KS_CASE(2, 4) SD_KS_CASE(2, 8) SD_KS_CASE(2, 16)
+    SD_KS_CASE(4, 2) SD_KS_CASE(4, 4) SD_KS_CASE(4, 8)
+    SD_KS_CASE(8, 2) SD_KS_CASE(8, 4)
+#undef SD_KS_CASE
+    return cudaErrorInvalidValue;
+}
+
 inline int narrow_group_override() {
     static const int v = [] {
         const char *e = getenv("SD_NARROW_G");   // measurement switch: lanes per row (1..32, power of two)

@@ -381,6 +381,36 @@ def test_row_and_column_shards_of_one_product(world, dtype):
     check(w, Cd.cpu().numpy())
 
 
+@pytest.mark.parametrize("dtype,N", [(W.SD_F32, 8), (W.SD_F32, 16), (W.SD_F32, 32), (W.SD_BF16, 8), (W.SD_BF16, 16),
+                                     (W.SD_BF16, 32), (W.SD_BF16, 64)])
+@pytest.mark.parametrize("mean", [20, 40, 70, 300])
+def test_rowsplit_long_rows_several_lane_sets_per_row(mean, N, dtype):
+    """Row-split family at 8 to 32 fp32 (8 to 64 bf16) columns with long rows: 2 to 16 lane sets share a
+    row and meet by shuffles; empty rows, one row far beyond the mean (two-level sum), ragged row count,
+    padded leading dimensions, and a misaligned call that must take the plain kernel."""
+    rng = np.random.default_rng(mean * 100 + N)
+    M, K = 517, 3000
+    lengths = np.clip(rng.poisson(mean, M), 0, K)
+    lengths[::13] = 0
+    lengths[7] = K
+    lengths[M - 1] = 1
+    w = W.random_csr(M, K, N, lengths, seed=mean + N, dtype=dtype, alpha=1.5, beta=-0.25)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_ROWSPLIT)
+    vw = 4 if dtype == W.SD_F32 else 8
+    for kw in (dict(), dict(pad_b=vw, pad_c=4), dict(offset=1)):
+        got, intact = run_spmm(plan, w, **kw)
+        assert intact
+        check(w, got)
+    got2, _ = run_spmm(plan, w)
+    got3, _ = run_spmm(plan, w)
+    assert np.array_equal(got2, got3)
+    poison = np.full((M, N), np.nan, np.float32)
+    got4, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got4, beta=0.0)
+    plan.close()
+
+
 @pytest.mark.parametrize("N", [8, 32, 128])
 def test_symmetric_adjacency_forward_plan_serves_the_backward_product(N):
     """Sec. 5, GCN evaluation: the backward aggregation is a product with the transposed adjacency;

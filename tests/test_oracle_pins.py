@@ -408,7 +408,7 @@ def test_o4_merge_coords_match_closed_form():
 def test_o4_block_rule_thresholds_by_width_and_value_type():
     # the block form is taken while 256 * nnzb <= rho_max * nnz; rho_max by dense width and value type
     # (integer arithmetic: the boundary itself is inside)
-    table = {(oracle.F32, 64): (3, 2), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (11, 4), (oracle.F32, 1024): (11, 4),
+    table = {(oracle.F32, 64): (3, 2), (oracle.F32, 96): (3, 2), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (11, 4), (oracle.F32, 1024): (11, 4),
              (oracle.BF16, 64): (3, 1), (oracle.BF16, 128): (5, 1), (oracle.BF16, 192): (5, 1), (oracle.BF16, 256): (7, 1)}
     w = W.g4_block(Mb=16, Kb=16, N=4, nblocks=30)
     base = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
@@ -422,7 +422,7 @@ def test_o4_block_rule_thresholds_by_width_and_value_type():
             info.max_r = 1
             assert (oracle.decide(info, dt) == oracle.BSR_TC) == want, (dt, N, nnz)
     # widths that are not whole 128-byte column groups never take the block form, however dense the blocks
-    for dt, N in ((oracle.F32, 1), (oracle.F32, 4), (oracle.F32, 16), (oracle.F32, 48), (oracle.F32, 100),
+    for dt, N in ((oracle.F32, 1), (oracle.F32, 4), (oracle.F32, 16), (oracle.F32, 32), (oracle.F32, 48), (oracle.F32, 100),
                   (oracle.BF16, 32), (oracle.BF16, 96), (oracle.BF16, 255)):
         info = oracle.Info.from_buffer_copy(base)
         info.N = N
