@@ -69,7 +69,8 @@ typedef struct {
     int64_t M, K, N;       /* N: dense width the plan is tuned for (other widths still run) */
     int32_t dtype;         /* sd_dtype_t */
     int32_t family;        /* sd_family_t; SD_AUTO applies the rule */
-    int32_t windows;       /* column windows of the MERGE family: 0 = automatic, 1 = off, 2..64 */
+    int32_t windows;       /* column windows of the MERGE family: 0 = automatic, 1 = off, 2..64;
+                              -1 = one window, but with the class split of the window-major schedule */
     int32_t validate;      /* != 0: check rowptr monotone and 0 <= col < K on the device first */
     void *stream;          /* stream for the analysis kernels (plan creation still synchronises) */
 } sd_plan_desc_t;
@@ -98,11 +99,15 @@ typedef struct {
     int32_t windows;        /* column windows in use (1 = none) */
     int32_t tile_items;     /* merge items (row ends + nonzeros) per CTA tile, MERGE only */
     int64_t num_tiles;      /* MERGE: total tiles over all windows */
-    int64_t num_segments;   /* MERGE: rows, or (row, window) pairs when windows > 1 */
+    int64_t num_segments;   /* MERGE: rows, or (row, window) pairs with the class split */
     int64_t plan_bytes;     /* device memory owned by the plan */
     int32_t sm_count;       /* hardware context read at plan time (Sec. 3.1) */
     int32_t launches;       /* kernel launches one sd_spmm call issues on the vectorised path */
     int64_t l2_bytes;
+    int32_t class_split;    /* MERGE: 1 when the segments run by class (long ones as chunks, short ones one
+                               lane group each, one-nonzero ones flat) instead of merge-path tiles: always
+                               with windows > 1, and with one window where that alone pays */
+    int32_t reserved0;
 } sd_plan_info_t;
 
 /* sd_plan_create -- Sec. 3 (task <X, o, H> in, specialised implementation out) and
@@ -205,12 +210,12 @@ typedef struct {
     int32_t value_bytes;   /* vb: 4 or 2 */
     /* the plan as built (Eq. 10-13) */
     int64_t borrowed_bytes; /* caller's CSR arrays that sd_spmm reads: all three for SD_ROWSPLIT and for
-                               SD_MERGE without windows, none otherwise */
+                               SD_MERGE without the class split, none otherwise */
     int64_t plan_bytes;     /* device memory owned by the plan: representation, tables, scratch */
     int64_t d_r, d_s;       /* dense B: K N vb;  dense C: 4 M N */
     int64_t m_r, m_t;       /* m_r = borrowed + plan + d_r;  m_t = m_r + d_s */
     int64_t work_units;     /* rows (SD_ROWSPLIT), tiles (SD_MERGE), (row, window) segments (SD_MERGE with
-                               windows), block-rows (SD_BSR_TC) */
+                               the class split), block-rows (SD_BSR_TC) */
     int32_t sm_count;
     int32_t reserved;
     int64_t l2_bytes;
@@ -251,7 +256,7 @@ sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t 
  *   colind   int32 [nnz], vals [nnz]   nonzeros in window-major order (plan dtype)
  *   win_seg  int64 [3*windows + 1]     per window: first segment of each of the three classes;
  *                                      last entry = num_segments
- * Any pointer may be NULL.  SD_ERR_UNSUPPORTED when the plan has no windows. */
+ * Any pointer may be NULL.  SD_ERR_UNSUPPORTED when the plan does not use the class split. */
 sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_t *seg_row, int32_t *colind,
                                  void *vals, int64_t *win_seg);
 

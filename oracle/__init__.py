@@ -199,6 +199,11 @@ def decide_windows(info: Info, dtype: int, l2_bytes: int) -> int:
     return int(lib().sdo_decide_windows(C.byref(info), C.c_int(dtype), C.c_int64(l2_bytes)))
 
 
+def decide_class_split(info: Info, dtype: int) -> bool:
+    """O4: class split of the window-major schedule at one window (parity unpinned: this build's rule)."""
+    return bool(lib().sdo_decide_class_split(C.byref(info), C.c_int(dtype)))
+
+
 def window_segments(rowptr, colind, M, K, W, short_len=32):
     """O4: window-major segment list ordered by (window, class, row).
     Returns (seg_ptr, seg_row, perm, bounds[3W+1])."""

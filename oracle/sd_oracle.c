@@ -474,6 +474,17 @@ int sdo_decide_windows(const sdo_info_t *o, int dtype, int64_t l2_bytes)
     return w;
 }
 
+/* Class split at one window (this build's rule, parity unpinned): the window-major schedule
+ * (long segments cut into chunks, short ones one lane group each, one-nonzero rows flat) without
+ * column windows, taken by merge-family plans whose rows are sorted when a row of B is exactly
+ * 64 or 128 bytes; measured on the target GPU against the merge-path tiles, which stay ahead at
+ * 32 bytes and from 256 bytes on. */
+int sdo_decide_class_split(const sdo_info_t *o, int dtype)
+{
+    int64_t row_bytes = o->N * (dtype == SDO_F32 ? 4 : 2);
+    return o->unsorted_rows == 0 && o->nnz > 0 && (row_bytes == 64 || row_bytes == 128);
+}
+
 /* Window-major segment list.  Window of a column: col / ceil(K / W).  A segment is the part
  * of one row inside one window.  First ordering: the empty rows (zero-length segments of
  * window 0), then for w = 0..W-1, for ascending row, the row's nonzeros of window w in storage

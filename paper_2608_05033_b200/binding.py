@@ -43,7 +43,7 @@ class sd_plan_info_t(C.Structure):
                 ("family", C.c_int32), ("dtype", C.c_int32), ("windows", C.c_int32),
                 ("tile_items", C.c_int32), ("num_tiles", C.c_int64), ("num_segments", C.c_int64),
                 ("plan_bytes", C.c_int64), ("sm_count", C.c_int32), ("launches", C.c_int32),
-                ("l2_bytes", C.c_int64)]
+                ("l2_bytes", C.c_int64), ("class_split", C.c_int32), ("reserved0", C.c_int32)]
 
     def as_dict(self) -> dict:
         d = {}

@@ -529,6 +529,15 @@ static int decide_windows(const sd_plan_info_t &s, int dtype) {
     return w;
 }
 
+// One window, but still the class split (long segments as chunks, short ones one lane group each,
+// one-nonzero rows flat) instead of merge-path tiles: measured on the R-MAT matrix, the split is ahead
+// where a row of B is 64 or 128 bytes (0.322 against 0.362 ms and 0.414 against 0.482 ms) and behind at
+// 32 bytes and from 256 bytes on.  Needs ascending columns like the windows.
+static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
+    const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
+    return s.unsorted_rows == 0 && s.nnz > 0 && (row_bytes == 64 || row_bytes == 128);
+}
+
 __global__ void iota_kernel(int32_t *out, int64_t n) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i < n) out[i] = static_cast<int32_t>(i);
@@ -699,10 +708,14 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     return SD_OK;
 }
 
-static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
+// `split`: the segments are re-bucketed by (window, class) and run through the chunk / segment / single
+// kernels; always so with W > 1, and with W = 1 when the class split alone pays (decide_class_split).
+static sd_status_t build_merge(sd_plan *p, int W, bool split, cudaStream_t st) {
     sd_status_t s;
     std::vector<int64_t> win_seg;   // per window: start of the long class, start of the short class
-    if (W > 1) {
+    if (W < 1) W = 1;
+    if (W > 1) split = true;
+    if (split) {
         if ((s = build_windows(p, W, win_seg, st))) return s;
         p->m_ptr = p->w_ptr;
         p->m_col = p->w_col;
@@ -735,7 +748,7 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
         win.single_nz = win_nz[3 * w + 2];
         win.chunk_begin = win.chunk_end = 0;
         int64_t total = (win.seg_end - win.seg_begin) + (win_nz[3 * w + 1] - win_nz[3 * w]);
-        if (W > 1) total = 0;   // with windows the long segments run as chunks, not as merge-path tiles
+        if (split) total = 0;   // with windows the long segments run as chunks, not as merge-path tiles
         win.ntiles = static_cast<int32_t>((total + kMergeTile - 1) / kMergeTile);
         win.tile_base = ntiles;
         win.nshort = win.nlong = 0;
@@ -771,7 +784,7 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
                                            st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
     int launches = 0;
-    if (W > 1) {
+    if (split) {
         for (int i = 0; i < 2; ++i) {
             SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
             SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
@@ -781,7 +794,7 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
         p->ev_chunk.assign(W, nullptr);
         for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
     }
-    if (W > 1) {   // chunk ranges of the long segments
+    if (split) {   // chunk ranges of the long segments
         std::vector<int32_t> cb(2 * W, 0);
         for (int w = 0; w < W; ++w) {
             SD_CUDA_TRY(cudaMemcpyAsync(&cb[2 * w], p->seg_chunk + p->wins[w].seg_begin, 4, cudaMemcpyDeviceToHost, st));
@@ -822,10 +835,11 @@ static sd_status_t build_merge(sd_plan *p, int W, cudaStream_t st) {
     p->info.num_tiles = ntiles;
     p->info.num_segments = p->num_segments;
     p->info.windows = W;
+    p->info.class_split = split ? 1 : 0;
     p->info.launches = launches;
     // Narrow dense operands take the COO segmented reduction instead of the tile kernel (the tile
     // table above stays valid and inspectable): one row index per nonzero and two carry lists.
-    if (W == 1 && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !getenv("SD_NO_COO")) {
+    if (!split && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !getenv("SD_NO_COO")) {
         const int cchunk = coo_chunk(static_cast<int>(p->N));
         const int64_t chunks1 = (p->nnz + cchunk - 1) / cchunk, count2 = 2 * chunks1;
         const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk, count3 = 2 * chunks2;
@@ -1012,8 +1026,13 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     info.launches = 1;
     if (family == SD_MERGE && p->M > 0 && p->nnz > 0) {
         int W = d->windows == 0 ? decide_windows(info, p->dtype) : d->windows;
-        if (info.unsorted_rows != 0) W = 1;   // windows need ascending columns
-        if ((s = build_merge(p, W, st))) return s;
+        bool split = W > 1 || W == -1 || (d->windows == 0 && decide_class_split(info, p->dtype));
+        if (W < 1) W = 1;
+        if (info.unsorted_rows != 0) {   // windows and the class split need ascending columns
+            W = 1;
+            split = false;
+        }
+        if ((s = build_merge(p, W, split, st))) return s;
     } else if (family == SD_BSR_TC) {
         if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
     }
@@ -1105,8 +1124,8 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *d, sd_plan_t **out) {
         set_error(SD_ERR_INVALID_ARG, "unknown family %d", d->family);
         return SD_ERR_INVALID_ARG;
     }
-    if (d->windows < 0 || d->windows > 64) {
-        set_error(SD_ERR_INVALID_ARG, "windows must be in [0, 64]");
+    if (d->windows < -1 || d->windows > 64) {
+        set_error(SD_ERR_INVALID_ARG, "windows must be in [-1, 64]");
         return SD_ERR_INVALID_ARG;
     }
     sd_plan *p = new (std::nothrow) sd_plan;
@@ -1213,14 +1232,14 @@ sd_status_t sd_plan_get_features(sd_plan_t *plan, sd_features_t *out) {
         for (int k = 0; k < 3; ++k)
             f.rep_bytes[5 + k] = (vb * bs[k] * bs[k] + 4) * f.nnzb[k] + 4 * ((info.M + bs[k] - 1) / bs[k] + 1);
         f.shape_class = shape_class_of(info);
-        const bool reads_csr = info.family == SD_ROWSPLIT || (info.family == SD_MERGE && info.windows <= 1);
+        const bool reads_csr = info.family == SD_ROWSPLIT || (info.family == SD_MERGE && !info.class_split);
         f.borrowed_bytes = reads_csr ? f.rep_bytes[0] : 0;
         f.plan_bytes = info.plan_bytes;
         f.d_r = info.K * info.N * vb;
         f.d_s = 4 * info.M * info.N;
         f.m_r = f.borrowed_bytes + f.plan_bytes + f.d_r;
         f.m_t = f.m_r + f.d_s;
-        f.work_units = info.family == SD_MERGE ? (info.windows > 1 ? info.num_segments : info.num_tiles)
+        f.work_units = info.family == SD_MERGE ? (info.class_split ? info.num_segments : info.num_tiles)
                                                : (info.family == SD_BSR_TC ? (info.M + 15) / 16 : info.M);
         f.sm_count = info.sm_count;
         f.l2_bytes = info.l2_bytes;
@@ -1285,8 +1304,8 @@ sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_
         set_error(SD_ERR_INVALID_ARG, "plan is null");
         return SD_ERR_INVALID_ARG;
     }
-    if (plan->info.family != SD_MERGE || plan->wins.size() < 2) {
-        set_error(SD_ERR_UNSUPPORTED, "the plan holds no column-window segment list");
+    if (plan->info.family != SD_MERGE || !plan->info.class_split) {
+        set_error(SD_ERR_UNSUPPORTED, "the plan holds no window-major segment list");
         return SD_ERR_UNSUPPORTED;
     }
     const int64_t S = plan->num_segments;
@@ -1377,7 +1396,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         a.vals = plan->m_vals;
         a.seg_row = plan->m_seg_row;
         a.S = plan->num_segments;
-        const bool side = plan->wins.size() > 1 && plan->aux[0] && !getenv("SD_NO_SIDE_STREAMS");
+        const bool side = plan->aux[0] && !getenv("SD_NO_SIDE_STREAMS");
         // The chunk kernels only read A and B and write their own scratch rows: they run on a stream of
         // their own, up to `depth` windows ahead of the kernels that update C, which wait for their
         // window's event.

@@ -35,13 +35,13 @@ def compare(w, plan):
     assert as_dict(got, COUNT_FIELDS) == as_dict(want, COUNT_FIELDS)
     pinfo = plan.info()
     # Eq. 11-12 for the plan as built
-    reads_csr = pinfo.family == sd.SD_ROWSPLIT or (pinfo.family == sd.SD_MERGE and pinfo.windows <= 1)
+    reads_csr = pinfo.family == sd.SD_ROWSPLIT or (pinfo.family == sd.SD_MERGE and not pinfo.class_split)
     assert got.borrowed_bytes == (oracle.csr_bytes(info, vb) if reads_csr else 0)
     assert got.plan_bytes == pinfo.plan_bytes
     m_r, m_t = oracle.working_set_bytes(got.borrowed_bytes + got.plan_bytes, info, vb)
     assert (got.m_r, got.m_t) == (m_r, m_t)
     assert (got.d_r, got.d_s) == (w.K * w.N * vb, 4 * w.M * w.N)
-    units = {sd.SD_ROWSPLIT: w.M, sd.SD_MERGE: pinfo.num_segments if pinfo.windows > 1 else pinfo.num_tiles,
+    units = {sd.SD_ROWSPLIT: w.M, sd.SD_MERGE: pinfo.num_segments if pinfo.class_split else pinfo.num_tiles,
              sd.SD_BSR_TC: (w.M + 15) // 16}[pinfo.family]
     assert got.work_units == units
     assert (got.sm_count, got.l2_bytes) == (pinfo.sm_count, pinfo.l2_bytes)
@@ -83,7 +83,8 @@ def test_features_of_a_rowsplit_plan_are_the_csr_closed_forms():
 def test_features_with_windows_and_forced_families():
     w = W.config(4, M=1 << 14, scale_c=2.4e7 / 256, cap=800)
     dw = DeviceWorkload(w)
-    for kw in (dict(family=sd.SD_MERGE, windows=4), dict(family=sd.SD_MERGE, windows=1), dict(family=sd.SD_ROWSPLIT)):
+    for kw in (dict(family=sd.SD_MERGE, windows=4), dict(family=sd.SD_MERGE, windows=1), dict(family=sd.SD_MERGE, windows=-1),
+               dict(family=sd.SD_ROWSPLIT)):
         plan = dw.plan(**kw)
         f = compare(w, plan)
         assert sd.SHAPE_NAMES[f.shape_class] == "power-law"

@@ -182,9 +182,16 @@ def test_scaled_configs_auto_plan_and_plan_parity(name):
         assert mine[k] == v, k
     assert info.family == oracle.decide(ref, w.dtype) == EXPECTED_FAMILY[name]
     if info.family == sd.SD_MERGE:
+        assert bool(info.class_split) == (info.windows > 1 or oracle.decide_class_split(ref, w.dtype))
+    if info.family == sd.SD_MERGE and not info.class_split:
         tiles = sd.sd_plan_get_tiles(plan.handle)
         assert np.array_equal(tiles, oracle.merge_coords(w.rowptr, info.tile_items))
         assert info.num_tiles == tiles.size - 1
+    if info.family == sd.SD_MERGE and info.class_split:
+        seg_ptr, seg_row, colind, vals, win_seg = sd.sd_plan_get_segments(plan.handle)
+        rp, rr, perm, rw = oracle.window_segments(w.rowptr, w.colind, w.M, w.K, info.windows)
+        assert np.array_equal(seg_ptr, rp) and np.array_equal(seg_row, rr) and np.array_equal(win_seg, rw)
+        assert np.array_equal(colind, w.colind[perm]) and vals.tobytes() == w.vals[perm].tobytes()
     if info.family == sd.SD_BSR_TC:
         browptr, bcol, bval = sd.sd_plan_get_bsr(plan.handle)
         rb, rc, rv = oracle.bsr16(w.rowptr, w.colind, w.vals, w.M, w.K)
@@ -656,6 +663,51 @@ def test_merge_with_column_windows(kind, windows, N, dtype):
     got3, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
     check(w, got3, beta=0.0)
     plan.close()
+
+
+@pytest.mark.parametrize("kind", ["uniform", "skewed", "onelong"])
+@pytest.mark.parametrize("N,dtype", [(16, W.SD_F32), (32, W.SD_F32), (64, W.SD_BF16), (8, W.SD_F32), (100, W.SD_F32)])
+def test_merge_class_split_with_one_window(kind, N, dtype):
+    """windows = -1: the window-major schedule (chunks, one group per short segment, flat one-nonzero rows)
+    without column windows; segment list against the oracle's construction, results against the oracle."""
+    rng = np.random.default_rng(N)
+    M, K = 1500, 3001
+    lengths = shape_lengths(kind, M, K, rng)
+    lengths[100:110] = 0
+    w = W.random_csr(M, K, N, lengths, seed=N + 3, dtype=dtype, alpha=0.5, beta=1.25)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE, windows=-1)
+    info = plan.info()
+    assert info.windows == 1 and info.class_split == 1
+    seg_ptr, seg_row, colind, vals, win_seg = sd.sd_plan_get_segments(plan.handle)
+    rp, rr, perm, rw = oracle.window_segments(w.rowptr, w.colind, M, K, 1)
+    assert np.array_equal(seg_ptr, rp) and np.array_equal(seg_row, rr) and np.array_equal(win_seg, rw)
+    assert np.array_equal(colind, w.colind[perm]) and vals.tobytes() == w.vals[perm].tobytes()
+    assert not np.any(seg_row < 0)       # one window: no row is written twice
+    got, intact = run_spmm(plan, w)
+    assert intact
+    check(w, got)
+    got2, _ = run_spmm(plan, w)
+    assert np.array_equal(got, got2)
+    poison = np.full((M, N), np.nan, np.float32)
+    got3, _ = run_spmm(plan, w, c_fill=poison, beta=0.0)
+    check(w, got3, beta=0.0)
+    plan.close()
+
+
+def test_automatic_class_split_matches_the_rule():
+    for N, dtype in ((32, W.SD_F32), (16, W.SD_F32), (64, W.SD_F32), (64, W.SD_BF16), (8, W.SD_F32)):
+        w = W.config(2, scale=12, N=N, dtype=dtype)
+        dw = DeviceWorkload(w)
+        plan = dw.plan()
+        info = plan.info()
+        ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
+        assert info.family == sd.SD_MERGE == oracle.decide(ref, dtype)
+        assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes) == 1
+        assert bool(info.class_split) == oracle.decide_class_split(ref, dtype) == (N * (4 if dtype == W.SD_F32 else 2) in (64, 128))
+        got, _ = run_spmm(plan, w)
+        check(w, got)
+        plan.close()
 
 
 def test_automatic_window_choice_matches_the_rule():

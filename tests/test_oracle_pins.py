@@ -528,6 +528,23 @@ def test_o4_window_rule():
     assert oracle.decide_windows(info, oracle.F32, 126 * 2**20) == 1     # B fits
 
 
+def test_o4_class_split_rule_by_row_bytes_of_the_dense_operand():
+    info = oracle.Info()
+    info.M = info.K = 1 << 20
+    info.nnz = 32 << 20
+    for dt, N, want in ((oracle.F32, 8, False), (oracle.F32, 16, True), (oracle.F32, 32, True), (oracle.F32, 24, False),
+                        (oracle.F32, 64, False), (oracle.F32, 128, False), (oracle.BF16, 16, False),
+                        (oracle.BF16, 32, True), (oracle.BF16, 64, True), (oracle.BF16, 128, False)):
+        info.N = N
+        assert oracle.decide_class_split(info, dt) == want, (dt, N)
+    info.N = 32
+    info.unsorted_rows = 1
+    assert not oracle.decide_class_split(info, oracle.F32)      # needs ascending columns
+    info.unsorted_rows = 0
+    info.nnz = 0
+    assert not oracle.decide_class_split(info, oracle.F32)
+
+
 # ------------------------------------------------------------------ O5
 def _features_of(w, value_bytes=4):
     info = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
