@@ -476,13 +476,13 @@ int sdo_decide_windows(const sdo_info_t *o, int dtype, int64_t l2_bytes)
 
 /* Class split at one window (this build's rule, parity unpinned): the window-major schedule
  * (long segments cut into chunks, short ones one lane group each, one-nonzero rows flat) without
- * column windows, taken by merge-family plans whose rows are sorted when a row of B is exactly
- * 64 or 128 bytes; measured on the target GPU against the merge-path tiles, which stay ahead at
- * 32 bytes and from 256 bytes on. */
+ * column windows, taken by merge-family plans whose rows are sorted when the dense width is
+ * 16 to 32 columns, either value type; measured on the target GPU against the merge-path tiles,
+ * which stay ahead or level at 8 columns and from 64 columns on. */
 int sdo_decide_class_split(const sdo_info_t *o, int dtype)
 {
-    int64_t row_bytes = o->N * (dtype == SDO_F32 ? 4 : 2);
-    return o->unsorted_rows == 0 && o->nnz > 0 && (row_bytes == 64 || row_bytes == 128);
+    (void)dtype;
+    return o->unsorted_rows == 0 && o->nnz > 0 && o->N >= 16 && o->N <= 32;
 }
 
 /* Window-major segment list.  Window of a column: col / ceil(K / W).  A segment is the part

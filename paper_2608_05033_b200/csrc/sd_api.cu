@@ -530,12 +530,12 @@ static int decide_windows(const sd_plan_info_t &s, int dtype) {
 }
 
 // One window, but still the class split (long segments as chunks, short ones one lane group each,
-// one-nonzero rows flat) instead of merge-path tiles: measured on the R-MAT matrix, the split is ahead
-// where a row of B is 64 or 128 bytes (0.322 against 0.362 ms and 0.414 against 0.482 ms) and behind at
-// 32 bytes and from 256 bytes on.  Needs ascending columns like the windows.
+// one-nonzero rows flat) instead of merge-path tiles: measured on R-MAT and rank-size matrices, fp32 and
+// bf16, the split is ahead at 16 and 32 columns (0.68 to 0.92 of the tile kernel's time) and behind or
+// level at 8 and from 64 columns on.  Needs ascending columns like the windows.
 static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
-    const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
-    return s.unsorted_rows == 0 && s.nnz > 0 && (row_bytes == 64 || row_bytes == 128);
+    (void)dtype;
+    return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= 16 && s.N <= 32;
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {
