@@ -215,7 +215,19 @@ template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_seg_one(const SpmmArgs &a, bool scratch, cudaStream_t st) {
     const int per_cta = kSegThreads / LPR;
     const int64_t need = (a.S + per_cta - 1) / per_cta;
-    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * 8;   // 8 CTAs of 256 threads fill an SM
+    // persistent grid: exactly the CTAs that are resident together (the registers of an instance decide how
+    // many of the eight 256-thread CTAs an SM takes); a larger grid would run a thin second wave
+    static const int occ_scratch = [] {
+        int n = 8;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, seg_kernel<T, VW, LPR, NV, true>, kSegThreads, 0) != cudaSuccess) n = 8;
+        return n < 1 ? 1 : n;
+    }();
+    static const int occ_plain = [] {
+        int n = 8;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, seg_kernel<T, VW, LPR, NV, false>, kSegThreads, 0) != cudaSuccess) n = 8;
+        return n < 1 ? 1 : n;
+    }();
+    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * (scratch ? occ_scratch : occ_plain);
     dim3 grid(static_cast<unsigned>(need < cap ? need : cap),
               static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
     if (scratch) seg_kernel<T, VW, LPR, NV, true><<<grid, kSegThreads, 0, st>>>(a);
