@@ -10,9 +10,9 @@ cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st
         if (dtype == SD_F32) return launch_rowsplit_narrow<float>(a, vec, st);
         return launch_rowsplit_narrow<__nv_bfloat16>(a, vec, st);
     }
-    // 8 to 32 columns (fp32; 16 to 64 bf16) as whole 16-byte vectors and long rows: several lane sets per row
+    // 8 to 64 columns (fp32; 8 to 128 bf16) as whole 16-byte vectors and long rows: several lane sets per row
     const int vw = dtype == SD_F32 ? 4 : 8;
-    if (vec && a.N % vw == 0 && a.N / vw <= 8 && ((a.N / vw) & (a.N / vw - 1)) == 0) {
+    if (vec && a.N % vw == 0 && a.N / vw <= 16 && ((a.N / vw) & (a.N / vw - 1)) == 0) {
         const int lpr = a.N / vw;
         const int g = ksplit_group(a.mean_len, lpr);
         if (g > 1) {

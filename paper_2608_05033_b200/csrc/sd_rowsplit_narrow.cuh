@@ -118,7 +118,7 @@ rowsplit_narrow_kernel(const SpmmArgs a) {
     }
 }
 
-// The same scheme at 8 to 32 columns (one 16-byte vector per lane, LPR = 2..8 lanes across the columns):
+// The same scheme at 8 to 64 columns (one 16-byte vector per lane, LPR = 2..16 lanes across the columns):
 // G such lane sets share a row, set k takes the nonzeros p0 + k, p0 + k + G, ...; the G partial rows meet by
 // xor shuffles over the set index.  Pays when rows are long enough to keep G sets busy (the paper's
 // af_shell10 case: a few threads per row, each holding several outputs); short rows keep the plain kernel.
@@ -200,9 +200,11 @@ inline int ksplit_override() {
 // the mean row, at most 16 lanes per row below a mean of 128 nonzeros and a whole warp from there.
 inline int ksplit_group(int64_t mean_len, int lpr) {
     int g = 1;
-    const int lanes = mean_len >= 128 ? 32 : 16;
+    // 16 lanes across the columns (64 fp32 / 128 bf16 columns): two sets from a mean of 32 nonzeros
+    const int lanes = (mean_len >= 128 || lpr >= 16) ? 32 : 16;
+    const int64_t per_set = lpr >= 16 ? 16 : 8;
     if (const int o = ksplit_override()) g = o;
-    else while (2 * g * lpr <= lanes && 2 * g <= mean_len / 8) g <<= 1;
+    else while (2 * g * lpr <= lanes && 2 * g <= mean_len / per_set) g <<= 1;
     while (g > 1 && g * lpr > 32) g >>= 1;
     return g;
 }
@@ -221,7 +223,7 @@ cudaError_t launch_ksplit_g(const SpmmArgs &a, cudaStream_t st) {
     }
 }
 
-// N * sizeof(T) = 16 * LPR bytes exactly, LPR in {2, 4, 8}; g from ksplit_group (> 1).
+// N * sizeof(T) = 16 * LPR bytes exactly, LPR in {1, 2, 4, 8, 16}; g from ksplit_group (> 1).
 template <typename T>
 cudaError_t launch_rowsplit_ksplit(const SpmmArgs &a, int lpr, int g, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
@@ -231,6 +233,7 @@ cudaError_t launch_rowsplit_ksplit(const SpmmArgs &a, int lpr, int g, cudaStream
     SD_KS_CASE(2, 2) SD_KS_CASE(2, 4) SD_KS_CASE(2, 8) SD_KS_CASE(2, 16)
     SD_KS_CASE(4, 2) SD_KS_CASE(4, 4) SD_KS_CASE(4, 8)
     SD_KS_CASE(8, 2) SD_KS_CASE(8, 4)
+    SD_KS_CASE(16, 2)
 #undef SD_KS_CASE
     return cudaErrorInvalidValue;
 }

@@ -388,11 +388,11 @@ def test_row_and_column_shards_of_one_product(world, dtype):
     check(w, Cd.cpu().numpy())
 
 
-@pytest.mark.parametrize("dtype,N", [(W.SD_F32, 8), (W.SD_F32, 16), (W.SD_F32, 32), (W.SD_BF16, 8), (W.SD_BF16, 16),
-                                     (W.SD_BF16, 32), (W.SD_BF16, 64)])
+@pytest.mark.parametrize("dtype,N", [(W.SD_F32, 8), (W.SD_F32, 16), (W.SD_F32, 32), (W.SD_F32, 64), (W.SD_BF16, 8),
+                                     (W.SD_BF16, 16), (W.SD_BF16, 32), (W.SD_BF16, 64), (W.SD_BF16, 128)])
 @pytest.mark.parametrize("mean", [20, 40, 70, 300])
 def test_rowsplit_long_rows_several_lane_sets_per_row(mean, N, dtype):
-    """Row-split family at 8 to 32 fp32 (8 to 64 bf16) columns with long rows: 2 to 16 lane sets share a
+    """Row-split family at 8 to 64 fp32 (8 to 128 bf16) columns with long rows: 2 to 16 lane sets share a
     row and meet by shuffles; empty rows, one row far beyond the mean (two-level sum), ragged row count,
     padded leading dimensions, and a misaligned call that must take the plain kernel."""
     rng = np.random.default_rng(mean * 100 + N)
