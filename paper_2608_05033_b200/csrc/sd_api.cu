@@ -488,15 +488,20 @@ struct TempBuf {   // frees temporary device memory on every exit path
 // depends on the number of blocks only, the CSR kernels' time on the number of nonzeros; the
 // measured cross-over (random 16x16 blocks thinned to a given fill) by width and value type:
 //              N < 128   128 <= N < 256   N >= 256
-//     fp32       3/2          2              11/4
-//     bf16       3            5              7
+//     fp32       9/8          2              11/4
+//     bf16       9/4          4              7
 static int decide_family(const sd_plan_info_t &s, int dtype) {
     int64_t num, den = 1;
     if (dtype == SD_BF16) {
-        num = s.N < 128 ? 3 : (s.N < 256 ? 5 : 7);
+        if (s.N < 128) {
+            num = 9;
+            den = 4;
+        } else {
+            num = s.N < 256 ? 4 : 7;
+        }
     } else if (s.N < 128) {
-        num = 3;
-        den = 2;
+        num = 9;
+        den = 8;
     } else if (s.N < 256) {
         num = 2;
     } else {
