@@ -53,7 +53,7 @@ def test_forced_family_small(family, kind, N, dtype):
     M, K = 1237, 3001   # ragged: not multiples of any tile
     w = W.random_csr(M, K, N, shape_lengths(kind, M, K, rng), seed=N * 7 + 1, dtype=dtype, alpha=1.25, beta=-0.5)
     dw = DeviceWorkload(w)
-    plan = dw.plan(family=FAMILIES[family])
+    plan = dw.plan(family=FAMILIES[family], windows=1 if family == "merge" else 0)   # merge: the row-ordered tile kernel
     assert plan.info().family == FAMILIES[family]
     got, intact = run_spmm(plan, w)
     assert intact
@@ -75,12 +75,13 @@ def test_padding_and_misalignment(family, dtype):
     M, K, N = 300, 517, 32
     w = W.random_csr(M, K, N, np.clip(rng.poisson(6, M), 0, K), seed=77, dtype=dtype, beta=0.75)
     dw = DeviceWorkload(w)
-    plan = dw.plan(family=FAMILIES[family])
-    for pad_b, pad_c, off in [(3, 5, 0), (4, 8, 0), (0, 0, 1), (1, 2, 3), (8, 4, 4)]:
-        got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_c, offset=off)
-        assert intact, (pad_b, pad_c, off)
-        check(w, got)
-    plan.close()
+    for windows in ((1, -1) if family == "merge" else (0,)):   # merge: tile kernel, then the class split
+        plan = dw.plan(family=FAMILIES[family], windows=windows)
+        for pad_b, pad_c, off in [(3, 5, 0), (4, 8, 0), (0, 0, 1), (1, 2, 3), (8, 4, 4)]:
+            got, intact = run_spmm(plan, w, pad_b=pad_b, pad_c=pad_c, offset=off)
+            assert intact, (pad_b, pad_c, off)
+            check(w, got)
+        plan.close()
 
 
 @pytest.mark.parametrize("family", ["rowsplit", "merge", "bsr"])
@@ -277,7 +278,7 @@ def test_one_row_holds_every_nonzero_and_rows_straddle_many_tiles():
     r = np.full(40, 2600, np.int64)
     w = W.random_csr(40, 8192, 32, r, seed=3, beta=0.25)
     dw = DeviceWorkload(w)
-    plan = dw.plan(family=sd.SD_MERGE)
+    plan = dw.plan(family=sd.SD_MERGE, windows=1)
     got, _ = run_spmm(plan, w)
     check(w, got)
     plan.close()
@@ -443,7 +444,7 @@ def test_symmetric_adjacency_forward_plan_serves_the_backward_product(N):
     plan.close()
 
 
-@pytest.mark.parametrize("case", ["rowsplit", "merge", "merge_narrow", "merge_windows", "bsr_bf16", "bsr_f32"])
+@pytest.mark.parametrize("case", ["rowsplit", "merge", "merge_split", "merge_narrow", "merge_windows", "bsr_bf16", "bsr_f32"])
 def test_update_values_same_pattern(case):
     # new values for an unchanged pattern: every representation that holds its own copy of the values
     # (window-major lists, 16x16 blocks and their tensor-core images) must follow
@@ -458,7 +459,7 @@ def test_update_values_same_pattern(case):
         N = 3 if case == "merge_narrow" else 32
         lengths = shape_lengths("skewed", M, K, rng)
         family = sd.SD_ROWSPLIT if case == "rowsplit" else sd.SD_MERGE
-        windows = 4 if case == "merge_windows" else 0
+        windows = {"merge_windows": 4, "merge_split": -1, "merge": 1}.get(case, 0)   # merge: row-ordered tiles
     w = W.random_csr(M, K, N, lengths, seed=77, dtype=dtype, alpha=1.0, beta=0.0)
     dw = DeviceWorkload(w)
     plan = dw.plan(family=family, windows=windows)
