@@ -535,12 +535,13 @@ static int decide_windows(const sd_plan_info_t &s, int dtype) {
 }
 
 // One window, but still the class split (long segments as chunks, short ones one lane group each,
-// one-nonzero rows flat) instead of merge-path tiles: measured on R-MAT and rank-size matrices, fp32 and
-// bf16, the split is ahead at 16 and 32 columns (0.68 to 0.92 of the tile kernel's time) and behind or
-// level at 8 and from 64 columns on.  Needs ascending columns like the windows.
+// one-nonzero rows flat) instead of merge-path tiles: measured on R-MAT and rank-size matrices, the split
+// is ahead from 16 columns up to 64 fp32 / 32 bf16 columns (0.68 to 0.94 of the tile kernel's time) and
+// behind or level at 8 columns and beyond (bf16 at 128 columns: 1.27).  Needs ascending columns like the
+// windows.
 static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
-    (void)dtype;
-    return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= 16 && s.N <= 32;
+    const int64_t widest = dtype == SD_BF16 ? 32 : 64;
+    return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= 16 && s.N <= widest;
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {

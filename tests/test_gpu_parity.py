@@ -697,7 +697,8 @@ def test_merge_class_split_with_one_window(kind, N, dtype):
 
 
 def test_automatic_class_split_matches_the_rule():
-    for N, dtype in ((32, W.SD_F32), (16, W.SD_F32), (24, W.SD_F32), (64, W.SD_F32), (32, W.SD_BF16), (64, W.SD_BF16), (8, W.SD_F32)):
+    for N, dtype in ((32, W.SD_F32), (16, W.SD_F32), (24, W.SD_F32), (64, W.SD_F32), (128, W.SD_F32), (32, W.SD_BF16), (64, W.SD_BF16),
+                     (8, W.SD_F32)):
         w = W.config(2, scale=12, N=N, dtype=dtype)
         dw = DeviceWorkload(w)
         plan = dw.plan()
@@ -705,7 +706,7 @@ def test_automatic_class_split_matches_the_rule():
         ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
         assert info.family == sd.SD_MERGE == oracle.decide(ref, dtype)
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes) == 1
-        assert bool(info.class_split) == oracle.decide_class_split(ref, dtype) == (16 <= N <= 32)
+        assert bool(info.class_split) == oracle.decide_class_split(ref, dtype) == (16 <= N <= (64 if dtype == W.SD_F32 else 32))
         got, _ = run_spmm(plan, w)
         check(w, got)
         plan.close()
