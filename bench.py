@@ -341,7 +341,9 @@ def run_gpu(args, rank, local_rank, world):
 
     # ---- gather ceiling: the workload's own index stream as bare row gathers ------------------------
     if args.probe and rank == 0:
-        sink = torch.zeros(sd.sd_probe_gather(None, 0, None, 128), dtype=torch.float32, device=dev)
+        import bench_probes
+        bench_probes.build()
+        sink = torch.zeros(bench_probes.sink_floats(), dtype=torch.float32, device=dev)
         for c in cases:
             w = c["w"]
             row_bytes = w.N * (4 if w.dtype == W.SD_F32 else 2)
@@ -353,7 +355,7 @@ def run_gpu(args, rank, local_rank, world):
                 flush.fill_(1.0)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-                sd.sd_probe_gather(colind, w.nnz, c["B"], row_bytes, sink, stream)
+                bench_probes.gather(0, colind, w.nnz, c["B"], row_bytes, sink, stream=stream)
                 e1.record(stream)
                 torch.cuda.synchronize()
                 if i >= 3:
@@ -544,6 +546,70 @@ def run_gcn_epoch(args, local_rank):
         "clocks": clocks, "per_width": rows}))
 
 
+def run_probe_paths(args, local_rank):
+    """Fetch paths for the gathers of the dense operand, timed on the GCN workload's own column stream
+    (512-byte rows, storage order): plain loads with 4 / 8 / 16 gathers in flight per lane, L2 evict-last and
+    L1 no-allocate hints, tile order with staged indices, half a warp per row, bulk copies into a shared-memory
+    ring, and the hottest rows kept in the distributed shared memory of a thread-block cluster.  Every round
+    times every path once (cold L2), so drifts hit all paths alike; prints one JSON line of its own."""
+    import torch
+    import bench_probes as bp
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    bp.build()
+    kw = dict(SMALL_KW[2]) if args.small else {}
+    w = W.config(2, dtype=W.SD_F32, **kw)
+    assert w.N * 4 == 512
+    colind = torch.from_numpy(w.colind).to(dev)
+    table = torch.from_numpy(w.B).to(dev)
+    sink = torch.zeros(bp.sink_floats(), dtype=torch.float32, device=dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    # hub rows = the most referenced columns; their indices in the stream carry bit 31 and the hub slot
+    deg = np.bincount(w.colind, minlength=w.K)
+    order = np.argsort(-deg, kind="stable").astype(np.int32)
+    hub_streams = {}
+    for path, cl in bp.HUB_CLUSTER.items():
+        nh = cl * bp.HUB_ROWS_PER_CTA
+        slot = np.full(w.K, -1, dtype=np.int64)
+        slot[order[:nh]] = np.arange(nh)
+        s = slot[w.colind]
+        enc = np.where(s >= 0, s | 0x80000000, w.colind).astype(np.uint32).view(np.int32)
+        hub_streams[path] = (torch.from_numpy(enc).to(dev), torch.from_numpy(order[:nh].copy()).to(dev), float((s >= 0).mean()))
+    paths = sorted(bp.PATHS)
+    times = {p: [] for p in paths}
+    info = {}
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    rounds = max(args.steps, 5) + 2
+    for rep in range(rounds):
+        for p in paths:
+            idx, hub = (hub_streams[p][0], hub_streams[p][1]) if p in hub_streams else (colind, None)
+            flush.fill_(1.0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            info[p] = bp.gather(p, idx, w.nnz, table, 512, sink, err=err, hubrows=hub, stream=stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if rep >= 2:
+                times[p].append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
+    rows = []
+    for p in paths:
+        ms = float(np.median(times[p]))
+        row = {"path": p, "name": bp.PATHS[p], "ms_median": ms, "ms_min": float(np.min(times[p])),
+               "gathered_tbs": w.nnz * 512 / (ms * 1e-3) / 1e12, "resident": info[p]}
+        if p in hub_streams:
+            row["hub_fraction_of_gathers"] = hub_streams[p][2]
+        rows.append(row)
+    print(json.dumps({"mode": "probe-paths", "workload": w.name, "nnz": w.nnz, "row_bytes": 512, "rounds": rounds - 2,
+                      "bulk_ring_error_word": int(err.item()), "clocks": clocks, "paths": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -555,6 +621,8 @@ def main():
     ap.add_argument("--probe", action="store_true",
                     help="also replay every workload's colind stream as bare row gathers (sd_probe_gather) and "
                          "report its time beside the SpMM time: the gather ceiling of the memory system for that stream")
+    ap.add_argument("--probe-paths", action="store_true",
+                    help="time the fetch paths of bench_probes on the GCN workload's column stream (prints its own JSON line)")
     ap.add_argument("--width", type=int, default=0,
                     help="override the dense width N of every selected workload (width sweep: 1 = SpMV, 8, 32, "
                          "128, 256); not the benchmark configuration")
@@ -577,6 +645,10 @@ def main():
     if args.gcn_epoch:
         if rank == 0:
             run_gcn_epoch(args, local_rank)
+        return
+    if args.probe_paths:
+        if rank == 0:
+            run_probe_paths(args, local_rank)
         return
     run_gpu(args, rank, local_rank, world)
     if world > 1:

@@ -275,8 +275,9 @@ sd_status_t sd_plan_device_status(sd_plan_t *plan, int32_t *status);
  * take cudaMalloc's device-wide synchronisation; code under a fixed memory budget.  A plan
  * allocates its tile table and carry-out rows; here they live in one fixed 4 MiB array inside
  * the library's device image (every GPU that loads the library holds it until exit).
- *   rowptr [M+1], colind [nnz], vals [nnz]   device, as for sd_plan_create; nnz = rowptr[M]
- *                                            is passed in so that nothing is read back
+ *   rowptr [M+1], colind [nnz], vals [nnz]   device, as for sd_plan_create (rowptr[0] == 0 is
+ *                                            relied upon, not checked); nnz = rowptr[M] is passed
+ *                                            in so that nothing is read back
  *   B device [K, ldb] fp32, C device [M, ldc] fp32, ldb, ldc >= N; alpha/beta as sd_spmm.
  * Size limit: with T = ceil((M + nnz) / 1024) tiles, 4*(T+1) rounded up to 256, plus 8*T*N
  * bytes, must fit in 4 MiB (N = 32: about 16 million rows + nonzeros); beyond that the call
@@ -290,18 +291,6 @@ sd_status_t sd_spmm_merge_static(const int32_t *rowptr, const int32_t *colind, c
                                  int64_t M, int64_t K, int64_t N, int64_t nnz, const float *B,
                                  int64_t ldb, float *C, int64_t ldc, float alpha, float beta,
                                  void *stream);
-
-/* sd_probe_gather -- measurement aid (no counterpart in the paper).  Replays `count` row
- * indices idx[] (device, e.g. the colind array of a CSR matrix, in storage order) as bare
- * gathers of `row_bytes`-byte rows (16, 32, ..., 512; 16-byte aligned table, row pitch =
- * row_bytes) from `table` (device): the memory access stream of SpMM with the values of A, the
- * multiply-adds and the output removed.  Its time is the rate at which the memory system
- * delivers that gather stream, against which bench.py sets the time of the SpMM kernels.
- * `sink` (device) receives one partial sum per thread so that the loads stay alive; a call with
- * idx, table and sink all NULL only reports the floats `sink` must hold in *sink_floats_needed.
- * Asynchronous on `stream`; allocates nothing. */
-sd_status_t sd_probe_gather(const int32_t *idx, int64_t count, const void *table, int32_t row_bytes,
-                            float *sink, int32_t *sink_floats_needed, void *stream);
 
 /* sd_last_error -- copy the calling thread's last error text into buf (NUL-terminated,
  * at most n bytes); returns the last status code. */

@@ -22,7 +22,7 @@ SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_probe_gather", "sd_last_error",
+           "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_last_error",
            "sd_version"]
 
 
@@ -109,9 +109,6 @@ def load():
     lib.sd_spmm_merge_static.restype = C.c_int
     lib.sd_spmm_merge_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_float, C.c_float, C.c_void_p]
-    lib.sd_probe_gather.restype = C.c_int
-    lib.sd_probe_gather.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32),
-                                    C.c_void_p]
     lib.sd_last_error.restype = C.c_int
     lib.sd_last_error.argtypes = [C.c_char_p, C.c_size_t]
     lib.sd_version.restype = C.c_char_p
@@ -212,17 +209,6 @@ def sd_spmm_merge_static(rowptr, colind, vals, M: int, K: int, N: int, nnz: int,
                                      ldc, alpha, beta, _stream_handle(stream))
     if rc != SD_OK:
         _raise(rc)
-
-
-def sd_probe_gather(idx, count: int, table, row_bytes: int, sink=None, stream=None) -> int:
-    """Bare gather of `count` rows of `row_bytes` bytes by the index stream idx (see include/sd.h).
-    With idx = table = sink = None returns the number of floats `sink` must hold."""
-    need = C.c_int32(0)
-    rc = load().sd_probe_gather(_ptr(idx), count, _ptr(table), row_bytes, _ptr(sink), C.byref(need),
-                                _stream_handle(stream) if idx is not None else None)
-    if rc != SD_OK:
-        _raise(rc)
-    return need.value
 
 
 def sd_plan_destroy(plan):

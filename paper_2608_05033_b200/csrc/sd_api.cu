@@ -33,6 +33,31 @@ sd_status_t cuda_fail(cudaError_t e, const char *what) {
     return SD_ERR_CUDA;
 }
 
+static int env_int(const char *name, int dflt) {
+    const char *e = getenv(name);
+    return e ? atoi(e) : dflt;
+}
+
+const Switches &switches() {
+    static const Switches sw = [] {
+        Switches s;
+        s.no_coo = getenv("SD_NO_COO") != nullptr;
+        s.no_side_streams = getenv("SD_NO_SIDE_STREAMS") != nullptr;
+        s.no_chunk_ahead = getenv("SD_NO_CHUNK_AHEAD") != nullptr;
+        s.bsr_simt = getenv("SD_BSR_SIMT") != nullptr;
+        s.no_narrow = getenv("SD_NO_NARROW") != nullptr;
+        s.geom_nv = env_int("SD_GEOM_NV", 0);
+        s.ksplit_g = env_int("SD_KSPLIT_G", 0);
+        s.narrow_g = env_int("SD_NARROW_G", 0);
+        s.tc_sb = env_int("SD_TC_SB", 0);
+        s.tc_stages = env_int("SD_TC_STAGES", 0);
+        s.tc32_sb = env_int("SD_TC32_SB", 0);
+        s.tc32_stages = env_int("SD_TC32_STAGES", 0);
+        return s;
+    }();
+    return sw;
+}
+
 // =====================================================================================
 // structure scan kernels (Sec. 3.1, intrinsic pattern features; integers only)
 // =====================================================================================
@@ -845,7 +870,7 @@ static sd_status_t build_merge(sd_plan *p, int W, bool split, cudaStream_t st) {
     p->info.launches = launches;
     // Narrow dense operands take the COO segmented reduction instead of the tile kernel (the tile
     // table above stays valid and inspectable): one row index per nonzero and two carry lists.
-    if (!split && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !getenv("SD_NO_COO")) {
+    if (!split && p->N >= 1 && p->N <= kCooMaxN && p->nnz > 0 && !switches().no_coo) {
         const int cchunk = coo_chunk(static_cast<int>(p->N));
         const int64_t chunks1 = (p->nnz + cchunk - 1) / cchunk, count2 = 2 * chunks1;
         const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk, count3 = 2 * chunks2;
@@ -1402,11 +1427,11 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         a.vals = plan->m_vals;
         a.seg_row = plan->m_seg_row;
         a.S = plan->num_segments;
-        const bool side = plan->aux[0] && !getenv("SD_NO_SIDE_STREAMS");
+        const bool side = plan->aux[0] && !switches().no_side_streams;
         // The chunk kernels only read A and B and write their own scratch rows: they run on a stream of
         // their own, up to `depth` windows ahead of the kernels that update C, which wait for their
         // window's event.
-        const bool ahead = side && plan->chunk_stream && !getenv("SD_NO_CHUNK_AHEAD");
+        const bool ahead = side && plan->chunk_stream && !switches().no_chunk_ahead;
         auto launch_chunks = [&](size_t w, cudaStream_t cs) -> sd_status_t {
             const sd_plan::Window &win = plan->wins[w];
             SpmmArgs ca = a;
@@ -1534,7 +1559,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         b.beta = beta;
         const bool vec4 = aligned16(B) && aligned16(C) && N % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
                           (plan->dtype == SD_F32 || (reinterpret_cast<uintptr_t>(B) & 7u) == 0);
-        if (bsr_tc_usable(b, plan->dtype) && !getenv("SD_BSR_SIMT"))
+        if (bsr_tc_usable(b, plan->dtype) && !switches().bsr_simt)
             SD_CUDA_TRY(run_bsr_tc(b, plan->dtype, plan->dev_error, plan->info.sm_count, st));
         else
             SD_CUDA_TRY(run_bsr_simt(b, plan->dtype, vec4, st));

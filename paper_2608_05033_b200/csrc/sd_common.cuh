@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/sd.h"
 
 namespace sd {
@@ -153,6 +155,52 @@ struct SpmmArgs {
     int64_t max_len;        // longest row / segment if known (0: unknown); lets the row-split kernel drop its second accumulator
     int64_t mean_len;       // mean row length rounded up if known (0: unknown): lanes per row of the narrow row-split kernel
 };
+
+// A/B measurement switches (none is needed in normal use).  The environment is read once, at the
+// first use in the process (thread-safe), never on the sd_spmm path.
+struct Switches {
+    bool no_coo;           // SD_NO_COO: generic merge kernel at one to four columns
+    bool no_side_streams;  // SD_NO_SIDE_STREAMS: the classes of a window on one stream
+    bool no_chunk_ahead;   // SD_NO_CHUNK_AHEAD: chunk kernels in window order
+    bool bsr_simt;         // SD_BSR_SIMT: SIMT block kernel instead of the tensor-core one
+    bool no_narrow;        // SD_NO_NARROW: wide row-split kernel at one to four columns
+    int geom_nv;           // SD_GEOM_NV: 1 forces one vector per lane
+    int ksplit_g;          // SD_KSPLIT_G: lane sets per row (0: rule, 1: off)
+    int narrow_g;          // SD_NARROW_G: lanes per row of the narrow row-split kernel (0: rule)
+    int tc_sb, tc_stages, tc32_sb, tc32_stages;   // SD_TC_SB / SD_TC_STAGES / SD_TC32_SB / SD_TC32_STAGES: ring geometry (0: default)
+};
+const Switches &switches();
+
+// Per-device caches of launch facts (SM count, resident CTAs of a kernel instance, attributes already set):
+// one slot per device ordinal, published with atomics, so that a process driving several GPUs, or several
+// host threads making their first call together, never reads another device's value or a torn one.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+    return dev;
+}
+inline int sm_count_cached() {
+    static std::atomic<int> cache[kMaxDevices];
+    const int dev = current_device();
+    int v = dev < kMaxDevices ? cache[dev].load(std::memory_order_relaxed) : 0;
+    if (v > 0) return v;
+    v = 148;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    if (dev < kMaxDevices) cache[dev].store(v, std::memory_order_relaxed);
+    return v;
+}
+// CTAs of `kernel` (threads per CTA, no dynamic shared memory) that are resident together on one SM of the current device.
+template <typename Kernel>
+inline int occupancy_cached(std::atomic<int> (&cache)[kMaxDevices], Kernel kernel, int threads) {
+    const int dev = current_device();
+    int v = dev < kMaxDevices ? cache[dev].load(std::memory_order_relaxed) : 0;
+    if (v > 0) return v;
+    v = 8;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, kernel, threads, 0) != cudaSuccess || v < 1) v = v < 1 ? 1 : 8;
+    if (dev < kMaxDevices) cache[dev].store(v, std::memory_order_relaxed);
+    return v;
+}
 
 inline int ceil_div(int64_t a, int64_t b) { return static_cast<int>((a + b - 1) / b); }
 

@@ -122,7 +122,7 @@ coo_reduce_kernel(const CooArgs a) {
 #pragma unroll
             for (int u = 0; u < kCooU; ++u)
 #pragma unroll
-                for (int e = 0; e < N; ++e) p[u][e] *= av[u];
+                for (int e = 0; e < N; ++e) p[u][e] = (r[u] >= 0) ? p[u][e] * av[u] : 0.f;   // items past the end gathered row 0: never let its contents (Inf, NaN) in
         }
         if (!whole) {   // items past the end of the list continue the last row with zeros
             const int64_t last = a.count - 1;

@@ -82,11 +82,6 @@ bool bsr_tc_usable(const BsrArgs &a, int dtype) {
     return encode_tiled() != nullptr;
 }
 
-static int env_int(const char *name, int dflt) {
-    const char *e = getenv(name);
-    return e ? atoi(e) : dflt;
-}
-
 cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_count, cudaStream_t st) {
     const bool tf32 = dtype == SD_F32;
     const int group = tf32 ? 32 : 64, es = tf32 ? 4 : 2;
@@ -124,20 +119,23 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     // takes most of the shared memory: bf16 2 slots of 8 blocks (8.5 KB per block), fp32 3 slots
     // of 2 blocks (34 KB per block).  A barrier round trip costs far more than a block's work,
     // so slots hold several blocks.
-    t.sb = env_int(tf32 ? "SD_TC32_SB" : "SD_TC_SB", tf32 ? 2 : 8);
-    t.stages = env_int(tf32 ? "SD_TC32_STAGES" : "SD_TC_STAGES", tf32 ? 3 : 2);
+    const Switches &sw = switches();
+    t.sb = tf32 ? (sw.tc32_sb ? sw.tc32_sb : 2) : (sw.tc_sb ? sw.tc_sb : 8);
+    t.stages = tf32 ? (sw.tc32_stages ? sw.tc32_stages : 3) : (sw.tc_stages ? sw.tc_stages : 2);
     if (t.sb < 1) t.sb = 1;
     if (t.sb > 32) t.sb = 32;   // one mask bit per block of a ring slot
     if (t.stages < 1) t.stages = 1;
     if (t.stages > kTcMaxStages) t.stages = kTcMaxStages;
     const int smem = t.stages * tc_stage_bytes(tf32, t.sb) + 2048 + 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks + 2 * tc_mask_words(t.sb));
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
-    static int attr_set[2] = {0, 0};
-    if (attr_set[tf32] < smem) {
+    // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the kernel
+    static std::atomic<int> attr_set[kMaxDevices][2];
+    const int dev = current_device();
+    if (dev >= kMaxDevices || attr_set[dev][tf32].load(std::memory_order_acquire) < smem) {
         cudaError_t e = tf32 ? cudaFuncSetAttribute(bsr_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
                              : cudaFuncSetAttribute(bsr_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        attr_set[tf32] = smem;
+        if (dev < kMaxDevices) attr_set[dev][tf32].store(smem, std::memory_order_release);
     }
     const int grid = a.nparts;
     (void)sm_count;

@@ -31,19 +31,12 @@ static cudaError_t launch_coo_n(const CooPlan &cp, const SpmmArgs &s, bool vec, 
     const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk;
     const int64_t count3 = 2 * chunks2;
     // persistent grid: the CTAs that are resident together (the registers of the instance decide)
-    static const int occ_vec = [] {
-        int n = 8;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, coo_reduce_kernel<T, N, true, false>, 256, 0) != cudaSuccess) n = 8;
-        return n < 1 ? 1 : n;
-    }();
-    static const int occ_plain = [] {
-        int n = 8;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, coo_reduce_kernel<T, N, false, false>, 256, 0) != cudaSuccess) n = 8;
-        return n < 1 ? 1 : n;
-    }();
+    static std::atomic<int> occ_vec[kMaxDevices], occ_plain[kMaxDevices];
+    const int occ = vec ? occupancy_cached(occ_vec, coo_reduce_kernel<T, N, true, false>, 256)
+                        : occupancy_cached(occ_plain, coo_reduce_kernel<T, N, false, false>, 256);
     auto grid_for = [&](int64_t chunks) {
         const int64_t want = (chunks + 7) / 8;   // 8 warps per CTA, one chunk per warp step
-        const int64_t cap = static_cast<int64_t>(sm_count) * (vec ? occ_vec : occ_plain);
+        const int64_t cap = static_cast<int64_t>(sm_count) * occ;
         return static_cast<unsigned>(want < cap ? (want > 0 ? want : 1) : cap);
     };
     CooArgs a;

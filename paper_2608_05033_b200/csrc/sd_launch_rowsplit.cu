@@ -6,7 +6,7 @@
 namespace sd {
 
 cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
-    if (a.N >= 1 && a.N <= 4 && !getenv("SD_NO_NARROW")) {   // one to four columns: lanes share a row, not its columns
+    if (a.N >= 1 && a.N <= 4 && !switches().no_narrow) {   // one to four columns: lanes share a row, not its columns
         if (dtype == SD_F32) return launch_rowsplit_narrow<float>(a, vec, st);
         return launch_rowsplit_narrow<__nv_bfloat16>(a, vec, st);
     }

@@ -20,9 +20,9 @@ namespace sd {
 constexpr size_t kStaticScratchBytes = 4u << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-static void *g_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device
-static bool g_scratch_ready[kMaxDevices];
+// device address of g_static_scratch, per device; published with release / acquire so that two host
+// threads making their first call on a device together both end up with the complete address
+static std::atomic<void *> g_scratch_addr[kMaxDevices];
 
 // In host code the name g_static_scratch is only a handle for the runtime, not an address a
 // kernel could use; the real device address has to be asked for, once per device, with that
@@ -34,13 +34,12 @@ static sd_status_t static_scratch(void **out) {
         set_error(SD_ERR_UNSUPPORTED, "device ordinal %d is beyond the %d this entry point tracks", dev, kMaxDevices);
         return SD_ERR_UNSUPPORTED;
     }
-    if (!g_scratch_ready[dev]) {
-        void *p = nullptr;
+    void *p = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!p) {
         SD_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
-        g_scratch_addr[dev] = p;
-        g_scratch_ready[dev] = true;
+        g_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = p;
     return SD_OK;
 }
 

@@ -155,13 +155,7 @@ cudaError_t launch_rowsplit_one(const SpmmArgs &a, cudaStream_t st) {
 struct LaneGeom {
     int vw, lpr, nv;
 };
-inline int geom_nv_override() {
-    static const int v = [] {
-        const char *e = getenv("SD_GEOM_NV");   // bench-only switch: 1 forces one vector per lane
-        return e ? atoi(e) : 0;
-    }();
-    return v;
-}
+inline int geom_nv_override() { return switches().geom_nv; }
 inline LaneGeom lane_geometry(int64_t N, bool vec, int vecw, bool prefer_two = true) {
     LaneGeom g;
     g.vw = vec ? vecw : 1;

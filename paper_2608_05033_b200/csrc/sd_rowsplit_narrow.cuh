@@ -187,13 +187,7 @@ rowsplit_ksplit_kernel(const SpmmArgs a) {
     if (gk == 0 && row < a.S) store_cols<VW>(a.C + row * a.ldc + lc * VW, acc, a.alpha, a.beta, 0);
 }
 
-inline int ksplit_override() {
-    static const int v = [] {
-        const char *e = getenv("SD_KSPLIT_G");   // measurement switch: lane sets per row (0: rule, 1: off)
-        return e ? atoi(e) : 0;
-    }();
-    return v;
-}
+inline int ksplit_override() { return switches().ksplit_g; }
 
 // Lane sets per row for the kernel above: 1 (= use the plain row-split kernel) unless rows are long.
 // Swept on uniform rows of 16 to 131 nonzeros at 8, 16 and 32 columns: about one set per eight nonzeros of
@@ -238,13 +232,7 @@ cudaError_t launch_rowsplit_ksplit(const SpmmArgs &a, int lpr, int g, cudaStream
     return cudaErrorInvalidValue;
 }
 
-inline int narrow_group_override() {
-    static const int v = [] {
-        const char *e = getenv("SD_NARROW_G");   // measurement switch: lanes per row (1..32, power of two)
-        return e ? atoi(e) : 0;
-    }();
-    return v;
-}
+inline int narrow_group_override() { return switches().narrow_g; }
 
 // Lanes per row from the mean row length: the largest power of two up to a quarter of it, 1..16
 // (measured on uniform rows of 5 to 128 nonzeros: each lane should keep about four to eight gathers of

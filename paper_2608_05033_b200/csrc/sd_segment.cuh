@@ -13,15 +13,6 @@ namespace sd {
 
 constexpr int kSegThreads = 256;
 
-inline int sm_count_cached() {
-    static const int n = [] {
-        int dev = 0, v = 148;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v;
-    }();
-    return n;
-}
-
 // SCRATCH: the segments are chunks; chunk c writes its plain sum to row c of a.C (the scratch
 // matrix).  Otherwise a.seg_row gives the output row and whether an earlier window wrote it.
 // Up to four lanes per row: six CTAs per SM (40 registers) measure 6 % faster; wider groups lose with that cap.
@@ -75,7 +66,8 @@ seg_kernel(const SpmmArgs a) {
                 }
 #pragma unroll
                 for (int i = 0; i < STEP; ++i) {
-                    if (colok[0]) {
+                    // entries beyond the chunk's end are not gathered: 0 * B[0, :] would turn a non-finite row 0 into NaN
+                    if (colok[0] && p + i < p1) {
                         RowLoad<T, VW>::ld(b_row(Bl, cq[i], a.ldb_bytes), b[i]);
                     } else {
 #pragma unroll
@@ -106,10 +98,9 @@ seg_kernel(const SpmmArgs a) {
                 float b[QU][NV][VW];
 #pragma unroll
                 for (int qq = 0; qq < QU; ++qq) {
-                    // chunks: an entry beyond the end has column 0 and value 0, so it may be gathered
-                    // unconditionally (only a segment's last chunk has such entries); short segments
-                    // would waste most of their gathers that way and keep the test
-                    const bool valid = SCRATCH || (p + q0 + qq < p1);
+                    // an entry beyond the end has column 0 and value 0; it is not gathered, so that a
+                    // non-finite row 0 of B cannot reach rows that never name column 0
+                    const bool valid = p + q0 + qq < p1;
                     const T *brow = b_row(Bl, cq[qq], a.ldb_bytes);
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
@@ -253,17 +244,10 @@ cudaError_t launch_seg_one(const SpmmArgs &a, bool scratch, cudaStream_t st) {
     const int64_t need = (a.S + per_cta - 1) / per_cta;
     // persistent grid: exactly the CTAs that are resident together (the registers of an instance decide how
     // many of the eight 256-thread CTAs an SM takes); a larger grid would run a thin second wave
-    static const int occ_scratch = [] {
-        int n = 8;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, seg_kernel<T, VW, LPR, NV, true>, kSegThreads, 0) != cudaSuccess) n = 8;
-        return n < 1 ? 1 : n;
-    }();
-    static const int occ_plain = [] {
-        int n = 8;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, seg_kernel<T, VW, LPR, NV, false>, kSegThreads, 0) != cudaSuccess) n = 8;
-        return n < 1 ? 1 : n;
-    }();
-    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * (scratch ? occ_scratch : occ_plain);
+    static std::atomic<int> occ_scratch[kMaxDevices], occ_plain[kMaxDevices];
+    const int occ = scratch ? occupancy_cached(occ_scratch, seg_kernel<T, VW, LPR, NV, true>, kSegThreads)
+                            : occupancy_cached(occ_plain, seg_kernel<T, VW, LPR, NV, false>, kSegThreads);
+    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * occ;
     dim3 grid(static_cast<unsigned>(need < cap ? need : cap),
               static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
     if (scratch) seg_kernel<T, VW, LPR, NV, true><<<grid, kSegThreads, 0, st>>>(a);
