@@ -117,8 +117,8 @@ def spmm(rowptr, colind, vals, B, N, Cin=None, alpha=1.0, beta=0.0, want_abs=Tru
     return Cref, S
 
 
-def spmm_rows(rows, rowptr, colind, vals, B, N, Cin=None, alpha=1.0, beta=0.0):
-    """O1 on selected rows: returns (Cref, S) as float64 [len(rows), N]."""
+def spmm_rows(rows, rowptr, colind, vals, B, N, Cin=None, alpha=1.0, beta=0.0, want_abs=True):
+    """O1 on selected rows: returns (Cref, S) as float64 [len(rows), N]; S is None unless want_abs."""
     rowptr, colind, vals, dt = _csr(rowptr, colind, vals)
     rows = np.ascontiguousarray(rows, dtype=np.int64)
     B, ldb = _dense(B, dt)
@@ -128,7 +128,7 @@ def spmm_rows(rows, rowptr, colind, vals, B, N, Cin=None, alpha=1.0, beta=0.0):
         assert Cin.dtype == np.float32 and Cin.strides[1] == 4
         ldcin = Cin.strides[0] // 4
     Cref = np.empty((rows.size, N), dtype=np.float64)
-    S = np.empty((rows.size, N), dtype=np.float64)
+    S = np.empty((rows.size, N), dtype=np.float64) if want_abs else None
     rc = lib().sdo_spmm_rows(C.c_int64(rows.size), _p(rows), C.c_int64(N), _p(rowptr), _p(colind),
                              _p(vals), C.c_int(dt), _p(B), C.c_int64(ldb),
                              _p(Cin) if beta != 0.0 else None, C.c_int64(ldcin),
