@@ -73,6 +73,11 @@ typedef struct {
                               -1 = one window, but with the class split of the window-major schedule */
     int32_t validate;      /* != 0: check rowptr monotone and 0 <= col < K on the device first */
     void *stream;          /* stream for the analysis kernels (plan creation still synchronises) */
+    int32_t test_wait_expiry; /* TEST ONLY, leave 0.  != 0: in the tensor-core kernel of an SD_BSR_TC plan the first CTA's
+                              copy thread never fills its ring, and every wait gives up after a few thousand polls
+                              instead of a million: the kernel must return by itself, sd_plan_device_status must
+                              report a non-zero code, C is left incomplete */
+    int32_t reserved0;
 } sd_plan_desc_t;
 
 /* Integer structure summary (Sec. 3.1 "Intrinsic pattern features", Eq. 4) and the
@@ -170,6 +175,24 @@ sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float
 sd_status_t sd_spmm_host_async(sd_plan_t *plan, const void *B_host, int64_t ldb, float *C_host,
                                int64_t ldc, float alpha, float beta);
 sd_status_t sd_plan_sync(sd_plan_t *plan);
+
+/* sd_plan_save / sd_plan_load -- keep the outcome of the analysis across processes (paper Sec. 3.4, last
+ * paragraph: the winning implementation is cached per sparsity pattern, operator, platform and dense width, so
+ * that later calls skip the search; here the "implementation" is the plan: family, schedule parameters and the
+ * structure-only representation -- tile tables, window-major segment lists, block lists).
+ * The blob is keyed by (hash of rowptr and colind, N, value type, device model): sd_plan_load recomputes the
+ * hash of the arrays it is given (one pass over them on the device, no sort) and refuses a blob made for
+ * another pattern (SD_ERR_INVALID_ARG) or another GPU model (SD_ERR_UNSUPPORTED).  Values are NOT in the
+ * blob: the loaded plan takes them from `vals` as sd_plan_update_values would, so a pattern whose weights
+ * changed since the save loads fine.
+ *   sd_plan_save   buf == NULL: only *bytes (the size needed) is set.  Else `cap` >= that size; host buffer.
+ *                  Synchronous (device-to-host copies).
+ *   sd_plan_load   blob: host.  rowptr / colind / vals: device, borrowed like at creation, dtype and shapes as
+ *                  saved.  *out receives a plan equivalent to the saved one: same sd_plan_get_info, same
+ *                  representation, bit-identical sd_spmm results. */
+sd_status_t sd_plan_save(const sd_plan_t *plan, void *buf, size_t cap, size_t *bytes);
+sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, const int32_t *colind,
+                         const void *vals, sd_plan_t **out);
 
 /* sd_plan_destroy -- the `cleanup` entry.  Frees everything the plan owns.  NULL is a no-op. */
 void sd_plan_destroy(sd_plan_t *plan);

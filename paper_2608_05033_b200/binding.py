@@ -21,7 +21,7 @@ SD_F32, SD_BF16 = 0, 1
 SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
 FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
 
-EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_destroy",
+EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_save", "sd_plan_load", "sd_plan_destroy",
            "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_last_error",
            "sd_version"]
 
@@ -30,7 +30,8 @@ class sd_plan_desc_t(C.Structure):
     _fields_ = [("rowptr", C.c_void_p), ("colind", C.c_void_p), ("vals", C.c_void_p),
                 ("M", C.c_int64), ("K", C.c_int64), ("N", C.c_int64),
                 ("dtype", C.c_int32), ("family", C.c_int32), ("windows", C.c_int32),
-                ("validate", C.c_int32), ("stream", C.c_void_p)]
+                ("validate", C.c_int32), ("stream", C.c_void_p), ("test_wait_expiry", C.c_int32),
+                ("reserved0", C.c_int32)]
 
 
 class sd_plan_info_t(C.Structure):
@@ -92,6 +93,10 @@ def load():
     lib.sd_plan_update_values.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_sync.restype = C.c_int
     lib.sd_plan_sync.argtypes = [C.c_void_p]
+    lib.sd_plan_save.restype = C.c_int
+    lib.sd_plan_save.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
+    lib.sd_plan_load.restype = C.c_int
+    lib.sd_plan_load.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_void_p)]
     lib.sd_plan_destroy.restype = None
     lib.sd_plan_destroy.argtypes = [C.c_void_p]
     lib.sd_plan_get_info.restype = C.c_int
@@ -161,9 +166,10 @@ def sd_plan_create(rowptr, colind, vals, M: int, K: int, N: int):
 
 
 def sd_plan_create_ex(rowptr, colind, vals, M: int, K: int, N: int, dtype: int = SD_F32,
-                      family: int = SD_AUTO, windows: int = 0, validate: bool = False, stream=None):
+                      family: int = SD_AUTO, windows: int = 0, validate: bool = False, stream=None,
+                      test_wait_expiry: int = 0):
     d = sd_plan_desc_t(_ptr(rowptr), _ptr(colind), _ptr(vals), M, K, N, dtype, family, windows,
-                       int(validate), _stream_handle(stream) if stream is not None else None)
+                       int(validate), _stream_handle(stream) if stream is not None else None, test_wait_expiry, 0)
     out = C.c_void_p()
     rc = load().sd_plan_create_ex(C.byref(d), C.byref(out))
     if rc != SD_OK:
@@ -209,6 +215,27 @@ def sd_spmm_merge_static(rowptr, colind, vals, M: int, K: int, N: int, nnz: int,
                                      ldc, alpha, beta, _stream_handle(stream))
     if rc != SD_OK:
         _raise(rc)
+
+
+def sd_plan_save(plan) -> bytes:
+    """The plan's key and structure-only representation as a host blob (see include/sd.h)."""
+    need = C.c_size_t(0)
+    rc = load().sd_plan_save(plan, None, 0, C.byref(need))
+    if rc != SD_OK:
+        _raise(rc)
+    buf = (C.c_ubyte * need.value)()
+    rc = load().sd_plan_save(plan, buf, need.value, C.byref(need))
+    if rc != SD_OK:
+        _raise(rc)
+    return bytes(buf)
+
+
+def sd_plan_load(blob: bytes, rowptr, colind, vals):
+    out = C.c_void_p()
+    rc = load().sd_plan_load(blob, len(blob), _ptr(rowptr), _ptr(colind), _ptr(vals), C.byref(out))
+    if rc != SD_OK:
+        _raise(rc)
+    return out.value
 
 
 def sd_plan_destroy(plan):
@@ -284,13 +311,14 @@ class Plan:
     """Owns an sd_plan_t and keeps the borrowed CSR tensors alive."""
 
     def __init__(self, rowptr, colind, vals, M: int, K: int, N: int, dtype: int | None = None,
-                 family: int = SD_AUTO, windows: int = 0, validate: bool = False):
+                 family: int = SD_AUTO, windows: int = 0, validate: bool = False, test_wait_expiry: int = 0):
         import torch
         if dtype is None:
             dtype = SD_F32 if vals.dtype == torch.float32 else SD_BF16
         self._keep = (rowptr, colind, vals)
         self.M, self.K, self.N, self.dtype = M, K, N, dtype
-        self.handle = sd_plan_create_ex(rowptr, colind, vals, M, K, N, dtype, family, windows, validate)
+        self.handle = sd_plan_create_ex(rowptr, colind, vals, M, K, N, dtype, family, windows, validate,
+                                        test_wait_expiry=test_wait_expiry)
 
     def spmm(self, B, Cmat, alpha: float = 1.0, beta: float = 0.0, stream=None):
         sd_spmm(self.handle, B, B.stride(0), Cmat, Cmat.stride(0), alpha, beta, stream)
@@ -316,6 +344,19 @@ class Plan:
         """New values for the same pattern; `vals` is borrowed from now on."""
         sd_plan_update_values(self.handle, vals, stream)
         self._keep = (self._keep[0], self._keep[1], vals)
+
+    def save(self) -> bytes:
+        return sd_plan_save(self.handle)
+
+    @classmethod
+    def load(cls, blob: bytes, rowptr, colind, vals):
+        """A plan from a blob made by save(); the CSR arrays are borrowed like at creation."""
+        self = cls.__new__(cls)
+        self._keep = (rowptr, colind, vals)
+        self.handle = sd_plan_load(blob, rowptr, colind, vals)
+        info = sd_plan_get_info(self.handle)
+        self.M, self.K, self.N, self.dtype = int(info.M), int(info.K), int(info.N), int(info.dtype)
+        return self
 
     def device_status(self) -> int:
         return sd_plan_device_status(self.handle)

@@ -469,6 +469,8 @@ struct sd_plan {
     int32_t bsr_nparts = 0;
     int32_t *dev_error = nullptr;
     int64_t nnzb = 0;
+    mutable sd::TcMapCache tc_map;   // descriptor of the last dense operand (sd_spmm takes the plan as const)
+    int32_t test_wait_expiry = 0;
 
     // host-buffer entry point
     void *stage_B = nullptr;
@@ -739,6 +741,8 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     return SD_OK;
 }
 
+static sd_status_t create_split_streams(sd_plan *p, int W);
+
 // `split`: the segments are re-bucketed by (window, class) and run through the chunk / segment / single
 // kernels; always so with W > 1, and with W = 1 when the class split alone pays (decide_class_split).
 static sd_status_t build_merge(sd_plan *p, int W, bool split, cudaStream_t st) {
@@ -815,16 +819,7 @@ static sd_status_t build_merge(sd_plan *p, int W, bool split, cudaStream_t st) {
                                            st));
     if ((s = tmp.get(tb, "select scratch"))) return s;
     int launches = 0;
-    if (split) {
-        for (int i = 0; i < 2; ++i) {
-            SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
-            SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
-        }
-        SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
-        SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
-        p->ev_chunk.assign(W, nullptr);
-        for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
-    }
+    if (split && (s = create_split_streams(p, W))) return s;
     if (split) {   // chunk ranges of the long segments
         std::vector<int32_t> cb(2 * W, 0);
         for (int w = 0; w < W; ++w) {
@@ -934,6 +929,7 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
     p->K = d->K;
     p->N = d->N;
     p->dtype = d->dtype;
+    p->test_wait_expiry = d->test_wait_expiry;
     SD_CUDA_TRY(cudaGetDevice(&p->device));
     cudaDeviceProp prop;
     SD_CUDA_TRY(cudaGetDeviceProperties(&prop, p->device));
@@ -1112,6 +1108,111 @@ static void free_plan(sd_plan *p) {
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- plan serialisation ---------------------------------------------------------------------------
+// Position-dependent 64-bit hash of an int32 array: the sum over i of mix(i, x[i]) (a sum, so the order in which
+// the threads add does not matter and the value is the same on every run and every grid size).
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__global__ void __launch_bounds__(256)
+hash_array_kernel(const int32_t *__restrict__ x, int64_t n, unsigned long long salt, unsigned long long *__restrict__ out) {
+    unsigned long long h = 0;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        h += mix64((static_cast<unsigned long long>(i) + 1) * 0x9E3779B97F4A7C15ull ^
+                   (static_cast<unsigned long long>(static_cast<uint32_t>(x[i])) + salt));
+    for (int off = 16; off > 0; off >>= 1) h += __shfl_xor_sync(0xffffffffu, h, off);
+    if ((threadIdx.x & 31) == 0 && h) atomicAdd(out, h);
+}
+
+// Hash of the sparsity pattern (rowptr and colind; the values are not part of it).
+static sd_status_t pattern_hash(const int32_t *rowptr, const int32_t *colind, int64_t M, int64_t nnz, cudaStream_t st,
+                                uint64_t *out) {
+    TempBuf acc;
+    sd_status_t s;
+    if ((s = acc.get(sizeof(unsigned long long), "pattern hash"))) return s;
+    SD_CUDA_TRY(cudaMemsetAsync(acc.p, 0, sizeof(unsigned long long), st));
+    auto *d = static_cast<unsigned long long *>(acc.p);
+    if (M >= 0 && rowptr) {
+        hash_array_kernel<<<static_cast<unsigned>(std::min<int64_t>((M + 256) / 256, 148 * 8)), 256, 0, st>>>(rowptr, M + 1, 0x51ull, d);
+        SD_CUDA_TRY(cudaGetLastError());
+    }
+    if (nnz > 0) {
+        hash_array_kernel<<<static_cast<unsigned>(std::min<int64_t>((nnz + 255) / 256, 148 * 8)), 256, 0, st>>>(colind, nnz, 0xC0ull, d);
+        SD_CUDA_TRY(cudaGetLastError());
+    }
+    unsigned long long h = 0;
+    SD_CUDA_TRY(cudaMemcpyAsync(&h, d, sizeof h, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    *out = h;
+    return SD_OK;
+}
+
+constexpr uint64_t kBlobMagic = 0x31304E414C504453ull;   // "SDPLAN01"
+constexpr uint32_t kBlobVersion = 1;
+constexpr int kBlobArrays = 13;
+
+struct BlobHeader {
+    uint64_t magic;
+    uint32_t version, header_bytes;
+    uint64_t pattern;           // pattern_hash of (rowptr, colind)
+    int64_t M, K, N, nnz;
+    int32_t dtype, family;
+    char device_name[128];      // the plan was tuned on this GPU model (grid sizes, window count, thresholds)
+    int32_t sm_count, nwins;
+    int64_t l2_bytes;
+    sd_plan_info_t info;
+    int64_t num_segments, num_chunks, ntiles, nnzb;
+    int32_t bsr_nparts, has_coo;
+    uint64_t array_bytes[kBlobArrays];   // payload sizes, in the order of blob_arrays(); each padded to 16 bytes in the blob
+};
+
+struct BlobArray {
+    void **field;
+    size_t bytes;
+    const char *what;
+};
+
+static size_t pad16(size_t b) { return (b + 15) & ~static_cast<size_t>(15); }
+
+// The structure-only device arrays of a plan, in blob order.  Value copies (re-bucketed values, 16x16 blocks and their
+// tensor-core images) and scratch are not part of the blob: they are rebuilt from the caller's values at load time.
+static void blob_arrays(sd_plan *p, BlobArray (&arr)[kBlobArrays]) {
+    const int64_t S = p->num_segments, nnz = p->nnz, W = static_cast<int64_t>(p->wins.size());
+    const bool merge = p->info.family == SD_MERGE && !p->wins.empty();
+    const bool split = merge && p->info.class_split;
+    const bool bsr = p->info.family == SD_BSR_TC;
+    const int64_t Mb = (p->M + 15) / 16;
+    auto set = [&](int i, void *field, size_t bytes, const char *what) { arr[i] = {static_cast<void **>(field), bytes, what}; };
+    set(0, &p->w_ptr, split ? 4 * (S + 1) : 0, "segment pointers");
+    set(1, &p->w_col, split ? 4 * nnz : 0, "window-major colind");
+    set(2, &p->w_src, split ? 4 * nnz : 0, "window-major source positions");
+    set(3, &p->w_seg_row, split ? 4 * (S + 1) : 0, "segment rows");
+    set(4, &p->seg_chunk, split ? 4 * (S + 1) : 0, "segment chunks");
+    set(5, &p->chunk_ptr, split ? 4 * (p->num_chunks + W + 1) : 0, "chunk boundaries");
+    set(6, &p->tile_seg, merge ? 4 * (p->ntiles + W) : 0, "tile table");
+    set(7, &p->fix_short, merge ? 4 * (p->ntiles + 1) : 0, "fix-up list");
+    set(8, &p->fix_long, merge ? 4 * (p->ntiles + 1) : 0, "fix-up list");
+    set(9, &p->coo_row, (merge && p->coo_row) ? 4 * nnz : 0, "row index per nonzero");
+    set(10, &p->browptr, bsr ? 4 * (Mb + 1) : 0, "browptr");
+    set(11, &p->bcol, bsr ? 4 * p->nnzb : 0, "bcol");
+    set(12, &p->bsr_part, (bsr && p->bsr_nparts > 0) ? 4 * (static_cast<int64_t>(p->bsr_nparts) + 1) : 0, "block-row partition");
+}
+
+static sd_status_t create_split_streams(sd_plan *p, int W) {
+    for (int i = 0; i < 2; ++i) {
+        SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
+        SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
+    }
+    SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+    SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
+    p->ev_chunk.assign(W, nullptr);
+    for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
+    return SD_OK;
+}
 
 }  // namespace sd
 
@@ -1557,6 +1658,8 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         b.N = static_cast<int32_t>(N);
         b.alpha = alpha;
         b.beta = beta;
+        b.map_cache = &plan->tc_map;
+        b.test_wait_expiry = plan->test_wait_expiry;
         const bool vec4 = aligned16(B) && aligned16(C) && N % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
                           (plan->dtype == SD_F32 || (reinterpret_cast<uintptr_t>(B) & 7u) == 0);
         if (bsr_tc_usable(b, plan->dtype) && !switches().bsr_simt)
@@ -1652,6 +1755,215 @@ sd_status_t sd_spmm_host(sd_plan_t *plan, const void *B_host, int64_t ldb, float
                          float beta) {
     const sd_status_t s = sd_spmm_host_async(plan, B_host, ldb, C_host, ldc, alpha, beta);
     return s ? s : sd_plan_sync(plan);
+}
+
+sd_status_t sd_plan_save(const sd_plan_t *plan, void *buf, size_t cap, size_t *bytes) {
+    if (!plan || !bytes) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_save: plan and bytes must not be null");
+        return SD_ERR_INVALID_ARG;
+    }
+    sd_plan *p = const_cast<sd_plan *>(plan);   // only read
+    BlobArray arr[kBlobArrays];
+    blob_arrays(p, arr);
+    const size_t nwins = p->wins.size();
+    size_t need = pad16(sizeof(BlobHeader)) + pad16(nwins * sizeof(sd_plan::Window));
+    for (const BlobArray &a : arr) need += pad16(a.bytes);
+    *bytes = need;
+    if (!buf) return SD_OK;   // size query
+    if (cap < need) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_save: the buffer holds %zu bytes, the plan needs %zu", cap, need);
+        return SD_ERR_INVALID_ARG;
+    }
+    int prev = 0;
+    SD_CUDA_TRY(cudaGetDevice(&prev));
+    SD_CUDA_TRY(cudaSetDevice(p->device));
+    BlobHeader h;
+    memset(&h, 0, sizeof h);
+    h.magic = kBlobMagic;
+    h.version = kBlobVersion;
+    h.header_bytes = static_cast<uint32_t>(sizeof(BlobHeader));
+    sd_status_t s = pattern_hash(p->rowptr, p->colind, p->M, p->nnz, nullptr, &h.pattern);
+    if (s == SD_OK) {
+        cudaDeviceProp prop;
+        cudaError_t e = cudaGetDeviceProperties(&prop, p->device);
+        if (e != cudaSuccess) s = cuda_fail(e, "cudaGetDeviceProperties");
+        else strncpy(h.device_name, prop.name, sizeof h.device_name - 1);
+    }
+    if (s != SD_OK) {
+        cudaSetDevice(prev);
+        return s;
+    }
+    h.M = p->M; h.K = p->K; h.N = p->N; h.nnz = p->nnz;
+    h.dtype = p->dtype;
+    h.family = p->info.family;
+    h.sm_count = p->info.sm_count;
+    h.nwins = static_cast<int32_t>(nwins);
+    h.l2_bytes = p->info.l2_bytes;
+    h.info = p->info;
+    h.num_segments = p->num_segments;
+    h.num_chunks = p->num_chunks;
+    h.ntiles = p->ntiles;
+    h.nnzb = p->nnzb;
+    h.bsr_nparts = p->bsr_nparts;
+    h.has_coo = p->coo_row ? 1 : 0;
+    for (int i = 0; i < kBlobArrays; ++i) h.array_bytes[i] = arr[i].bytes;
+    unsigned char *out = static_cast<unsigned char *>(buf);
+    memset(out, 0, need);
+    memcpy(out, &h, sizeof h);
+    size_t off = pad16(sizeof(BlobHeader));
+    if (nwins) memcpy(out + off, p->wins.data(), nwins * sizeof(sd_plan::Window));
+    off += pad16(nwins * sizeof(sd_plan::Window));
+    for (const BlobArray &a : arr) {
+        if (a.bytes) {
+            cudaError_t e = cudaMemcpy(out + off, *a.field, a.bytes, cudaMemcpyDeviceToHost);
+            if (e != cudaSuccess) {
+                cudaSetDevice(prev);
+                return cuda_fail(e, a.what);
+            }
+        }
+        off += pad16(a.bytes);
+    }
+    cudaSetDevice(prev);
+    return SD_OK;
+}
+
+sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, const int32_t *colind, const void *vals,
+                         sd_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!blob || !out || bytes < sizeof(BlobHeader)) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_load: null argument or a blob shorter than its header");
+        return SD_ERR_INVALID_ARG;
+    }
+    BlobHeader h;
+    memcpy(&h, blob, sizeof h);
+    if (h.magic != kBlobMagic || h.version != kBlobVersion || h.header_bytes != sizeof(BlobHeader) || h.nwins < 0 ||
+        h.M < 0 || h.nnz < 0 || (h.dtype != SD_F32 && h.dtype != SD_BF16)) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_load: not a plan blob of this library version");
+        return SD_ERR_INVALID_ARG;
+    }
+    size_t need = pad16(sizeof(BlobHeader)) + pad16(static_cast<size_t>(h.nwins) * sizeof(sd_plan::Window));
+    for (int i = 0; i < kBlobArrays; ++i) need += pad16(h.array_bytes[i]);
+    if (bytes < need) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_load: the blob is truncated (%zu of %zu bytes)", bytes, need);
+        return SD_ERR_INVALID_ARG;
+    }
+    if ((h.M > 0 && !rowptr) || (h.nnz > 0 && (!colind || !vals))) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_load: the CSR arrays the plan was made for must be given again");
+        return SD_ERR_INVALID_ARG;
+    }
+    // key: device model, then the pattern itself
+    int dev = 0;
+    SD_CUDA_TRY(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    SD_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (strncmp(prop.name, h.device_name, sizeof h.device_name) != 0 || prop.multiProcessorCount != h.sm_count ||
+        static_cast<int64_t>(prop.l2CacheSize) != h.l2_bytes) {
+        set_error(SD_ERR_UNSUPPORTED, "sd_plan_load: the plan was made on '%s' (%d SMs), this device is '%s' (%d SMs)",
+                  h.device_name, h.sm_count, prop.name, prop.multiProcessorCount);
+        return SD_ERR_UNSUPPORTED;
+    }
+    if (h.M > 0) {
+        int32_t last = 0;
+        SD_CUDA_TRY(cudaMemcpy(&last, rowptr + h.M, sizeof last, cudaMemcpyDeviceToHost));
+        if (last != h.nnz) {
+            set_error(SD_ERR_INVALID_ARG, "sd_plan_load: rowptr[M] = %d, the plan was made for %lld nonzeros", last,
+                      (long long)h.nnz);
+            return SD_ERR_INVALID_ARG;
+        }
+    }
+    uint64_t pat = 0;
+    sd_status_t s = pattern_hash(rowptr, colind, h.M, h.nnz, nullptr, &pat);
+    if (s != SD_OK) return s;
+    if (pat != h.pattern) {
+        set_error(SD_ERR_INVALID_ARG, "sd_plan_load: the sparsity pattern differs from the one the plan was made for");
+        return SD_ERR_INVALID_ARG;
+    }
+    sd_plan *p = new (std::nothrow) sd_plan;
+    if (!p) {
+        set_error(SD_ERR_ALLOC, "host allocation failed");
+        return SD_ERR_ALLOC;
+    }
+    auto fail = [&](sd_status_t code) {
+        free_plan(p);
+        return code;
+    };
+    p->rowptr = rowptr;
+    p->colind = colind;
+    p->vals = vals;
+    p->M = h.M; p->K = h.K; p->N = h.N; p->nnz = h.nnz;
+    p->dtype = h.dtype;
+    p->device = dev;
+    p->info = h.info;
+    p->num_segments = h.num_segments;
+    p->num_chunks = h.num_chunks;
+    p->ntiles = h.ntiles;
+    p->nnzb = h.nnzb;
+    p->bsr_nparts = h.bsr_nparts;
+    const unsigned char *in = static_cast<const unsigned char *>(blob);
+    size_t off = pad16(sizeof(BlobHeader));
+    p->wins.resize(h.nwins);
+    if (h.nwins) memcpy(p->wins.data(), in + off, static_cast<size_t>(h.nwins) * sizeof(sd_plan::Window));
+    off += pad16(static_cast<size_t>(h.nwins) * sizeof(sd_plan::Window));
+    // the array list depends on coo_row being set: mark it before sizing, allocate below
+    BlobArray arr[kBlobArrays];
+    if (h.has_coo) p->coo_row = reinterpret_cast<int32_t *>(1);
+    blob_arrays(p, arr);
+    p->coo_row = nullptr;
+    for (int i = 0; i < kBlobArrays; ++i) {
+        if (arr[i].bytes != h.array_bytes[i]) {
+            set_error(SD_ERR_INVALID_ARG, "sd_plan_load: the blob's array sizes do not fit its header");
+            return fail(SD_ERR_INVALID_ARG);
+        }
+        if (arr[i].bytes) {
+            if ((s = dev_alloc(p, arr[i].field, arr[i].bytes, arr[i].what))) return fail(s);
+            cudaError_t e = cudaMemcpy(*arr[i].field, in + off, arr[i].bytes, cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) return fail(cuda_fail(e, arr[i].what));
+        }
+        off += pad16(arr[i].bytes);
+    }
+    // scratch and value copies, as plan creation allocates them
+    const size_t es = p->dtype == SD_F32 ? 4 : 2;
+    if (p->info.family == SD_MERGE && !p->wins.empty()) {
+        const int W = static_cast<int>(p->wins.size());
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_head), sizeof(float) * p->ntiles * p->N, "tile heads"))) return fail(s);
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->tile_tail), sizeof(float) * p->ntiles * p->N, "tile tails"))) return fail(s);
+        if (p->info.class_split) {
+            if ((s = dev_alloc(p, &p->w_vals, es * p->nnz, "window-major values"))) return fail(s);
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * p->num_chunks * p->N, "chunk sums"))) return fail(s);
+            if ((s = create_split_streams(p, W))) return fail(s);
+            p->m_ptr = p->w_ptr;
+            p->m_col = p->w_col;
+            p->m_vals = p->w_vals;
+            p->m_seg_row = p->w_seg_row;
+        } else {
+            p->m_ptr = p->rowptr;
+            p->m_col = p->colind;
+            p->m_vals = p->vals;
+            p->m_seg_row = nullptr;
+        }
+        if (h.has_coo) {
+            const int cchunk = coo_chunk(static_cast<int>(p->N));
+            const int64_t chunks1 = (p->nnz + cchunk - 1) / cchunk, count2 = 2 * chunks1;
+            const int64_t chunks2 = (count2 + kCooCarryChunk - 1) / kCooCarryChunk, count3 = 2 * chunks2;
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_row), sizeof(int32_t) * count2, "carry rows"))) return fail(s);
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c1_val), sizeof(float) * count2 * p->N, "carry sums"))) return fail(s);
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_row), sizeof(int32_t) * count3, "carry rows (level 2)"))) return fail(s);
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_val), sizeof(float) * count3 * p->N, "carry sums (level 2)"))) return fail(s);
+        }
+    } else if (p->info.family == SD_BSR_TC) {
+        if ((s = dev_alloc(p, &p->bval, es * 256 * p->nnzb, "bval"))) return fail(s);
+        if ((s = dev_alloc(p, &p->bval_mma, (p->dtype == SD_BF16 ? 512 : 2048) * static_cast<size_t>(p->nnzb), "bval (tensor-core image)"))) return fail(s);
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->dev_error), sizeof(int32_t), "error word"))) return fail(s);
+        cudaError_t e = cudaMemset(p->dev_error, 0, sizeof(int32_t));
+        if (e != cudaSuccess) return fail(cuda_fail(e, "cudaMemset"));
+    }
+    // the value copies come from the values given now (the blob is keyed by the pattern only)
+    if ((s = sd_plan_update_values(p, vals, nullptr))) return fail(s);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceSynchronize"));
+    p->info = h.info;
+    *out = p;
+    return SD_OK;
 }
 
 #pragma GCC visibility pop

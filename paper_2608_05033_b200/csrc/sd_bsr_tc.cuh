@@ -68,6 +68,17 @@ __host__ __device__ constexpr int tc_stage_bytes(bool tf32, int sb) {
            ((sb * (tf32 ? kTcImgBytesTf32 : kTcImgBytesBf16) + 1023) / 1024) * 1024;
 }
 
+// The M = 64 / 128 instruction shapes read block-image rows that do not exist: 768 bytes (bf16: six more 8-row
+// cores of both k halves) or 1,536 bytes (fp32: twelve more per k step) past the end of a block's image.  For
+// every block but the last of the last ring slot that is the next image or the next slot; for that last one it
+// is what follows the ring in the dynamic allocation: the barrier words and the staged metadata (sized in
+// run_bsr_tc as 8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks + masks) bytes, plus at
+// least 1,025 bytes of alignment slack).  The products of those rows land in accumulator rows nobody reads.
+constexpr int kTcOverReadBf16 = 768, kTcOverReadTf32 = 1536;
+static_assert(8 * (3 * kTcMaxStages + 8) + 4 * (2 * kTcBatchItems + kTcBatchBlocks) >= kTcOverReadTf32 &&
+                  kTcOverReadTf32 >= kTcOverReadBf16,
+              "the operand over-read of the last block image must stay inside the kernel's own shared memory");
+
 struct TcArgs {
     const int32_t *browptr;
     const int32_t *bcol;
@@ -84,6 +95,8 @@ struct TcArgs {
     int32_t box_bytes;      // bytes one TMA box copy delivers
     int32_t stages;         // ring slots in use
     int32_t sb;             // blocks per ring slot
+    uint32_t spin_limit;    // polls before a wait gives up (kTcSpinLimit; a few thousand in the wait-expiry test)
+    int32_t withhold;       // test only: CTA 0's copy thread never fills its ring
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -112,8 +125,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false when the limit ran out or another warp already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error,
-                                          int code) {
-    for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
+                                          int code, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -214,8 +227,8 @@ __device__ __forceinline__ uint32_t ld_acquire(uint32_t addr) {
 }
 // Bounded wait until the counter at `addr` has reached `target`.
 __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, volatile int *abort_flag, int32_t *error,
-                                             int code) {
-    for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
+                                             int code, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (static_cast<int32_t>(ld_acquire(addr) - target) >= 0) return true;
         if (*abort_flag) return false;
     }
@@ -238,7 +251,8 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
     const int stage_bytes = tc_stage_bytes(TF32, a.sb);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + a.stages * stage_bytes);
     uint64_t *full = bars, *empty = bars + kTcMaxStages, *conv = bars + 2 * kTcMaxStages, *acc_full = bars + 3 * kTcMaxStages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * kTcMaxStages + 2);
+    uint64_t *drain = acc_full + 2;   // after an expired wait: the issuer's outstanding tensor-core work arrives here
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * kTcMaxStages + 3);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     uint32_t *epi_done = tmem_slot + 2;                                 // [2] rows whose accumulator each epilogue warp has read
     int32_t *meta_b0 = reinterpret_cast<int32_t *>(tmem_slot + 4);      // [kTcBatchItems + 1] block-row pointers
@@ -254,6 +268,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
             mbar_init(smem_u32(conv + s), kTcConvWarps);
         }
         for (int s = 0; s < 2; ++s) mbar_init(smem_u32(acc_full + s), 1);
+        mbar_init(smem_u32(drain), 1);
         epi_done[0] = 0;
         epi_done[1] = 0;
         *abort_flag = 0;
@@ -338,6 +353,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                 const uint32_t tx1 = static_cast<uint32_t>(a.box_bytes + kImgBytes);
                 uint32_t ahead = mbar_test_wait(empty0 + p_stage * 8, p_phase ^ 1);
                 for (int fb = 0; fb < total && ok; fb += sb) {
+                    if (a.withhold && blockIdx.x == 0) break;   // wait-expiry test: nothing is ever copied in
                     const int cnt = min(sb, total - fb);
                     uint32_t ns = p_stage + 1, np = p_phase;
                     if (ns == static_cast<uint32_t>(a.stages)) {
@@ -345,7 +361,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                         np ^= 1;
                     }
                     const uint32_t ahead_next = mbar_test_wait(empty0 + ns * 8, np ^ 1);   // a look at the next slot
-                    if (!ahead && !(ok = mbar_wait(empty0 + p_stage * 8, p_phase ^ 1, abort_flag, a.error, 1))) break;
+                    if (!ahead && !(ok = mbar_wait(empty0 + p_stage * 8, p_phase ^ 1, abort_flag, a.error, 1, a.spin_limit))) break;
                     ++p_issued;
                     uint32_t dst = ring0 + p_stage * stage_bytes;
                     const uint32_t fbar = full0 + p_stage * 8;
@@ -397,7 +413,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                         fm = si == 0 ? 1u : 0u;
                         lm = si == nstages - 1 ? 1u << (cnt - 1) : 0u;
                     }
-                    if (!ahead && !(ok = mbar_wait(wait0 + ms * 8, mp, abort_flag, a.error, 3))) break;
+                    if (!ahead && !(ok = mbar_wait(wait0 + ms * 8, mp, abort_flag, a.error, 3, a.spin_limit))) break;
                     tc_fence_after();
                     const uint32_t stage0 = ring0 + ms * stage_bytes;
                     uint64_t slab16 = static_cast<uint64_t>((stage0 & 0x3FFFFu) >> 4);
@@ -410,7 +426,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                             d0 = tmem_base + as * kTcSlabCols;
                             if (n >= 2) {
                                 for (int h = 0; h < nhalves && ok; ++h)
-                                    ok = counter_wait(done0 + h * 4, n - 1, abort_flag, a.error, 2);
+                                    ok = counter_wait(done0 + h * 4, n - 1, abort_flag, a.error, 2, a.spin_limit);
                                 if (!ok) break;
                                 tc_fence_after();
                             }
@@ -440,6 +456,13 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                     mp = np;
                     ahead = ahead_next;
                 }
+                if (!ok) {
+                    // a wait ran out: tensor-core instructions issued before it may still be reading shared memory and
+                    // writing TMEM; let them retire (bounded) before the CTA gives both back
+                    tc_commit(smem_u32(drain));
+                    for (uint32_t i = 0; i < 65536 && !mbar_try_wait(smem_u32(drain), 0); ++i) {
+                    }
+                }
             }
         } else if (warp == 0 || warp == 4) {
             // -------------------------------------------------------------- epilogue warps
@@ -456,7 +479,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                 const uint32_t as = n & 1u, aphase = (n >> 1) & 1u;
                 if (has_blocks) {
                     // one lane polls the barrier (spinning threads would crowd the barrier unit)
-                    if (lane == 0) ok = mbar_wait(smem_u32(acc_full + as), aphase, abort_flag, a.error, 4);
+                    if (lane == 0) ok = mbar_wait(smem_u32(acc_full + as), aphase, abort_flag, a.error, 4, a.spin_limit);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     if (!ok) break;
                     tc_fence_after();
@@ -505,7 +528,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
             uint32_t cs = m_stage, cp = m_phase;
             for (int fb = 0; fb < total && ok; fb += sb) {
                 const int cnt = min(sb, total - fb);
-                if (lane == 0) ok = mbar_wait(smem_u32(full + cs), cp, abort_flag, a.error, 5);
+                if (lane == 0) ok = mbar_wait(smem_u32(full + cs), cp, abort_flag, a.error, 5, a.spin_limit);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 uint8_t *sbp = smem + cs * stage_bytes;

@@ -67,6 +67,15 @@ cudaError_t run_coo(const CooPlan &cp, const SpmmArgs &s, int dtype, bool vec, i
 cudaError_t build_coo_rows(const int32_t *rowptr, int64_t M, int64_t nnz, int32_t *row, cudaStream_t st);
 
 // Family (c).
+// The TMA descriptor of B as the tensor-core kernel reads it, kept by the plan for the last (B, ldb) it ran with:
+// encoding one costs a driver call on the host, and a serving loop calls sd_spmm with the same operand buffer.
+struct alignas(64) TcMapCache {
+    unsigned char map[128];   // a CUtensorMap
+    const void *B = nullptr;
+    int64_t ldb = 0, K = 0;
+    int32_t N = 0;
+    int32_t valid = 0;
+};
 struct BsrArgs {
     const int32_t *browptr;  // [Mb + 1]
     const int32_t *bcol;     // [nnzb]
@@ -81,6 +90,8 @@ struct BsrArgs {
     int32_t Mb;
     int32_t N;
     float alpha, beta;
+    TcMapCache *map_cache;      // may be null: the descriptor is then encoded for this call only
+    int32_t test_wait_expiry;   // see sd_plan_desc_t
 };
 cudaError_t run_bsr_simt(const BsrArgs &a, int dtype, bool vec, cudaStream_t st);
 // Tensor-core form.  bsr_tc_usable: dtype, dense width and the TMA alignment rules allow it.

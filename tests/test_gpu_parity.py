@@ -720,3 +720,41 @@ def test_automatic_window_choice_matches_the_rule():
     ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
     assert info.windows == oracle.decide_windows(ref, oracle.F32, info.l2_bytes) == 1   # B fits in L2 here
     plan.close()
+
+
+def _without_column_zero(w, poison):
+    """The same matrix with every column index moved up by one (so column 0 is never referenced) and a new
+    row 0 of B holding `poison`."""
+    es = np.float32 if w.dtype == W.SD_F32 else np.uint16
+    row0 = np.full((1, w.N), poison, dtype=np.float32)
+    if w.dtype == W.SD_BF16:
+        row0 = W.f32_to_bf16_bits(row0).reshape(1, w.N)
+    B = np.concatenate([row0.astype(es), w.B], axis=0)
+    return W.Workload(w.name + "_no_col0", w.M, w.K + 1, w.N, w.rowptr, (w.colind + 1).astype(np.int32), w.vals, B,
+                      w.C0, w.alpha, w.beta, w.dtype, dict(w.meta))
+
+
+@pytest.mark.parametrize("poison", [np.inf, np.nan])
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+@pytest.mark.parametrize("N,windows", [(32, -1), (32, 4), (8, -1), (1, 1), (3, 1), (4, 1), (64, 1)])
+def test_non_finite_row_zero_of_b_stays_out_of_rows_that_do_not_name_it(poison, dtype, N, windows):
+    """Kernels that pad a batch of nonzeros with (column 0, value 0) must not let B[0, :] into the sum: with
+    B[0, :] = Inf or NaN and no entry in column 0, every result is finite and right.  Long segments of 129 to
+    255 nonzeros (a partly filled last chunk) under the class split and under column windows, and one to four
+    columns with a nonzero count that is not a multiple of the reduction's chunk."""
+    rng = np.random.default_rng(99 + N)
+    M, K = 700, 2600
+    lengths = rng.integers(0, 6, M)
+    lengths[rng.choice(M, 40, replace=False)] = rng.integers(129, 256, 40)
+    lengths[5] = 2047
+    w0 = W.random_csr(M, K, N, lengths, seed=321 + N, dtype=dtype)
+    assert w0.nnz % 256 != 0 and w0.nnz % 128 != 0
+    w = _without_column_zero(w0, poison)
+    dw = DeviceWorkload(w)
+    plan = dw.plan(family=sd.SD_MERGE, windows=windows)
+    got, intact = run_spmm(plan, w)
+    assert intact and np.all(np.isfinite(got))
+    # the oracle on the shifted matrix never touches row 0 of B either; compare with the original problem
+    r = oracle.check(w0.rowptr, w0.colind, w0.vals, w0.B, w0.N, got, None, w0.alpha, w0.beta)
+    assert r["ok"], r
+    plan.close()

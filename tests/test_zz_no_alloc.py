@@ -62,3 +62,45 @@ def test_static_scratch_entry_point_refuses_what_does_not_fit():
     assert e.value.code == sd.SD_ERR_UNSUPPORTED and "4194304" in str(e.value)
     torch.cuda.synchronize()
     assert float(Cm[0, 0]) == 3.0      # nothing was launched
+
+
+@pytest.mark.parametrize("N,offset", [(7, 0), (32, 1), (128, 0)])
+def test_static_scratch_entry_point_scalar_paths_empty_rows_and_scalars(N, offset):
+    """Dense widths and base pointers that force the scalar kernels, leading and trailing rows without
+    nonzeros, beta = 0 over a NaN-filled C, alpha = 0, and a small call after a larger one (the larger call's
+    leftovers beyond the small call's tiles must not matter)."""
+    import paper_2608_05033_b200 as sd
+
+    rng = np.random.default_rng(11 + N)
+    M, K = 900, 1500
+    lengths = rng.integers(0, 9, M)
+    lengths[:17] = 0
+    lengths[-9:] = 0
+    lengths[400] = 1400
+    w = W.random_csr(M, K, N, lengths, seed=55 + N)
+    big = W.g5_skewed(M=1 << 14, N=N, scale_c=2.4e7 / 256, cap=5000, seed=3)
+    rowptr, colind, vals = _dev(w.rowptr), _dev(w.colind), _dev(w.vals)
+
+    def run(ws, rp, ci, va, alpha, beta, cin):
+        Bh = np.zeros(ws.K * ws.N + offset + 4, dtype=np.float32)
+        Bh[offset:offset + ws.K * ws.N] = ws.B.reshape(-1)
+        Ch = np.zeros(ws.M * ws.N + offset + 4, dtype=np.float32)
+        Ch[offset:offset + ws.M * ws.N] = cin.reshape(-1)
+        Bd, Cd = _dev(Bh), _dev(Ch)
+        sd.sd_spmm_merge_static(rp, ci, va, ws.M, ws.K, ws.N, ws.nnz, Bd.data_ptr() + 4 * offset, ws.N,
+                                Cd.data_ptr() + 4 * offset, ws.N, alpha, beta)
+        torch.cuda.synchronize()
+        return Cd.cpu().numpy()[offset:offset + ws.M * ws.N].reshape(ws.M, ws.N)
+
+    # a larger problem first: it leaves more tiles' worth of carry rows in the shared array
+    cb = run(big, _dev(big.rowptr), _dev(big.colind), _dev(big.vals), 1.0, 0.0, np.zeros((big.M, big.N), np.float32))
+    assert oracle.check(big.rowptr, big.colind, big.vals, big.B, big.N, cb, None, 1.0, 0.0)["ok"]
+    nan_c = np.full((M, N), np.nan, np.float32)
+    got = run(w, rowptr, colind, vals, 1.5, 0.0, nan_c)                 # beta = 0 never reads C
+    assert oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, got, None, 1.5, 0.0)["ok"]
+    assert np.all(got[:17] == 0) and np.all(got[-9:] == 0)              # rows without nonzeros are written
+    cin = rng.standard_normal((M, N)).astype(np.float32)
+    got = run(w, rowptr, colind, vals, 0.0, 0.5, cin)                   # alpha = 0: C = beta * C
+    assert np.array_equal(got, np.float32(0.5) * cin)
+    got = run(w, rowptr, colind, vals, -0.75, 2.0, cin)
+    assert oracle.check(w.rowptr, w.colind, w.vals, w.B, w.N, got, cin, -0.75, 2.0)["ok"]
