@@ -629,6 +629,79 @@ def run_gcn_epoch(args, local_rank):
         "clocks": clocks, "per_width": rows}))
 
 
+def run_row_split(args, rank, local_rank, world):
+    """--split rows: ONE product (the GCN workload) over all ranks.  Rank k owns a contiguous range of rows of A and
+    C (balanced by rows + nonzeros) and an equal piece of the rows of B; every step gathers B into the rank's own
+    memory with one NCCL all-gather and then runs the rank's plan on it (no kernel reads a peer's memory).  Total
+    work is fixed: strong scaling.  At one rank the gather is a local copy."""
+    import torch
+    import torch.distributed as dist
+    import paper_2608_05033_b200 as sd
+    from paper_2608_05033_b200.shard import RowSplitSpmm, b_row_shard
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    sd.load()
+    kw = dict(SMALL_KW[2]) if args.small else {}
+    if args.width:
+        kw["N"] = args.width
+    w = W.config(2, dtype=W.SD_F32, **kw)            # every rank draws the same seeded matrix, keeps its share
+    rs = RowSplitSpmm(w.rowptr, w.colind, w.vals, w.M, w.K, w.N, w.dtype, dev)
+    k0, k1, per = b_row_shard(w.K, world, rank)
+    piece = np.zeros((per, w.N), dtype=np.float32)
+    piece[:k1 - k0] = w.B[k0:k1]
+    b_local = torch.from_numpy(piece).to(dev)
+    c_local = torch.zeros((rs.r1 - rs.r0, w.N), dtype=torch.float32, device=dev)
+    flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        flush.fill_(1.0)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        bf = None
+        from paper_2608_05033_b200.shard import gather_b
+        bf = gather_b(b_local, w.K, out=rs.b_full)
+        e1.record(stream)
+        if rs.r1 > rs.r0:
+            rs.plan.spmm(bf, c_local, w.alpha, w.beta, stream)
+        e2.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e2), e0.elapsed_time(e1)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ts = [step() for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    local_ms = float(np.mean([t[0] for t in ts]))
+    gather_ms = float(np.mean([t[1] for t in ts]))
+    ms = max_over_ranks(local_ms, dev)
+    gms = max_over_ranks(gather_ms, dev)
+    my_nnz = float(rs.plan.info().nnz)
+    if rank == 0:
+        print(json.dumps({
+            "mode": "split-rows", "metric": METRIC, "value": w.flops() / (ms * 1e-3) / 1e9, "unit": "GFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "all_gather_ms": gms, "higher_is_better": True, "scaling": "strong", "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{w.name}: one product split by rows over {world} rank(s), B row-sharded and "
+                                   "gathered into local memory every step (one all-gather), cold L2"},
+            "rank0_rows": [rs.r0, rs.r1], "rank0_nnz": my_nnz, "b_bytes_gathered_per_rank": int(world * per * w.N * 4),
+            "clocks": clocks}))
+    rs.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_probe_paths(args, local_rank):
     """Fetch paths for the gathers of the dense operand, timed on the GCN workload's own column stream
     (512-byte rows, storage order): plain loads with 4 / 8 / 16 gathers in flight per lane, L2 evict-last and
@@ -704,6 +777,9 @@ def main():
     ap.add_argument("--probe", action="store_true",
                     help="also replay every workload's colind stream as bare row gathers (sd_probe_gather) and "
                          "report its time beside the SpMM time: the gather ceiling of the memory system for that stream")
+    ap.add_argument("--split", default="", choices=["", "rows"],
+                    help="rows: one product (the GCN workload) split by rows over all ranks, B row-sharded and gathered "
+                         "into local memory with one all-gather per step (strong scaling; prints its own JSON line)")
     ap.add_argument("--probe-paths", action="store_true",
                     help="time the fetch paths of bench_probes on the GCN workload's column stream (prints its own JSON line)")
     ap.add_argument("--width", type=int, default=0,
@@ -732,6 +808,9 @@ def main():
     if args.probe_paths:
         if rank == 0:
             run_probe_paths(args, local_rank)
+        return
+    if args.split == "rows":
+        run_row_split(args, rank, local_rank, world)
         return
     run_gpu(args, rank, local_rank, world)
     if world > 1:

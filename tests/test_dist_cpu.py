@@ -130,3 +130,66 @@ def test_two_ranks_row_and_column_shards_reassemble_the_product():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert res == (True, True)
+
+
+# ---- row split with a row-sharded B: one all-gather into local memory, then the rank's own rows ----
+def test_b_row_shards_cover_every_row_once():
+    sys.path.insert(0, ROOT)
+    from paper_2608_05033_b200.shard import b_row_shard
+    for K, world in ((1000, 2), (1001, 4), (5, 8), (0, 3), (64, 1)):
+        pieces = [b_row_shard(K, world, r) for r in range(world)]
+        assert pieces[0][0] == 0 and pieces[-1][1] == K
+        for (a0, a1, per), (b0, b1, _) in zip(pieces, pieces[1:]):
+            assert a1 == b0 and a1 - a0 <= per
+        assert len({p[2] for p in pieces}) == 1 and pieces[0][2] * world >= K
+
+
+def _gather_worker(rank, world, port, out):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import oracle
+    import workloads as W
+    from paper_2608_05033_b200.shard import b_row_shard, gather_b, row_shard_bounds, row_shard_csr
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    w = W.g3_gcn_rmat(scale=10, N=12)                       # K = 1024 + an odd split below
+    K = w.K - 3                                             # make the last piece short: drop three rows / columns
+    keep = w.colind < K
+    lengths = np.add.reduceat(keep.astype(np.int64), w.rowptr[:-1]) * (np.diff(w.rowptr) > 0)
+    rowptr = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    colind, vals, B = w.colind[keep], w.vals[keep], np.ascontiguousarray(w.B[:K])
+    k0, k1, per = b_row_shard(K, world, rank)
+    piece = np.zeros((per, w.N), dtype=np.float32)          # this rank only ever sees its own rows of B
+    piece[:k1 - k0] = B[k0:k1]
+    piece[k1 - k0:] = np.nan                                # pad rows lie beyond K: they must never be read
+    b_full = gather_b(torch.from_numpy(piece), K).numpy()   # one collective, lands in this rank's memory
+    same_b = bool(np.array_equal(b_full, B))
+    bounds = row_shard_bounds(rowptr, world)
+    r0, r1 = int(bounds[rank]), int(bounds[rank + 1])
+    rp, cj, v = row_shard_csr(rowptr, colind, vals, r0, r1)
+    mine, _ = oracle.spmm(rp, cj, v, np.ascontiguousarray(b_full), w.N)
+    full = torch.zeros((w.M, w.N), dtype=torch.float64)
+    full[r0:r1] = torch.from_numpy(mine)
+    dist.all_reduce(full)                                   # test-side assembly only
+    flags = torch.tensor([1.0 if same_b else 0.0])
+    dist.all_reduce(flags, op=dist.ReduceOp.MIN)
+    if rank == 0:
+        ref, _ = oracle.spmm(rowptr, colind, vals, B, w.N)
+        out.put((bool(flags.item() == 1.0), bool(np.array_equal(full.numpy(), ref))))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_gather_row_sharded_b_then_compute_their_rows():
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = out.get(timeout=180)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == (True, True)

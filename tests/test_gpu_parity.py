@@ -758,3 +758,42 @@ def test_non_finite_row_zero_of_b_stays_out_of_rows_that_do_not_name_it(poison, 
     r = oracle.check(w0.rowptr, w0.colind, w0.vals, w0.B, w0.N, got, None, w0.alpha, w0.beta)
     assert r["ok"], r
     plan.close()
+
+
+@pytest.mark.parametrize("dtype", [W.SD_F32, W.SD_BF16])
+def test_row_split_with_row_sharded_b_gathers_into_local_memory_first(dtype):
+    """The row split whose dense operand is dealt out by rows: every rank's piece goes into the exchange layout
+    (equal, padded pieces), the gather lands them in one local buffer, and the rank's plan reads B from there.
+    One process here: the gather is the single-rank copy, and the pieces of a three-rank deal are put together
+    by hand the way all_gather_into_tensor lays them out, then every rank's rows are run in turn."""
+    from paper_2608_05033_b200.shard import RowSplitSpmm, b_row_shard, row_shard_bounds, row_shard_csr
+    from util import dev
+    w = W.config(2, scale=11, N=64, dtype=dtype)
+    K = w.K
+    # single rank through the class: B travels through the gather buffer
+    one = RowSplitSpmm(w.rowptr, w.colind, w.vals, w.M, K, w.N, dtype, "cuda")
+    assert (one.r0, one.r1, one.per) == (0, w.M, K)
+    Cd = torch.full((w.M, w.N), float("nan"), device="cuda")
+    one.run(dev(w.B), Cd)
+    torch.cuda.synchronize()
+    check(w, Cd.cpu().numpy())
+    one.close()
+    # three ranks' pieces laid out as the collective would, the last piece short
+    world = 3
+    per = b_row_shard(K, world, 0)[2]
+    full = np.full((world * per, w.N), 0x7FC0 if dtype == W.SD_BF16 else np.nan, dtype=w.B.dtype)
+    for rank in range(world):
+        k0, k1, _ = b_row_shard(K, world, rank)
+        full[rank * per:rank * per + (k1 - k0)] = w.B[k0:k1]
+    assert np.array_equal(full[:K], w.B)                      # consecutive pieces: the first K rows are B
+    Bd = dev(full)[:K]
+    Cd = torch.full((w.M, w.N), float("nan"), device="cuda")
+    b = row_shard_bounds(w.rowptr, world)
+    for rank in range(world):
+        r0, r1 = int(b[rank]), int(b[rank + 1])
+        rp, cj, v = row_shard_csr(w.rowptr, w.colind, w.vals, r0, r1)
+        plan = sd.Plan(dev(rp), dev(cj), dev(v), r1 - r0, K, w.N, dtype=dtype)
+        plan.spmm(Bd, Cd[r0:r1], 1.0, 0.0)
+        torch.cuda.synchronize()
+        plan.close()
+    check(w, Cd.cpu().numpy())
