@@ -629,6 +629,102 @@ def run_gcn_epoch(args, local_rank):
         "clocks": clocks, "per_width": rows}))
 
 
+# --------------------------------------------------------------------------- the decision rules against the clock
+def regret_rows(level: str, device_index: int = 0, log=None):
+    """The plan's fixed rules (family by block fill, class split by dense width, column windows) against measured
+    times (the paper ranks plans by measured runtime, Sec. 3.2-3.3; it prints no thresholds, so the clock on this
+    GPU is what the constants can be held to).  For every point each alternative is forced and timed (cold L2,
+    median), then the automatic plan; regret = automatic / fastest - 1.  `level`: "full" = the sweep behind the
+    committed table, "test" = a subset that a GPU test can afford."""
+    import torch
+    import paper_2608_05033_b200 as sd
+
+    dev = torch.device("cuda", device_index)
+    torch.cuda.set_device(dev)
+    sd.load()
+    flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).to(dev)
+
+    def median_ms(plan, Bd, Cd, w, reps):
+        ts = []
+        for i in range(reps + 3):
+            flush.fill_(1.0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            plan.spmm(Bd, Cd, w.alpha, w.beta, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    def point(rule, w, label, alternatives, reps):
+        """alternatives: {name: plan options}; the automatic plan is timed last."""
+        rowptr, colind, vals, Bd = to_dev(w.rowptr), to_dev(w.colind), to_dev(w.vals), to_dev(w.B)
+        Cd = torch.zeros((w.M, w.N), dtype=torch.float32, device=dev)
+        times = {}
+        for name, opts in alternatives.items():
+            plan = sd.Plan(rowptr, colind, vals, w.M, w.K, w.N, dtype=w.dtype, **opts)
+            times[name] = median_ms(plan, Bd, Cd, w, reps)
+            plan.close()
+        plan = sd.Plan(rowptr, colind, vals, w.M, w.K, w.N, dtype=w.dtype)
+        info = plan.info()
+        auto_ms = median_ms(plan, Bd, Cd, w, reps)
+        plan.close()
+        best = min(times.values())
+        row = {"rule": rule, "point": label, "dtype": "bf16" if w.dtype == W.SD_BF16 else "f32", "N": w.N, "nnz": w.nnz,
+               "ms": {k: round(v, 4) for k, v in times.items()}, "automatic_ms": round(auto_ms, 4),
+               "automatic": {"family": sd.FAMILY_NAMES[info.family], "windows": int(info.windows),
+                             "class_split": int(info.class_split)},
+               "regret": auto_ms / best - 1.0}
+        if log:
+            log(row)
+        return row
+
+    full = level == "full"
+    reps = 9 if full else 5
+    rows = []
+    # (A) 16x16 blocks on the tensor cores or CSR kernels: block fill x dense width x value type
+    fills = (1.0, 0.8, 0.5, 0.35, 0.2, 0.13) if full else (1.0, 0.5, 0.2)
+    widths = (64, 128, 256) if full else (64, 256)
+    for dt in (W.SD_F32, W.SD_BF16):
+        for N in widths:
+            base = W.g4_block(N=N, dtype=W.SD_F32)
+            for fill in fills:
+                w = W.thin_blocks(base, fill)
+                if dt == W.SD_BF16:
+                    w = W.Workload(w.name, w.M, w.K, w.N, w.rowptr, w.colind, W.f32_to_bf16_bits(w.vals),
+                                   W.f32_to_bf16_bits(w.B).reshape(w.B.shape), None, w.alpha, w.beta, W.SD_BF16, dict(w.meta))
+                rows.append(point("family: blocks on tensor cores vs CSR kernels", w, f"block fill {fill:g}",
+                                  {"bsr_tc": dict(family=sd.SD_BSR_TC), "rowsplit": dict(family=sd.SD_ROWSPLIT),
+                                   "merge": dict(family=sd.SD_MERGE)}, reps))
+    # (B) merge family: class split or merge-path tiles, by dense width
+    for dt in (W.SD_F32, W.SD_BF16):
+        for N in ((8, 16, 32, 64, 128) if full else (8, 32, 128)):
+            w = W.config(2, dtype=dt, N=N, **({} if full else dict(scale=18)))
+            rows.append(point("merge family: class split vs tiles", w, "R-MAT scale %d" % (20 if full else 18),
+                              {"tiles": dict(family=sd.SD_MERGE, windows=1), "class_split": dict(family=sd.SD_MERGE, windows=-1)},
+                              reps))
+    # (C) column windows of the skewed workload: none, the rule's count, twice that
+    w = W.config(4, **({} if full else dict(M=1 << 20, scale_c=2.4e7 / 4, cap=50000)))
+    rule_w = 8 if full else 2
+    rows.append(point("merge family: column windows", w, f"rank-size rows, M = {w.M}",
+                      {"tiles, no windows": dict(family=sd.SD_MERGE, windows=1),
+                       "class split, one window": dict(family=sd.SD_MERGE, windows=-1),
+                       f"{rule_w} windows": dict(family=sd.SD_MERGE, windows=rule_w),
+                       f"{2 * rule_w} windows": dict(family=sd.SD_MERGE, windows=2 * rule_w)}, reps))
+    return rows
+
+
+def run_regret(args, local_rank):
+    rows = regret_rows("test" if args.small else "full", local_rank, log=lambda r: print(json.dumps(r), file=sys.stderr, flush=True))
+    print(json.dumps({"mode": "regret", "level": "test" if args.small else "full", "worst_regret": max(r["regret"] for r in rows),
+                      "rows": rows}))
+
+
 def run_row_split(args, rank, local_rank, world):
     """--split rows: ONE product (the GCN workload) over all ranks.  Rank k owns a contiguous range of rows of A and
     C (balanced by rows + nonzeros) and an equal piece of the rows of B; every step gathers B into the rank's own
@@ -777,6 +873,10 @@ def main():
     ap.add_argument("--probe", action="store_true",
                     help="also replay every workload's colind stream as bare row gathers (sd_probe_gather) and "
                          "report its time beside the SpMM time: the gather ceiling of the memory system for that stream")
+    ap.add_argument("--regret", action="store_true",
+                    help="time every alternative of the plan's fixed rules (family by block fill, class split by width, "
+                         "column windows) against the automatic choice; prints its own JSON line (--small: the subset "
+                         "the GPU test runs)")
     ap.add_argument("--split", default="", choices=["", "rows"],
                     help="rows: one product (the GCN workload) split by rows over all ranks, B row-sharded and gathered "
                          "into local memory with one all-gather per step (strong scaling; prints its own JSON line)")
@@ -808,6 +908,10 @@ def main():
     if args.probe_paths:
         if rank == 0:
             run_probe_paths(args, local_rank)
+        return
+    if args.regret:
+        if rank == 0:
+            run_regret(args, local_rank)
         return
     if args.split == "rows":
         run_row_split(args, rank, local_rank, world)

@@ -484,12 +484,14 @@ int sdo_decide_windows(const sdo_info_t *o, int dtype, int64_t l2_bytes)
 /* Class split at one window (this build's rule, parity unpinned): the window-major schedule
  * (long segments cut into chunks, short ones one lane group each, one-nonzero rows flat) without
  * column windows, taken by merge-family plans whose rows are sorted when the dense width is
- * 16 to 64 columns (fp32 values) or 16 to 32 columns (bf16 values); measured on the target GPU
- * against the merge-path tiles, which stay ahead or level at 8 columns and beyond those widths. */
+ * 16 to 64 columns (fp32 values) or 8 to 32 columns (bf16 values); measured on the target GPU
+ * against the merge-path tiles (the sweep of `bench.py --regret`), which stay ahead or level at
+ * 8 fp32 columns and beyond those widths. */
 int sdo_decide_class_split(const sdo_info_t *o, int dtype)
 {
     int64_t widest = dtype == SDO_BF16 ? 32 : 64;
-    return o->unsorted_rows == 0 && o->nnz > 0 && o->N >= 16 && o->N <= widest;
+    int64_t narrowest = dtype == SDO_BF16 ? 8 : 16;
+    return o->unsorted_rows == 0 && o->nnz > 0 && o->N >= narrowest && o->N <= widest;
 }
 
 /* Window-major segment list.  Window of a column: col / ceil(K / W).  A segment is the part

@@ -563,12 +563,13 @@ static int decide_windows(const sd_plan_info_t &s, int dtype) {
 
 // One window, but still the class split (long segments as chunks, short ones one lane group each,
 // one-nonzero rows flat) instead of merge-path tiles: measured on R-MAT and rank-size matrices, the split
-// is ahead from 16 columns up to 64 fp32 / 32 bf16 columns (0.68 to 0.94 of the tile kernel's time) and
-// behind or level at 8 columns and beyond (bf16 at 128 columns: 1.27).  Needs ascending columns like the
-// windows.
+// is ahead from 16 fp32 / 8 bf16 columns up to 64 fp32 / 32 bf16 columns (0.68 to 0.94 of the tile kernel's
+// time; 0.80 at 8 bf16 columns) and behind or level at 8 fp32 columns and beyond those widths (the sweep of
+// `bench.py --regret`).  Needs ascending columns like the windows.
 static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
     const int64_t widest = dtype == SD_BF16 ? 32 : 64;
-    return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= 16 && s.N <= widest;
+    const int64_t narrowest = dtype == SD_BF16 ? 8 : 16;
+    return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= narrowest && s.N <= widest;
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {

@@ -534,7 +534,7 @@ def test_o4_class_split_rule_by_dense_width():
     info.nnz = 32 << 20
     for dt, N, want in ((oracle.F32, 8, False), (oracle.F32, 15, False), (oracle.F32, 16, True), (oracle.F32, 24, True),
                         (oracle.F32, 32, True), (oracle.F32, 33, True), (oracle.F32, 64, True), (oracle.F32, 65, False),
-                        (oracle.F32, 128, False), (oracle.BF16, 8, False), (oracle.BF16, 16, True), (oracle.BF16, 32, True),
+                        (oracle.F32, 128, False), (oracle.BF16, 7, False), (oracle.BF16, 8, True), (oracle.BF16, 16, True), (oracle.BF16, 32, True),
                         (oracle.BF16, 33, False), (oracle.BF16, 64, False)):
         info.N = N
         assert oracle.decide_class_split(info, dt) == want, (dt, N)

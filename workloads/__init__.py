@@ -243,6 +243,19 @@ def g4_block(Mb: int = 4096, Kb: int = 4096, N: int = 256, nblocks: int | None =
     return _maybe_bf16(w, dtype)
 
 
+def thin_blocks(w: Workload, fill: float, seed: int = SEED_BASE + 44) -> Workload:
+    """The block workload with every stored entry kept with probability `fill` (partly filled 16x16 blocks; the
+    occupied blocks stay the same unless a block loses all of its entries).  Values and B are those of `w`."""
+    if fill >= 1.0:
+        return w
+    rng = np.random.Generator(np.random.PCG64(seed))
+    keep = rng.random(w.nnz) < fill
+    rows = np.repeat(np.arange(w.M, dtype=np.int64), np.diff(w.rowptr))
+    lengths = np.bincount(rows[keep], minlength=w.M).astype(np.int64)
+    return Workload(f"{w.name}_fill{fill:g}", w.M, w.K, w.N, _rowptr_from_lengths(lengths), w.colind[keep], w.vals[keep],
+                    w.B, None, w.alpha, w.beta, w.dtype, {"generator": "G4 thinned", "fill": fill, "seed": seed})
+
+
 # --------------------------------------------------------------------------
 # config 5: skewed rank-size row lengths
 # --------------------------------------------------------------------------
