@@ -57,7 +57,11 @@ typedef enum {
     SD_AUTO = 0,     /* decide from the structure summary */
     SD_ROWSPLIT = 1, /* sub-warp per row, vectorised gathers of B rows */
     SD_MERGE = 2,    /* merge-path split of (row ends + nonzeros), segmented reduction,
-                        deterministic carry-out fix-up */
+                        deterministic carry-out fix-up.  There is no separate "hybrid" family (light rows
+                        row-wise, heavy rows in chunks, as in the paper's appendix listing): that schedule
+                        is this family's class split (sd_plan_info_t.class_split; long segments as
+                        128-nonzero chunks, short ones one lane group each, one-nonzero rows flat),
+                        chosen by dense width and forced with windows = -1 */
     SD_BSR_TC = 3    /* 16x16 blocks on the tensor cores (tcgen05 / TMEM / TMA) */
 } sd_family_t;
 
