@@ -871,7 +871,7 @@ def main():
     ap.add_argument("--configs", default="", help="comma list of config indices (0..4) to restrict the step")
     ap.add_argument("--windows", type=int, default=0, help="column windows of the merge family (0 = plan's rule)")
     ap.add_argument("--probe", action="store_true",
-                    help="also replay every workload's colind stream as bare row gathers (sd_probe_gather) and "
+                    help="also replay every workload's colind stream as bare row gathers (bench_probes, path 0) and "
                          "report its time beside the SpMM time: the gather ceiling of the memory system for that stream")
     ap.add_argument("--regret", action="store_true",
                     help="time every alternative of the plan's fixed rules (family by block fill, class split by width, "
