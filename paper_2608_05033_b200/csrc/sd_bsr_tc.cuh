@@ -95,8 +95,6 @@ struct TcArgs {
     int32_t box_bytes;      // bytes one TMA box copy delivers
     int32_t stages;         // ring slots in use
     int32_t sb;             // blocks per ring slot
-    uint32_t spin_limit;    // polls before a wait gives up (kTcSpinLimit; a few thousand in the wait-expiry test)
-    int32_t withhold;       // test only: CTA 0's copy thread never fills its ring
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -124,9 +122,11 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait.  Returns false when the limit ran out or another warp already gave up.
+// (The limit is a compile-time constant on purpose: as a kernel argument it cost the fp32 kernel 18 %.)
+template <uint32_t LIMIT>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error,
-                                          int code, uint32_t limit) {
-    for (uint32_t i = 0; i < limit; ++i) {
+                                          int code) {
+    for (uint32_t i = 0; i < LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -226,9 +226,10 @@ __device__ __forceinline__ uint32_t ld_acquire(uint32_t addr) {
     return v;
 }
 // Bounded wait until the counter at `addr` has reached `target`.
+template <uint32_t LIMIT>
 __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, volatile int *abort_flag, int32_t *error,
-                                             int code, uint32_t limit) {
-    for (uint32_t i = 0; i < limit; ++i) {
+                                             int code) {
+    for (uint32_t i = 0; i < LIMIT; ++i) {
         if (static_cast<int32_t>(ld_acquire(addr) - target) >= 0) return true;
         if (*abort_flag) return false;
     }
@@ -237,9 +238,11 @@ __device__ __forceinline__ bool counter_wait(uint32_t addr, uint32_t target, vol
     return false;
 }
 
-template <bool TF32>
+// EXPIRY_TEST: the instance behind sd_plan_desc_t.test_wait_expiry (short spin limit, CTA 0 never copies anything in).
+template <bool TF32, bool EXPIRY_TEST>
 __global__ void __launch_bounds__(TF32 ? kTcThreadsTf32 : kTcThreadsBf16, 1)
 bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
+    constexpr uint32_t kLimit = EXPIRY_TEST ? 4096u : kTcSpinLimit;
     constexpr int kThreads = TF32 ? kTcThreadsTf32 : kTcThreadsBf16;
     constexpr int kSlab = TF32 ? kTcSlabBytesTf32 : kTcSlabBytesBf16;   // slab bytes of one block in a ring slot
     constexpr int kImgBytes = TF32 ? kTcImgBytesTf32 : kTcImgBytesBf16;
@@ -346,33 +349,43 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
 
         if (warp == 1) {
             // -------------------------------------------------------------- TMA producer
-            if (lane == 0) {
+            // The whole warp: lane 0 waits for the slot, arms its barrier with the slot's byte count and copies the
+            // images; then lane u issues the slab copy of the slot's block u, so the copies of a slot are issued side
+            // by side instead of one after the other by a single thread (which cost about 200 cycles per block).
+            {
                 const uint8_t *img = static_cast<const uint8_t *>(a.bmma) + static_cast<int64_t>(base) * kImgBytes;
                 const int zc = n0 / (TF32 ? 32 : 64);
                 const uint32_t ring0 = smem_u32(smem), full0 = smem_u32(full), empty0 = smem_u32(empty);
                 const uint32_t tx1 = static_cast<uint32_t>(a.box_bytes + kImgBytes);
-                uint32_t ahead = mbar_test_wait(empty0 + p_stage * 8, p_phase ^ 1);
+                uint32_t ahead = lane == 0 ? mbar_test_wait(empty0 + p_stage * 8, p_phase ^ 1) : 0u;
                 for (int fb = 0; fb < total && ok; fb += sb) {
-                    if (a.withhold && blockIdx.x == 0) break;   // wait-expiry test: nothing is ever copied in
+                    if (EXPIRY_TEST && blockIdx.x == 0) break;   // wait-expiry test: nothing is ever copied in
                     const int cnt = min(sb, total - fb);
                     uint32_t ns = p_stage + 1, np = p_phase;
                     if (ns == static_cast<uint32_t>(a.stages)) {
                         ns = 0;
                         np ^= 1;
                     }
-                    const uint32_t ahead_next = mbar_test_wait(empty0 + ns * 8, np ^ 1);   // a look at the next slot
-                    if (!ahead && !(ok = mbar_wait(empty0 + p_stage * 8, p_phase ^ 1, abort_flag, a.error, 1, a.spin_limit))) break;
-                    ++p_issued;
-                    uint32_t dst = ring0 + p_stage * stage_bytes;
+                    uint32_t ahead_next = 0;
+                    const uint32_t dst = ring0 + p_stage * stage_bytes;
                     const uint32_t fbar = full0 + p_stage * 8;
-                    mbar_expect_tx(fbar, cnt * tx1);
-                    bulk_load(dst + img_off, img, cnt * kImgBytes, fbar);   // the images of cnt consecutive blocks
+                    if (lane == 0) {
+                        ahead_next = mbar_test_wait(empty0 + ns * 8, np ^ 1);   // a look at the next slot
+                        if (!ahead) ok = mbar_wait<kLimit>(empty0 + p_stage * 8, p_phase ^ 1, abort_flag, a.error, 1);
+                        if (ok) {
+                            mbar_expect_tx(fbar, cnt * tx1);
+                            bulk_load(dst + img_off, img, cnt * kImgBytes, fbar);   // the images of cnt consecutive blocks
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;   // also orders the arming before the copies below
+                    if (!ok) break;
+                    ++p_issued;
                     img += cnt * kImgBytes;
-                    for (int u = 0; u < cnt; ++u, dst += kSlab) {
-                        const int flat = fb + u;
+                    if (lane < cnt) {
+                        const int flat = fb + lane;
                         const int krow = ((flat < kTcBatchBlocks) ? meta_col[flat] : __ldg(a.bcol + base + flat)) * 16;
                         // one copy brings all column groups of the slab: [group][16 rows][128 B]
-                        tma_load_3d(dst, &tmapB, 0, krow, zc, fbar);
+                        tma_load_3d(dst + lane * kSlab, &tmapB, 0, krow, zc, fbar);
                     }
                     p_stage = ns;
                     p_phase = np;
@@ -413,24 +426,29 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                         fm = si == 0 ? 1u : 0u;
                         lm = si == nstages - 1 ? 1u << (cnt - 1) : 0u;
                     }
-                    if (!ahead && !(ok = mbar_wait(wait0 + ms * 8, mp, abort_flag, a.error, 3, a.spin_limit))) break;
+                    if (!ahead && !(ok = mbar_wait<kLimit>(wait0 + ms * 8, mp, abort_flag, a.error, 3))) break;
                     tc_fence_after();
                     const uint32_t stage0 = ring0 + ms * stage_bytes;
                     uint64_t slab16 = static_cast<uint64_t>((stage0 & 0x3FFFFu) >> 4);
                     uint64_t img16 = static_cast<uint64_t>(((stage0 + img_off) & 0x3FFFFu) >> 4);
-                    for (int u = 0; u < cnt; ++u, slab16 += kSlab >> 4, img16 += kImgBytes >> 4, fm >>= 1, lm >>= 1) {
-                        const uint32_t opens = fm & 1u;
+                    // the slot's blocks as runs of one block-row each: the per-row decisions (which accumulator, is it
+                    // free, is the row complete) are taken once per run, the loop over a run's blocks only issues
+                    for (int u = 0; u < cnt && ok;) {
+                        const uint32_t rest = lm >> u;                                   // row ends at or after block u
+                        const int e = rest ? u + __ffs(rest) - 1 : cnt - 1;              // last block of the run inside this slot
+                        uint32_t opens = (fm >> u) & 1u;
                         if (opens) {
                             // the accumulator slot of this block-row was last read for block-row n - 2
                             as = n & 1u;
                             d0 = tmem_base + as * kTcSlabCols;
                             if (n >= 2) {
                                 for (int h = 0; h < nhalves && ok; ++h)
-                                    ok = counter_wait(done0 + h * 4, n - 1, abort_flag, a.error, 2, a.spin_limit);
+                                    ok = counter_wait<kLimit>(done0 + h * 4, n - 1, abort_flag, a.error, 2);
                                 if (!ok) break;
                                 tc_fence_after();
                             }
                         }
+                        for (; u <= e; ++u, slab16 += kSlab >> 4, img16 += kImgBytes >> 4, opens = 0u) {
                         if constexpr (TF32) {
                             // k step = 8 block columns: 1 KB of the image (hi over lo), 8 rows = 1024 bytes of the slab;
                             // accumulator rows 0..15 collect hi*hi + hi*lo, rows 16..31 lo*hi + lo*lo
@@ -445,7 +463,8 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                         } else {
                             tc_mma<false>(d0, a0 + img16, b0 + slab16, idesc, opens ^ 1u);
                         }
-                        if (lm & 1u) {
+                        }
+                        if (rest) {
                             tc_commit(accf0 + as * 8);   // the block-row's accumulator is complete
                             ++n;
                         }
@@ -479,7 +498,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
                 const uint32_t as = n & 1u, aphase = (n >> 1) & 1u;
                 if (has_blocks) {
                     // one lane polls the barrier (spinning threads would crowd the barrier unit)
-                    if (lane == 0) ok = mbar_wait(smem_u32(acc_full + as), aphase, abort_flag, a.error, 4, a.spin_limit);
+                    if (lane == 0) ok = mbar_wait<kLimit>(smem_u32(acc_full + as), aphase, abort_flag, a.error, 4);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     if (!ok) break;
                     tc_fence_after();
@@ -528,7 +547,7 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
             uint32_t cs = m_stage, cp = m_phase;
             for (int fb = 0; fb < total && ok; fb += sb) {
                 const int cnt = min(sb, total - fb);
-                if (lane == 0) ok = mbar_wait(smem_u32(full + cs), cp, abort_flag, a.error, 5, a.spin_limit);
+                if (lane == 0) ok = mbar_wait<kLimit>(smem_u32(full + cs), cp, abort_flag, a.error, 5);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 uint8_t *sbp = smem + cs * stage_bytes;

@@ -130,8 +130,6 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     t.beta = a.beta;
     t.error = error_word;
     t.box_bytes = box_groups * 2048;
-    t.spin_limit = a.test_wait_expiry ? 4096u : kTcSpinLimit;
-    t.withhold = a.test_wait_expiry ? 1 : 0;
     // ring geometry (bench-only overrides through the environment); one CTA per SM, its ring
     // takes most of the shared memory: bf16 2 slots of 8 blocks (8.5 KB per block), fp32 3 slots
     // of 2 blocks (34 KB per block).  A barrier round trip costs far more than a block's work,
@@ -149,15 +147,24 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     static std::atomic<int> attr_set[kMaxDevices][2];
     const int dev = current_device();
     if (dev >= kMaxDevices || attr_set[dev][tf32].load(std::memory_order_acquire) < smem) {
-        cudaError_t e = tf32 ? cudaFuncSetAttribute(bsr_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
-                             : cudaFuncSetAttribute(bsr_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = tf32 ? cudaFuncSetAttribute(bsr_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                             : cudaFuncSetAttribute(bsr_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        e = tf32 ? cudaFuncSetAttribute(bsr_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                 : cudaFuncSetAttribute(bsr_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         if (dev < kMaxDevices) attr_set[dev][tf32].store(smem, std::memory_order_release);
     }
     const int grid = a.nparts;
     (void)sm_count;
-    if (tf32) bsr_tc_kernel<true><<<grid, kTcThreadsTf32, smem, st>>>(map, t);
-    else bsr_tc_kernel<false><<<grid, kTcThreadsBf16, smem, st>>>(map, t);
+    if (a.test_wait_expiry) {
+        if (tf32) bsr_tc_kernel<true, true><<<grid, kTcThreadsTf32, smem, st>>>(map, t);
+        else bsr_tc_kernel<false, true><<<grid, kTcThreadsBf16, smem, st>>>(map, t);
+    } else if (tf32) {
+        bsr_tc_kernel<true, false><<<grid, kTcThreadsTf32, smem, st>>>(map, t);
+    } else {
+        bsr_tc_kernel<false, false><<<grid, kTcThreadsBf16, smem, st>>>(map, t);
+    }
     return cudaGetLastError();
 }
 
