@@ -95,6 +95,7 @@ struct TcArgs {
     int32_t box_bytes;      // bytes one TMA box copy delivers
     int32_t stages;         // ring slots in use
     int32_t sb;             // blocks per ring slot
+    int32_t wide_store;     // C and ldc allow 32-byte stores
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -523,7 +524,19 @@ bsr_tc_kernel(const __grid_constant__ CUtensorMap tmapB, const TcArgs a) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = 0.f;
                     }
-                    if (mine) {
+                    if (mine && a.wide_store && a.beta == 0.f) {
+                        // 32-byte stores: every instruction fills whole 32-byte sectors of 16 different rows (the 16-byte
+                        // form writes half sectors, twice as many instructions and L2 write requests for the same bytes)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            float *p = crow + c0 + 8 * q;
+                            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p),
+                                         "f"(a.alpha * r[8 * q]), "f"(a.alpha * r[8 * q + 1]), "f"(a.alpha * r[8 * q + 2]),
+                                         "f"(a.alpha * r[8 * q + 3]), "f"(a.alpha * r[8 * q + 4]), "f"(a.alpha * r[8 * q + 5]),
+                                         "f"(a.alpha * r[8 * q + 6]), "f"(a.alpha * r[8 * q + 7])
+                                         : "memory");
+                        }
+                    } else if (mine) {
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
                             float4 *p = reinterpret_cast<float4 *>(crow + c0) + q;

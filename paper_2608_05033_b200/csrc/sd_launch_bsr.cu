@@ -130,13 +130,14 @@ cudaError_t run_bsr_tc(const BsrArgs &a, int dtype, int32_t *error_word, int sm_
     t.beta = a.beta;
     t.error = error_word;
     t.box_bytes = box_groups * 2048;
+    t.wide_store = ((reinterpret_cast<uintptr_t>(a.C) & 31u) == 0 && a.ldc % 8 == 0) ? 1 : 0;
     // ring geometry (bench-only overrides through the environment); one CTA per SM, its ring
-    // takes most of the shared memory: bf16 2 slots of 8 blocks (8.5 KB per block), fp32 3 slots
+    // takes most of the shared memory: bf16 3 slots of 8 blocks (8.5 KB per block), fp32 3 slots
     // of 2 blocks (34 KB per block).  A barrier round trip costs far more than a block's work,
     // so slots hold several blocks.
     const Switches &sw = switches();
     t.sb = tf32 ? (sw.tc32_sb ? sw.tc32_sb : 2) : (sw.tc_sb ? sw.tc_sb : 8);
-    t.stages = tf32 ? (sw.tc32_stages ? sw.tc32_stages : 3) : (sw.tc_stages ? sw.tc_stages : 2);
+    t.stages = tf32 ? (sw.tc32_stages ? sw.tc32_stages : 3) : (sw.tc_stages ? sw.tc_stages : 3);
     if (t.sb < 1) t.sb = 1;
     if (t.sb > 32) t.sb = 32;   // one mask bit per block of a ring slot
     if (t.stages < 1) t.stages = 1;
