@@ -6,6 +6,8 @@
 // warp may run different trip counts, and the grid-stride loops need no warp-wide agreement.
 #pragma once
 
+#include <type_traits>
+
 #include "sd_common.cuh"
 #include "sd_rowsplit.cuh"
 
@@ -44,18 +46,23 @@ seg_kernel(const SpmmArgs a) {
         for (int v = 0; v < NV; ++v)
 #pragma unroll
             for (int e = 0; e < VW; ++e) acc[v][e] = 0.f;
+        // A step takes LPR (or 2 LPR) nonzeros.  Whole steps run without any test; only a segment's last, partly
+        // filled step tests every entry: its entries beyond the end have column 0 and value 0, and neither their
+        // gather nor their product may happen, or a non-finite row 0 of B would reach rows that never name
+        // column 0 (0 * Inf is NaN).
         if constexpr (SCRATCH && LPR <= 2 && NV * VW < 8) {
             // chunks with one or two lanes per row: a lane fetches two (column, value) pairs per step, so that twice
             // as many gathers are in flight per lane (skewed matrix at 8 columns 0.689 -> 0.642 ms; with four lanes it loses)
             constexpr int STEP = 2 * LPR;
-            for (int p = p0; p < p1; p += STEP) {
+            auto step = [&](int p, auto whole_tag) {
+                constexpr bool WHOLE = decltype(whole_tag)::value;
                 int myc[2];
                 float myv[2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const bool ok = p + h * LPR + lg < p1;
+                    const bool ok = WHOLE || p + h * LPR + lg < p1;
                     myc[h] = ok ? __ldg(a.colind + p + h * LPR + lg) : 0;
-                    myv[h] = ok ? to_float(vals[p + h * LPR + lg]) : 0.f;   // 0 beyond the end: such products vanish
+                    myv[h] = ok ? to_float(vals[p + h * LPR + lg]) : 0.f;
                 }
                 int cq[STEP];
                 float aq[STEP], b[STEP][VW];
@@ -66,8 +73,7 @@ seg_kernel(const SpmmArgs a) {
                 }
 #pragma unroll
                 for (int i = 0; i < STEP; ++i) {
-                    // entries beyond the chunk's end are not gathered: 0 * B[0, :] would turn a non-finite row 0 into NaN
-                    if (colok[0] && p + i < p1) {
+                    if (colok[0] && (WHOLE || p + i < p1)) {
                         RowLoad<T, VW>::ld(b_row(Bl, cq[i], a.ldb_bytes), b[i]);
                     } else {
 #pragma unroll
@@ -78,46 +84,57 @@ seg_kernel(const SpmmArgs a) {
                 for (int i = 0; i < STEP; ++i)
 #pragma unroll
                     for (int e = 0; e < VW; ++e) acc[0][e] = fmaf(aq[i], b[i][e], acc[0][e]);
-            }
-        } else
-        for (int p = p0; p < p1; p += LPR) {
-            int myc = 0;
-            float myv = 0.f;   // 0 beyond the segment's end: such products vanish
-            if (p + lg < p1) {
-                myc = __ldg(a.colind + p + lg);
-                myv = to_float(vals[p + lg]);
-            }
-            for (int q0 = 0; q0 < LPR && p + q0 < p1; q0 += QU) {
-                int cq[QU];
-                float aq[QU];
-#pragma unroll
-                for (int qq = 0; qq < QU; ++qq) {
-                    cq[qq] = (LPR == 1) ? myc : __shfl_sync(gmask, myc, q0 + qq, LPR);
-                    aq[qq] = (LPR == 1) ? myv : __shfl_sync(gmask, myv, q0 + qq, LPR);
+            };
+            int p = p0;
+            for (; p + STEP <= p1; p += STEP) step(p, std::true_type{});
+            if (p < p1) step(p, std::false_type{});
+        } else {
+            auto step = [&](int p, auto whole_tag) {
+                constexpr bool WHOLE = decltype(whole_tag)::value;
+                int myc = 0;
+                float myv = 0.f;
+                if (WHOLE || p + lg < p1) {
+                    myc = __ldg(a.colind + p + lg);
+                    myv = to_float(vals[p + lg]);
                 }
-                float b[QU][NV][VW];
+                for (int q0 = 0; q0 < LPR && (WHOLE || p + q0 < p1); q0 += QU) {
+                    int cq[QU];
+                    float aq[QU];
 #pragma unroll
-                for (int qq = 0; qq < QU; ++qq) {
-                    // an entry beyond the end has column 0 and value 0; it is not gathered, so that a
-                    // non-finite row 0 of B cannot reach rows that never name column 0
-                    const bool valid = p + q0 + qq < p1;
-                    const T *brow = b_row(Bl, cq[qq], a.ldb_bytes);
+                    for (int qq = 0; qq < QU; ++qq) {
+                        cq[qq] = (LPR == 1) ? myc : __shfl_sync(gmask, myc, q0 + qq, LPR);
+                        aq[qq] = (LPR == 1) ? myv : __shfl_sync(gmask, myv, q0 + qq, LPR);
+                    }
+                    float b[QU][NV][VW];
 #pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        if (valid && colok[v]) {
-                            RowLoad<T, VW>::ld(brow + v * LPR * VW, b[qq][v]);
-                        } else {
+                    for (int qq = 0; qq < QU; ++qq) {
+                        const bool valid = WHOLE || (p + q0 + qq < p1);
+                        const T *brow = b_row(Bl, cq[qq], a.ldb_bytes);
 #pragma unroll
-                            for (int e = 0; e < VW; ++e) b[qq][v][e] = 0.f;
+                        for (int v = 0; v < NV; ++v) {
+                            if (valid && colok[v]) {
+                                RowLoad<T, VW>::ld(brow + v * LPR * VW, b[qq][v]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < VW; ++e) b[qq][v][e] = 0.f;
+                            }
                         }
                     }
+#pragma unroll
+                    for (int qq = 0; qq < QU; ++qq)
+#pragma unroll
+                        for (int v = 0; v < NV; ++v)
+#pragma unroll
+                            for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(aq[qq], b[qq][v][e], acc[v][e]);
                 }
-#pragma unroll
-                for (int qq = 0; qq < QU; ++qq)
-#pragma unroll
-                    for (int v = 0; v < NV; ++v)
-#pragma unroll
-                        for (int e = 0; e < VW; ++e) acc[v][e] = fmaf(aq[qq], b[qq][v][e], acc[v][e]);
+            };
+            int p = p0;
+            if constexpr (SCRATCH) {
+                for (; p + LPR <= p1; p += LPR) step(p, std::true_type{});
+                if (p < p1) step(p, std::false_type{});
+            } else {
+                // short segments are mostly shorter than a step: one tested form (two copies of the loop cost 14 % here)
+                for (; p < p1; p += LPR) step(p, std::false_type{});
             }
         }
         if (SCRATCH) {
