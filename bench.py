@@ -715,7 +715,15 @@ def regret_rows(level: str, device_index: int = 0, log=None):
                       {"tiles, no windows": dict(family=sd.SD_MERGE, windows=1),
                        "class split, one window": dict(family=sd.SD_MERGE, windows=-1),
                        f"{rule_w} windows": dict(family=sd.SD_MERGE, windows=rule_w),
-                       f"{2 * rule_w} windows": dict(family=sd.SD_MERGE, windows=2 * rule_w)}, reps))
+                       f"{2 * rule_w} windows": dict(family=sd.SD_MERGE, windows=2 * rule_w),
+                       f"hybrid, {rule_w} windows": dict(family=sd.SD_HYBRID, windows=rule_w)}, reps))
+    # (D) hybrid family or windowed class split, by the bytes of one row of B
+    for dt, widths in ((W.SD_F32, (16, 24, 32, 48, 64) if full else (16, 32, 64)),
+                       (W.SD_BF16, (32, 48, 64, 128) if full else (64,))):
+        for N in widths:
+            w = W.config(4, dtype=dt, N=N, **({} if full else dict(M=1 << 20, scale_c=2.4e7 / 4, cap=50000)))
+            rows.append(point("hybrid family vs windowed class split", w, f"rank-size rows, M = {w.M}",
+                              {"class split, windows": dict(family=sd.SD_MERGE), "hybrid": dict(family=sd.SD_HYBRID)}, reps))
     return rows
 
 

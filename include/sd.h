@@ -57,12 +57,20 @@ typedef enum {
     SD_AUTO = 0,     /* decide from the structure summary */
     SD_ROWSPLIT = 1, /* sub-warp per row, vectorised gathers of B rows */
     SD_MERGE = 2,    /* merge-path split of (row ends + nonzeros), segmented reduction,
-                        deterministic carry-out fix-up.  There is no separate "hybrid" family (light rows
-                        row-wise, heavy rows in chunks, as in the paper's appendix listing): that schedule
-                        is this family's class split (sd_plan_info_t.class_split; long segments as
-                        128-nonzero chunks, short ones one lane group each, one-nonzero rows flat),
+                        deterministic carry-out fix-up; or its class split (sd_plan_info_t.class_split:
+                        the (row, column window) segments re-bucketed window by window, long ones as
+                        128-nonzero chunks, short ones one lane group each, one-nonzero ones flat),
                         chosen by dense width and forced with windows = -1 */
-    SD_BSR_TC = 3    /* 16x16 blocks on the tensor cores (tcgen05 / TMEM / TMA) */
+    SD_BSR_TC = 3,   /* 16x16 blocks on the tensor cores (tcgen05 / TMEM / TMA) */
+    SD_HYBRID = 4    /* the schedule of the paper's appendix listing (light rows row-wise, heavy rows in
+                        chunks), without its atomics: rows below heavy_len nonzeros are summed row-wise,
+                        several rows per lane group, longest first; every heavy row is cut, column window by
+                        column window, into chunks of at most 128 nonzeros of the caller's own CSR arrays
+                        (no re-bucketed copy of A), the chunks are summed window-major into scratch rows
+                        and one warp (or CTA) per heavy row adds its scratch rows in order.  Four launches
+                        at most, plan memory of a few bytes per row.  Needs ascending columns.  AUTO takes
+                        it in place of the windowed class split where the rows of B are 128 bytes
+                        (measured; see sd_plan_info_t.family) */
 } sd_family_t;
 
 /* Options of sd_plan_create_ex.  Zero-initialise, then set fields. */
@@ -81,7 +89,8 @@ typedef struct {
                               copy thread never fills its ring, and every wait gives up after a few thousand polls
                               instead of a million: the kernel must return by itself, sd_plan_device_status must
                               report a non-zero code, C is left incomplete */
-    int32_t reserved0;
+    int32_t heavy_len;     /* SD_HYBRID: rows of at least this many nonzeros run as chunks; 0 = the library's default
+                              (256, the long-row threshold of the paper's appendix listing); clamped to 2 .. 256 */
 } sd_plan_desc_t;
 
 /* Integer structure summary (Sec. 3.1 "Intrinsic pattern features", Eq. 4) and the
@@ -107,8 +116,8 @@ typedef struct {
     int32_t dtype;
     int32_t windows;        /* column windows in use (1 = none) */
     int32_t tile_items;     /* merge items (row ends + nonzeros) per CTA tile, MERGE only */
-    int64_t num_tiles;      /* MERGE: total tiles over all windows */
-    int64_t num_segments;   /* MERGE: rows, or (row, window) pairs with the class split */
+    int64_t num_tiles;      /* MERGE: total tiles over all windows.  HYBRID: number of heavy rows */
+    int64_t num_segments;   /* MERGE: rows, or (row, window) pairs with the class split.  HYBRID: number of chunks */
     int64_t plan_bytes;     /* device memory owned by the plan */
     int32_t sm_count;       /* hardware context read at plan time (Sec. 3.1) */
     int32_t launches;       /* kernel launches one sd_spmm call issues on the vectorised path */
@@ -116,7 +125,7 @@ typedef struct {
     int32_t class_split;    /* MERGE: 1 when the segments run by class (long ones as chunks, short ones one
                                lane group each, one-nonzero ones flat) instead of merge-path tiles: always
                                with windows > 1, and with one window where that alone pays */
-    int32_t reserved0;
+    int32_t heavy_len;      /* HYBRID: rows of at least this many nonzeros run as chunks (0 for the other families) */
 } sd_plan_info_t;
 
 /* sd_plan_create -- Sec. 3 (task <X, o, H> in, specialised implementation out) and
@@ -286,6 +295,22 @@ sd_status_t sd_plan_get_tiles(const sd_plan_t *plan, int32_t *tile_seg, int64_t 
  * Any pointer may be NULL.  SD_ERR_UNSUPPORTED when the plan does not use the class split. */
 sd_status_t sd_plan_get_segments(const sd_plan_t *plan, int32_t *seg_ptr, int32_t *seg_row, int32_t *colind,
                                  void *vals, int64_t *win_seg);
+
+/* sd_plan_get_hybrid -- HYBRID family: copy the schedule to HOST arrays (nl = info.num_tiles heavy rows,
+ * nc = info.num_segments chunks, W = info.windows, window of a column = col / ceil(K / W)).
+ *   heavy_rows  int32 [nl]       rows of at least info.heavy_len nonzeros, ascending
+ *   chunk_ptr   int32 [nl + 1]   first chunk of every heavy row; chunks are numbered row by row, inside a row
+ *                                window by window, inside a (row, window) piece by position
+ *   ranges      int32 [nc][2]    nonzero range [begin, end) of every chunk in the caller's colind / vals:
+ *                                a (row, window) piece of n nonzeros makes ceil(n / 128) chunks, all of 128
+ *                                nonzeros but the last
+ *   order       int32 [nc]       chunk numbers in the order the chunk kernel takes them: by window, then row,
+ *                                then position
+ *   light_rows  int32 [M - nl]   the other rows, longest first, ascending inside a length (rows without
+ *                                nonzeros last)
+ * Any pointer may be NULL.  SD_ERR_UNSUPPORTED for other families. */
+sd_status_t sd_plan_get_hybrid(const sd_plan_t *plan, int32_t *heavy_rows, int32_t *chunk_ptr, int32_t *ranges,
+                               int32_t *order, int32_t *light_rows);
 
 /* sd_plan_device_status -- every wait inside the library's kernels (mbarrier waits of the
  * tensor-core kernel) is bounded; a wait that runs out makes its CTA record a non-zero code

@@ -16,8 +16,8 @@ _SRC = os.path.join(_HERE, "sd_oracle.c")
 _SO = os.path.join(_HERE, "libsd_oracle.so")
 
 F32, BF16 = 0, 1
-ROWSPLIT, MERGE, BSR_TC = 1, 2, 3
-FAMILY_NAMES = {ROWSPLIT: "rowsplit", MERGE: "merge", BSR_TC: "bsr_tc"}
+ROWSPLIT, MERGE, BSR_TC, HYBRID = 1, 2, 3, 4
+FAMILY_NAMES = {ROWSPLIT: "rowsplit", MERGE: "merge", BSR_TC: "bsr_tc", HYBRID: "hybrid"}
 
 
 def build(force: bool = False) -> str:
@@ -217,6 +217,37 @@ def window_segments(rowptr, colind, M, K, W, short_len=32):
     S = int(lib().sdo_window_segments(C.c_int64(M), C.c_int64(K), _p(rowptr), _p(colind), C.c_int32(W),
                                       C.c_int32(short_len), _p(seg_ptr), _p(seg_row), _p(perm), _p(bounds)))
     return seg_ptr[:S + 1].copy(), seg_row[:S].copy(), perm[:nnz].copy(), bounds
+
+
+def decide_hybrid(info: Info, dtype: int, windows: int) -> bool:
+    """O4: hybrid family in place of the windowed class split (parity unpinned: this build's rule)."""
+    return bool(lib().sdo_decide_hybrid(C.byref(info), C.c_int(dtype), C.c_int(windows)))
+
+
+def decide_family(info: Info, dtype: int, l2_bytes: int) -> int:
+    """O4: the family a plan is built with (decide, then the hybrid family where decide_hybrid says so)."""
+    return int(lib().sdo_decide_family(C.byref(info), C.c_int(dtype), C.c_int64(l2_bytes)))
+
+
+def hybrid_schedule(rowptr, colind, M, K, W, heavy_len, chunk_nnz=128):
+    """O4: schedule of the hybrid family by its sequential definition.
+    Returns (heavy_rows, chunk_ptr, ranges [nc, 2], order, light_rows)."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    colind = np.ascontiguousarray(colind, dtype=np.int32)
+    nnz = int(rowptr[-1])
+    heavy = np.zeros(max(M, 1), np.int32)
+    chunk_ptr = np.zeros(M + 1, np.int32)
+    ranges = np.zeros(2 * max(nnz, 1), np.int32)
+    order = np.zeros(max(nnz, 1), np.int32)
+    light = np.zeros(max(M, 1), np.int32)
+    counts = np.zeros(3, np.int64)
+    rc = lib().sdo_hybrid_schedule(C.c_int64(M), C.c_int64(K), _p(rowptr), _p(colind), C.c_int32(W),
+                                   C.c_int32(heavy_len), C.c_int32(chunk_nnz), _p(heavy), _p(chunk_ptr), _p(ranges),
+                                   _p(order), _p(light), _p(counts))
+    assert rc == 0
+    nl, nc, nlight = (int(x) for x in counts)
+    return (heavy[:nl].copy(), chunk_ptr[:nl + 1].copy(), ranges[:2 * nc].reshape(nc, 2).copy(), order[:nc].copy(),
+            light[:nlight].copy())
 
 
 def hist_bin(v: int) -> int:

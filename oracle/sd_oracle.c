@@ -391,6 +391,7 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
 #define SDO_ROWSPLIT 1
 #define SDO_MERGE 2
 #define SDO_BSR_TC 3
+#define SDO_HYBRID 4
 
 /* Family rule on O3's integers (thresholds are this build's reading; the
  * paper gives none).  parity unpinned.
@@ -563,6 +564,88 @@ int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const i
     free(row);
     free(key);
     return S;
+}
+
+/* Hybrid family in place of the windowed class split (this build's rule, parity unpinned): a
+ * merge-family matrix that would run with column windows (sdo_decide_windows > 1) takes the hybrid
+ * schedule instead when one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns,
+ * 48 or 64 bf16 columns): measured on the target GPU on the rank-size matrix, the hybrid schedule
+ * takes 0.92 to 0.97 of the windowed schedule's time there and is behind it at narrower rows (1.05)
+ * and at wider ones (1.03 to 1.30: the light rows then gather wide rows of B from DRAM, which the
+ * windowed schedule finds in L2). */
+int sdo_decide_hybrid(const sdo_info_t *o, int dtype, int windows)
+{
+    int64_t row_bytes = o->N * (dtype == SDO_F32 ? 4 : 2);
+    return windows > 1 && o->unsorted_rows == 0 && row_bytes > 64 && row_bytes <= 128;
+}
+
+/* The family a plan is built with: sdo_decide, then the hybrid family in place of a merge family
+ * that would use column windows (l2_bytes: the L2 size the window rule works with). */
+int sdo_decide_family(const sdo_info_t *o, int dtype, int64_t l2_bytes)
+{
+    int family = sdo_decide(o, dtype);
+    if (family == SDO_MERGE && o->M > 0 && o->nnz > 0 &&
+        sdo_decide_hybrid(o, dtype, sdo_decide_windows(o, dtype, l2_bytes)))
+        family = SDO_HYBRID;
+    return family;
+}
+
+/* Hybrid schedule (the paper's appendix listing: rows below a length threshold run row-wise, the
+ * others are cut into chunks of bounded length; here the chunks also respect column windows and no
+ * atomics are used).  Sequential definition:
+ *   heavy rows   rows of at least heavy_len nonzeros, ascending
+ *   chunks       for every heavy row in order, for w = 0..W-1, the row's nonzeros whose column lies in
+ *                window w (col / ceil(K / W) == w; contiguous, columns ascend) cut into runs of
+ *                chunk_nnz nonzeros, the last one shorter; numbered in that order.
+ *                ranges[2c], ranges[2c+1] = first and one-past-last nonzero of chunk c;
+ *                chunk_ptr[i] = first chunk of the i-th heavy row, chunk_ptr[nl] = chunk count
+ *   order        the chunk numbers sorted by (window, heavy row, position): the window-major walk
+ *   light rows   all other rows by falling length, ascending row inside a length
+ * counts[0] = heavy rows, counts[1] = chunks, counts[2] = light rows.  heavy_rows and light_rows need
+ * room for M entries, chunk_ptr for M + 1, ranges for 2 nnz, order for nnz. */
+int sdo_hybrid_schedule(int64_t M, int64_t K, const int32_t *rowptr, const int32_t *colind, int32_t W,
+                        int32_t heavy_len, int32_t chunk_nnz, int32_t *heavy_rows, int32_t *chunk_ptr,
+                        int32_t *ranges, int32_t *order, int32_t *light_rows, int64_t *counts)
+{
+    int64_t wcols = (K + W - 1) / W, nl = 0, nc = 0, nlight = 0;
+    int32_t *win_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)(M > 0 ? rowptr[M] + 1 : 1));
+    for (int64_t i = 0; i < M; ++i) {
+        if (rowptr[i + 1] - rowptr[i] < heavy_len)
+            continue;
+        heavy_rows[nl] = (int32_t)i;
+        chunk_ptr[nl] = (int32_t)nc;
+        ++nl;
+        for (int32_t w = 0; w < W; ++w) {
+            int64_t run = 0;
+            for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+                if (colind[p] / wcols != w)
+                    continue;
+                if (run == 0) { /* a new chunk starts here */
+                    ranges[2 * nc] = (int32_t)p;
+                    win_of[nc] = w;
+                    ++nc;
+                }
+                ranges[2 * nc - 1] = (int32_t)(p + 1);
+                if (++run == chunk_nnz)
+                    run = 0;
+            }
+        }
+    }
+    chunk_ptr[nl] = (int32_t)nc;
+    int64_t q = 0;
+    for (int32_t w = 0; w < W; ++w)
+        for (int64_t c = 0; c < nc; ++c)
+            if (win_of[c] == w)
+                order[q++] = (int32_t)c;
+    for (int64_t len = heavy_len - 1; len >= 0; --len)
+        for (int64_t i = 0; i < M; ++i)
+            if (rowptr[i + 1] - rowptr[i] == len)
+                light_rows[nlight++] = (int32_t)i;
+    counts[0] = nl;
+    counts[1] = nc;
+    counts[2] = nlight;
+    free(win_of);
+    return q == nc ? 0 : 1;
 }
 
 /* ------------------------------------------------------------------ O5 */

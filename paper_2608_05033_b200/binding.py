@@ -18,11 +18,11 @@ LIB_PATH = os.path.join(PKG, "libsd.so")
 
 SD_OK, SD_ERR_INVALID_ARG, SD_ERR_UNSUPPORTED, SD_ERR_ALLOC, SD_ERR_CUDA, SD_ERR_INTERNAL = range(6)
 SD_F32, SD_BF16 = 0, 1
-SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC = 0, 1, 2, 3
-FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc"}
+SD_AUTO, SD_ROWSPLIT, SD_MERGE, SD_BSR_TC, SD_HYBRID = 0, 1, 2, 3, 4
+FAMILY_NAMES = {SD_ROWSPLIT: "rowsplit", SD_MERGE: "merge", SD_BSR_TC: "bsr_tc", SD_HYBRID: "hybrid"}
 
 EXPORTS = ["sd_plan_create", "sd_plan_create_ex", "sd_spmm", "sd_spmm_host", "sd_spmm_host_async", "sd_plan_sync", "sd_plan_update_values", "sd_plan_save", "sd_plan_load", "sd_plan_destroy",
-           "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_device_status", "sd_spmm_merge_static", "sd_last_error",
+           "sd_plan_get_info", "sd_plan_get_features", "sd_plan_get_bsr", "sd_plan_get_tiles", "sd_plan_get_segments", "sd_plan_get_hybrid", "sd_plan_device_status", "sd_spmm_merge_static", "sd_last_error",
            "sd_version"]
 
 
@@ -31,7 +31,7 @@ class sd_plan_desc_t(C.Structure):
                 ("M", C.c_int64), ("K", C.c_int64), ("N", C.c_int64),
                 ("dtype", C.c_int32), ("family", C.c_int32), ("windows", C.c_int32),
                 ("validate", C.c_int32), ("stream", C.c_void_p), ("test_wait_expiry", C.c_int32),
-                ("reserved0", C.c_int32)]
+                ("heavy_len", C.c_int32)]
 
 
 class sd_plan_info_t(C.Structure):
@@ -44,7 +44,7 @@ class sd_plan_info_t(C.Structure):
                 ("family", C.c_int32), ("dtype", C.c_int32), ("windows", C.c_int32),
                 ("tile_items", C.c_int32), ("num_tiles", C.c_int64), ("num_segments", C.c_int64),
                 ("plan_bytes", C.c_int64), ("sm_count", C.c_int32), ("launches", C.c_int32),
-                ("l2_bytes", C.c_int64), ("class_split", C.c_int32), ("reserved0", C.c_int32)]
+                ("l2_bytes", C.c_int64), ("class_split", C.c_int32), ("heavy_len", C.c_int32)]
 
     def as_dict(self) -> dict:
         d = {}
@@ -109,6 +109,8 @@ def load():
     lib.sd_plan_get_tiles.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
     lib.sd_plan_get_segments.restype = C.c_int
     lib.sd_plan_get_segments.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.sd_plan_get_hybrid.restype = C.c_int
+    lib.sd_plan_get_hybrid.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.sd_plan_device_status.restype = C.c_int
     lib.sd_plan_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     lib.sd_spmm_merge_static.restype = C.c_int
@@ -167,9 +169,10 @@ def sd_plan_create(rowptr, colind, vals, M: int, K: int, N: int):
 
 def sd_plan_create_ex(rowptr, colind, vals, M: int, K: int, N: int, dtype: int = SD_F32,
                       family: int = SD_AUTO, windows: int = 0, validate: bool = False, stream=None,
-                      test_wait_expiry: int = 0):
+                      test_wait_expiry: int = 0, heavy_len: int = 0):
     d = sd_plan_desc_t(_ptr(rowptr), _ptr(colind), _ptr(vals), M, K, N, dtype, family, windows,
-                       int(validate), _stream_handle(stream) if stream is not None else None, test_wait_expiry, 0)
+                       int(validate), _stream_handle(stream) if stream is not None else None, test_wait_expiry,
+                       heavy_len)
     out = C.c_void_p()
     rc = load().sd_plan_create_ex(C.byref(d), C.byref(out))
     if rc != SD_OK:
@@ -286,6 +289,22 @@ def sd_plan_get_segments(plan):
     return seg_ptr, seg_row, colind, vals, win_seg
 
 
+def sd_plan_get_hybrid(plan):
+    """Returns (heavy_rows, chunk_ptr, ranges [nc, 2], order, light_rows) of a plan of the hybrid family."""
+    info = sd_plan_get_info(plan)
+    nl, nc = info.num_tiles, info.num_segments
+    heavy = np.zeros(nl, np.int32)
+    chunk_ptr = np.zeros(nl + 1, np.int32)
+    ranges = np.zeros((nc, 2), np.int32)
+    order = np.zeros(nc, np.int32)
+    light = np.zeros(info.M - nl, np.int32)
+    rc = load().sd_plan_get_hybrid(plan, heavy.ctypes.data, chunk_ptr.ctypes.data, ranges.ctypes.data, order.ctypes.data,
+                                   light.ctypes.data)
+    if rc != SD_OK:
+        _raise(rc)
+    return heavy, chunk_ptr, ranges, order, light
+
+
 def sd_plan_device_status(plan) -> int:
     st = C.c_int32(0)
     rc = load().sd_plan_device_status(plan, C.byref(st))
@@ -311,14 +330,15 @@ class Plan:
     """Owns an sd_plan_t and keeps the borrowed CSR tensors alive."""
 
     def __init__(self, rowptr, colind, vals, M: int, K: int, N: int, dtype: int | None = None,
-                 family: int = SD_AUTO, windows: int = 0, validate: bool = False, test_wait_expiry: int = 0):
+                 family: int = SD_AUTO, windows: int = 0, validate: bool = False, test_wait_expiry: int = 0,
+                 heavy_len: int = 0):
         import torch
         if dtype is None:
             dtype = SD_F32 if vals.dtype == torch.float32 else SD_BF16
         self._keep = (rowptr, colind, vals)
         self.M, self.K, self.N, self.dtype = M, K, N, dtype
         self.handle = sd_plan_create_ex(rowptr, colind, vals, M, K, N, dtype, family, windows, validate,
-                                        test_wait_expiry=test_wait_expiry)
+                                        test_wait_expiry=test_wait_expiry, heavy_len=heavy_len)
 
     def spmm(self, B, Cmat, alpha: float = 1.0, beta: float = 0.0, stream=None):
         sd_spmm(self.handle, B, B.stride(0), Cmat, Cmat.stride(0), alpha, beta, stream)

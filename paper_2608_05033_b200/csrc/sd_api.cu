@@ -455,6 +455,18 @@ struct sd_plan {
     float *tile_tail = nullptr;
     int64_t ntiles = 0;
 
+    // HYBRID: rows of at least h_T nonzeros ("heavy") run as chunks of the caller's CSR arrays, the rest row-wise
+    int32_t *h_rows = nullptr;       // [h_nl] heavy rows, ascending
+    int32_t *h_chunk_ptr = nullptr;  // [h_nl + 1] first chunk of every heavy row (chunks are numbered row by row)
+    int2 *h_ranges = nullptr;        // [h_nc] nonzero range of every chunk
+    int32_t *h_order = nullptr;      // [h_nc] chunk ids in the order the chunk kernel takes them: by column window
+    int32_t *h_giant = nullptr;      // [h_ng] positions in h_rows of the rows of more than kGiantChunks chunks (a CTA sums each)
+    int64_t h_ng = 0;
+    int32_t *h_light = nullptr;      // [M - h_nl] light rows, longest first, ascending inside a length
+    int64_t h_nm = 0;                // the first h_nm of them have at least kHybridMedium nonzeros: one lane group per row
+    int64_t h_nl = 0, h_nc = 0;
+    int32_t h_T = 0;
+
     // narrow dense operands (N <= kCooMaxN) of the merge family
     int32_t *coo_row = nullptr;
     int32_t *coo_c1_row = nullptr, *coo_c2_row = nullptr;
@@ -572,6 +584,16 @@ static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
     return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= narrowest && s.N <= widest;
 }
 
+// The hybrid family in place of the windowed class split: where the merge family would run with column windows and
+// one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns, 48 or 64 bf16 columns).  Measured on the
+// rank-size matrix (`bench.py --regret`): 0.92 to 0.97 of the windowed class split's time there (4 launches instead of
+// 32, a tenth of the plan memory); behind it at 64 bytes and below (1.05) and beyond 128 bytes (1.03 to 1.30), where
+// the light rows gather wide rows of B from DRAM that the windowed schedule finds in L2.
+static bool decide_hybrid(const sd_plan_info_t &s, int dtype, int windows) {
+    const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
+    return windows > 1 && s.unsorted_rows == 0 && row_bytes > 64 && row_bytes <= 128;
+}
+
 __global__ void iota_kernel(int32_t *out, int64_t n) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i < n) out[i] = static_cast<int32_t>(i);
@@ -579,6 +601,12 @@ __global__ void iota_kernel(int32_t *out, int64_t n) {
 
 constexpr int kChunkNnz = 128;      // long segments are cut into pieces of at most this many nonzeros
 constexpr int kShortSegment = 32;   // segments up to this many nonzeros go to the group-per-segment kernel
+constexpr int kHybridHeavy = 256;   // hybrid family: rows of at least this many nonzeros run as chunks: the long-row threshold
+                                    // of the paper's appendix listing; measured on the rank-size matrix at 128-byte rows of
+                                    // B, 64 / 128 / 192 / 256 give 1.054 / 0.987 / 0.956 / 0.950 ms
+constexpr int kHybridMedium = 16;   // light rows of at least this many nonzeros take one lane group each, a step of nonzeros
+                                    // at a time; shorter ones run several rows per lane group, a nonzero at a time
+constexpr int kHybridHeavyMax = 256;   // upper limit: a light row is one running sum
 
 // Re-buckets the nonzeros by column window and builds the (row, window) segment list, ordered by
 // (window, class, row): inside a window the long segments come first (merge-path kernel), then the
@@ -882,6 +910,214 @@ static sd_status_t build_merge(sd_plan *p, int W, bool split, cudaStream_t st) {
     return SD_OK;
 }
 
+// ---- HYBRID: light rows row-wise, heavy rows as chunks inside column windows --------------------------------
+struct GiantRow {
+    const int32_t *chunk_ptr;
+    __device__ bool operator()(int32_t i) const { return chunk_ptr[i + 1] - chunk_ptr[i] > kGiantChunks; }
+};
+
+struct HeavyRow {
+    const int32_t *rowptr;
+    int32_t T;
+    __device__ bool operator()(int32_t r) const { return rowptr[r + 1] - rowptr[r] >= T; }
+};
+
+__device__ __forceinline__ int32_t first_not_below(const int32_t *__restrict__ colind, int32_t lo, int32_t hi, int64_t col) {
+    while (lo < hi) {
+        const int32_t mid = lo + ((hi - lo) >> 1);
+        if (colind[mid] < col) lo = mid + 1;
+        else hi = mid;
+    }
+    return lo;
+}
+
+// One thread per (heavy row i, window w): the nonzeros of the row whose columns fall in the window are a contiguous
+// range (columns ascend); counts its chunks into a row-major and a window-major table.
+__global__ void __launch_bounds__(256)
+hybrid_count_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, const int32_t *__restrict__ rows,
+                    int64_t nl, int32_t W, int64_t wcols, int32_t *__restrict__ start, int32_t *__restrict__ by_row,
+                    int32_t *__restrict__ by_win) {
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= nl * W) return;
+    const int64_t i = t / W;
+    const int32_t w = static_cast<int32_t>(t % W);
+    const int32_t r = rows[i], p0 = rowptr[r], p1 = rowptr[r + 1];
+    const int32_t lo = w == 0 ? p0 : first_not_below(colind, p0, p1, w * wcols);
+    const int32_t hi = w == W - 1 ? p1 : first_not_below(colind, lo, p1, (w + 1) * wcols);
+    const int32_t n = (hi - lo + kChunkNnz - 1) / kChunkNnz;
+    start[2 * t] = lo;
+    start[2 * t + 1] = hi;
+    by_row[t] = n;
+    by_win[static_cast<int64_t>(w) * nl + i] = n;
+}
+
+__global__ void __launch_bounds__(256)
+hybrid_fill_kernel(const int32_t *__restrict__ start, const int32_t *__restrict__ row_off, const int32_t *__restrict__ win_off,
+                   int64_t nl, int32_t W, int2 *__restrict__ ranges, int32_t *__restrict__ order,
+                   int32_t *__restrict__ chunk_ptr) {
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t > nl * W) return;
+    if (t == nl * W) {
+        chunk_ptr[nl] = row_off[t];
+        return;
+    }
+    const int64_t i = t / W;
+    const int32_t w = static_cast<int32_t>(t % W);
+    const int32_t c = row_off[t], o = win_off[static_cast<int64_t>(w) * nl + i];
+    if (w == 0) chunk_ptr[i] = c;
+    const int32_t lo = start[2 * t], hi = start[2 * t + 1];
+    for (int32_t j = 0, x = lo; x < hi; ++j, x += kChunkNnz) {
+        ranges[c + j] = make_int2(x, min(x + kChunkNnz, hi));
+        order[o + j] = c + j;
+    }
+}
+
+// Sort key of the light-row list: heavy rows first (they are not part of the list), then light rows by falling length.
+__global__ void __launch_bounds__(256)
+hybrid_light_key_kernel(const int32_t *__restrict__ rowptr, int64_t M, int32_t T, int32_t *__restrict__ key,
+                        int32_t *__restrict__ id) {
+    const int64_t r = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (r >= M) return;
+    const int32_t len = rowptr[r + 1] - rowptr[r];
+    key[r] = len >= T ? 0 : T - len;
+    id[r] = static_cast<int32_t>(r);
+}
+
+// Number of entries of the ascending array `key` that are <= v (one thread).
+__global__ void count_not_above_kernel(const int32_t *__restrict__ key, int64_t n, int32_t v, int64_t *__restrict__ out) {
+    int64_t lo = 0, hi = n;
+    while (lo < hi) {
+        const int64_t mid = lo + ((hi - lo) >> 1);
+        if (key[mid] <= v) lo = mid + 1;
+        else hi = mid;
+    }
+    *out = lo;
+}
+
+static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
+    sd_status_t s;
+    if (W < 1) W = 1;
+    if (T < 2) T = 2;
+    if (T > kHybridHeavyMax) T = kHybridHeavyMax;
+    p->h_T = T;
+    TempBuf sel, nsel, tmp, start, by_row, by_win, row_off, win_off;
+    if ((s = sel.get(sizeof(int32_t) * p->M, "heavy rows"))) return s;
+    if ((s = nsel.get(sizeof(int64_t), "heavy row count"))) return s;
+    size_t tb = 0;
+    cub::CountingInputIterator<int32_t> ids(0);
+    HeavyRow pred{p->rowptr, T};
+    SD_CUDA_TRY(cub::DeviceSelect::If(nullptr, tb, ids, static_cast<int32_t *>(sel.p), static_cast<int32_t *>(nsel.p),
+                                      static_cast<int32_t>(p->M), pred, st));
+    if ((s = tmp.get(tb, "select scratch"))) return s;
+    SD_CUDA_TRY(cub::DeviceSelect::If(tmp.p, tb, ids, static_cast<int32_t *>(sel.p), static_cast<int32_t *>(nsel.p),
+                                      static_cast<int32_t>(p->M), pred, st));
+    int32_t nl = 0;
+    SD_CUDA_TRY(cudaMemcpyAsync(&nl, nsel.p, sizeof nl, cudaMemcpyDeviceToHost, st));
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    p->h_nl = nl;
+    p->h_nc = 0;
+    if ((s = create_split_streams(p, 1))) return s;
+    p->info.windows = W;
+    p->info.launches = 1;
+    if (nl > 0) {
+        const int64_t cells = static_cast<int64_t>(nl) * W;
+        if (cells + 1 > INT32_MAX) {
+            set_error(SD_ERR_UNSUPPORTED, "too many (heavy row, window) pairs");
+            return SD_ERR_UNSUPPORTED;
+        }
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_rows), sizeof(int32_t) * nl, "heavy rows"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_chunk_ptr), sizeof(int32_t) * (nl + 1), "chunk pointers"))) return s;
+        SD_CUDA_TRY(cudaMemcpyAsync(p->h_rows, sel.p, sizeof(int32_t) * nl, cudaMemcpyDeviceToDevice, st));
+        if ((s = start.get(sizeof(int32_t) * 2 * cells, "window ranges"))) return s;
+        if ((s = by_row.get(sizeof(int32_t) * (cells + 1), "chunk counts"))) return s;
+        if ((s = by_win.get(sizeof(int32_t) * (cells + 1), "chunk counts"))) return s;
+        if ((s = row_off.get(sizeof(int32_t) * (cells + 1), "chunk offsets"))) return s;
+        if ((s = win_off.get(sizeof(int32_t) * (cells + 1), "chunk offsets"))) return s;
+        SD_CUDA_TRY(cudaMemsetAsync(static_cast<int32_t *>(by_row.p) + cells, 0, sizeof(int32_t), st));
+        SD_CUDA_TRY(cudaMemsetAsync(static_cast<int32_t *>(by_win.p) + cells, 0, sizeof(int32_t), st));
+        const int64_t wcols = (p->K + W - 1) / W;
+        hybrid_count_kernel<<<ceil_div(cells, 256), 256, 0, st>>>(p->rowptr, p->colind, p->h_rows, nl, W, wcols,
+                                                                 static_cast<int32_t *>(start.p),
+                                                                 static_cast<int32_t *>(by_row.p),
+                                                                 static_cast<int32_t *>(by_win.p));
+        SD_CUDA_TRY(cudaGetLastError());
+        size_t tb2 = 0;
+        SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(nullptr, tb2, static_cast<int32_t *>(by_row.p),
+                                                  static_cast<int32_t *>(row_off.p), static_cast<int32_t>(cells + 1), st));
+        TempBuf tmp2;
+        if ((s = tmp2.get(tb2, "scan scratch"))) return s;
+        SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(tmp2.p, tb2, static_cast<int32_t *>(by_row.p),
+                                                  static_cast<int32_t *>(row_off.p), static_cast<int32_t>(cells + 1), st));
+        SD_CUDA_TRY(cub::DeviceScan::ExclusiveSum(tmp2.p, tb2, static_cast<int32_t *>(by_win.p),
+                                                  static_cast<int32_t *>(win_off.p), static_cast<int32_t>(cells + 1), st));
+        int32_t nc = 0;
+        SD_CUDA_TRY(cudaMemcpyAsync(&nc, static_cast<int32_t *>(row_off.p) + cells, sizeof nc, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        p->h_nc = nc;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_ranges), sizeof(int2) * nc, "chunk ranges"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_order), sizeof(int32_t) * nc, "chunk order"))) return s;
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * nc * p->N, "chunk sums"))) return s;
+        hybrid_fill_kernel<<<ceil_div(cells + 1, 256), 256, 0, st>>>(static_cast<int32_t *>(start.p),
+                                                                    static_cast<int32_t *>(row_off.p),
+                                                                    static_cast<int32_t *>(win_off.p), nl, W, p->h_ranges,
+                                                                    p->h_order, p->h_chunk_ptr);
+        SD_CUDA_TRY(cudaGetLastError());
+        // rows of very many chunks: summed by a whole CTA each
+        GiantRow giant{p->h_chunk_ptr};
+        SD_CUDA_TRY(cub::DeviceSelect::If(tmp.p, tb, ids, static_cast<int32_t *>(sel.p), static_cast<int32_t *>(nsel.p), nl,
+                                          giant, st));
+        int32_t ng = 0;
+        SD_CUDA_TRY(cudaMemcpyAsync(&ng, nsel.p, sizeof ng, cudaMemcpyDeviceToHost, st));
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        p->h_ng = ng;
+        if (ng > 0) {
+            if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_giant), sizeof(int32_t) * ng, "giant rows"))) return s;
+            SD_CUDA_TRY(cudaMemcpyAsync(p->h_giant, sel.p, sizeof(int32_t) * ng, cudaMemcpyDeviceToDevice, st));
+            SD_CUDA_TRY(cudaStreamSynchronize(st));
+        }
+        p->info.launches = (nl < p->M ? 1 : 0) + 2 + (ng > 0 ? 1 : 0);
+    }
+    if (nl < p->M) {   // the light rows, longest first
+        TempBuf key, key_out, id, id_out, tmp3;
+        if ((s = key.get(sizeof(int32_t) * p->M, "light keys"))) return s;
+        if ((s = key_out.get(sizeof(int32_t) * p->M, "light keys"))) return s;
+        if ((s = id.get(sizeof(int32_t) * p->M, "row ids"))) return s;
+        if ((s = id_out.get(sizeof(int32_t) * p->M, "row ids"))) return s;
+        hybrid_light_key_kernel<<<ceil_div(p->M, 256), 256, 0, st>>>(p->rowptr, p->M, T, static_cast<int32_t *>(key.p),
+                                                                    static_cast<int32_t *>(id.p));
+        SD_CUDA_TRY(cudaGetLastError());
+        int bits = 1;
+        while ((1 << bits) <= T) ++bits;
+        size_t tb3 = 0;
+        SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, tb3, static_cast<int32_t *>(key.p), static_cast<int32_t *>(key_out.p),
+                                                    static_cast<int32_t *>(id.p), static_cast<int32_t *>(id_out.p),
+                                                    static_cast<int32_t>(p->M), 0, bits, st));
+        if ((s = tmp3.get(tb3, "sort scratch"))) return s;
+        SD_CUDA_TRY(cub::DeviceRadixSort::SortPairs(tmp3.p, tb3, static_cast<int32_t *>(key.p), static_cast<int32_t *>(key_out.p),
+                                                    static_cast<int32_t *>(id.p), static_cast<int32_t *>(id_out.p),
+                                                    static_cast<int32_t>(p->M), 0, bits, st));
+        if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_light), sizeof(int32_t) * (p->M - nl), "light rows"))) return s;
+        SD_CUDA_TRY(cudaMemcpyAsync(p->h_light, static_cast<int32_t *>(id_out.p) + nl, sizeof(int32_t) * (p->M - nl),
+                                    cudaMemcpyDeviceToDevice, st));
+        // sorted keys: 0 for the heavy rows, then T - length ascending; lengths of at least kHybridMedium have keys up to T - kHybridMedium
+        int64_t upto = nl;
+        if (T > kHybridMedium) {
+            count_not_above_kernel<<<1, 1, 0, st>>>(static_cast<int32_t *>(key_out.p), p->M, T - kHybridMedium,
+                                                    static_cast<int64_t *>(nsel.p));
+            SD_CUDA_TRY(cudaGetLastError());
+            SD_CUDA_TRY(cudaMemcpyAsync(&upto, nsel.p, sizeof upto, cudaMemcpyDeviceToHost, st));
+        }
+        SD_CUDA_TRY(cudaStreamSynchronize(st));
+        p->h_nm = upto - nl;
+        p->info.launches += (p->h_nm > 0 ? 1 : 0) - (p->h_nm == p->M - nl ? 1 : 0);   // medium rows add a launch; no shorter rows: one less
+    }
+    p->num_chunks = p->h_nc;
+    p->info.num_segments = p->h_nc;
+    p->info.num_tiles = p->h_nl;
+    p->info.heavy_len = T;
+    return SD_OK;
+}
+
 template <typename T>
 static cudaError_t fill_bsr(sd_plan *p, cudaStream_t st) {
     bsr_fill_kernel<T><<<148 * 8, 256, 0, st>>>(p->rowptr, p->colind, static_cast<const T *>(p->vals), p->M,
@@ -1040,6 +1276,17 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
 
     // ---- decision ------------------------------------------------------------------------------
     int family = d->family == SD_AUTO ? decide_family(info, p->dtype) : d->family;
+    if (d->family == SD_AUTO && family == SD_MERGE && d->windows == 0 && p->M > 0 && p->nnz > 0 &&
+        decide_hybrid(info, p->dtype, decide_windows(info, p->dtype)))
+        family = SD_HYBRID;
+    if (family == SD_HYBRID && info.unsorted_rows != 0) {   // the chunks of a window are ranges of the rows only if columns ascend
+        if (d->family == SD_HYBRID) {
+            set_error(SD_ERR_UNSUPPORTED, "the hybrid family needs ascending columns in every row (%lld rows are not)",
+                      (long long)info.unsorted_rows);
+            return SD_ERR_UNSUPPORTED;
+        }
+        family = SD_MERGE;
+    }
     if (family == SD_BSR_TC && (info.unsorted_rows != 0 || p->nnz == 0)) {
         if (d->family == SD_BSR_TC && info.unsorted_rows != 0) {
             set_error(SD_ERR_UNSUPPORTED, "BSR needs strictly ascending columns in every row (%lld rows are not)",
@@ -1063,6 +1310,10 @@ static sd_status_t create_plan(const sd_plan_desc_t *d, sd_plan *p) {
         if ((s = build_merge(p, W, split, st))) return s;
     } else if (family == SD_BSR_TC) {
         if ((s = build_bsr(p, static_cast<unsigned long long *>(keys_a.p), nnzb, st))) return s;
+    } else if (family == SD_HYBRID && p->M > 0 && p->nnz > 0) {
+        int W = d->windows == 0 ? decide_windows(info, p->dtype) : d->windows;
+        const int32_t T = d->heavy_len > 0 ? d->heavy_len : kHybridHeavy;
+        if ((s = build_hybrid(p, W, T, st))) return s;
     }
     info.plan_bytes = p->owned;
     return SD_OK;
@@ -1083,6 +1334,12 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->fix_long);
     cudaFree(p->tile_head);
     cudaFree(p->tile_tail);
+    cudaFree(p->h_rows);
+    cudaFree(p->h_chunk_ptr);
+    cudaFree(p->h_ranges);
+    cudaFree(p->h_order);
+    cudaFree(p->h_light);
+    cudaFree(p->h_giant);
     cudaFree(p->coo_row);
     cudaFree(p->coo_c1_row);
     cudaFree(p->coo_c1_val);
@@ -1153,8 +1410,8 @@ static sd_status_t pattern_hash(const int32_t *rowptr, const int32_t *colind, in
 }
 
 constexpr uint64_t kBlobMagic = 0x31304E414C504453ull;   // "SDPLAN01"
-constexpr uint32_t kBlobVersion = 1;
-constexpr int kBlobArrays = 13;
+constexpr uint32_t kBlobVersion = 2;
+constexpr int kBlobArrays = 19;
 
 struct BlobHeader {
     uint64_t magic;
@@ -1168,6 +1425,8 @@ struct BlobHeader {
     sd_plan_info_t info;
     int64_t num_segments, num_chunks, ntiles, nnzb;
     int32_t bsr_nparts, has_coo;
+    int64_t h_nl, h_nc, h_ng, h_nm;
+    int32_t h_T, reserved;
     uint64_t array_bytes[kBlobArrays];   // payload sizes, in the order of blob_arrays(); each padded to 16 bytes in the blob
 };
 
@@ -1201,6 +1460,14 @@ static void blob_arrays(sd_plan *p, BlobArray (&arr)[kBlobArrays]) {
     set(10, &p->browptr, bsr ? 4 * (Mb + 1) : 0, "browptr");
     set(11, &p->bcol, bsr ? 4 * p->nnzb : 0, "bcol");
     set(12, &p->bsr_part, (bsr && p->bsr_nparts > 0) ? 4 * (static_cast<int64_t>(p->bsr_nparts) + 1) : 0, "block-row partition");
+    const bool hyb = p->info.family == SD_HYBRID && p->h_T > 0;
+    const bool heavy = hyb && p->h_nl > 0;
+    set(13, &p->h_rows, heavy ? 4 * p->h_nl : 0, "heavy rows");
+    set(14, &p->h_chunk_ptr, heavy ? 4 * (p->h_nl + 1) : 0, "chunk pointers");
+    set(15, &p->h_ranges, heavy ? 8 * p->h_nc : 0, "chunk ranges");
+    set(16, &p->h_order, heavy ? 4 * p->h_nc : 0, "chunk order");
+    set(17, &p->h_giant, (heavy && p->h_ng > 0) ? 4 * p->h_ng : 0, "giant rows");
+    set(18, &p->h_light, (hyb && p->h_nl < p->M) ? 4 * (p->M - p->h_nl) : 0, "light rows");
 }
 
 static sd_status_t create_split_streams(sd_plan *p, int W) {
@@ -1253,7 +1520,7 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *d, sd_plan_t **out) {
         set_error(SD_ERR_INVALID_ARG, "unknown dtype %d", d->dtype);
         return SD_ERR_INVALID_ARG;
     }
-    if (d->family < SD_AUTO || d->family > SD_BSR_TC) {
+    if (d->family < SD_AUTO || d->family > SD_HYBRID) {
         set_error(SD_ERR_INVALID_ARG, "unknown family %d", d->family);
         return SD_ERR_INVALID_ARG;
     }
@@ -1365,7 +1632,8 @@ sd_status_t sd_plan_get_features(sd_plan_t *plan, sd_features_t *out) {
         for (int k = 0; k < 3; ++k)
             f.rep_bytes[5 + k] = (vb * bs[k] * bs[k] + 4) * f.nnzb[k] + 4 * ((info.M + bs[k] - 1) / bs[k] + 1);
         f.shape_class = shape_class_of(info);
-        const bool reads_csr = info.family == SD_ROWSPLIT || (info.family == SD_MERGE && !info.class_split);
+        const bool reads_csr = info.family == SD_ROWSPLIT || info.family == SD_HYBRID ||
+                               (info.family == SD_MERGE && !info.class_split);
         f.borrowed_bytes = reads_csr ? f.rep_bytes[0] : 0;
         f.plan_bytes = info.plan_bytes;
         f.d_r = info.K * info.N * vb;
@@ -1373,7 +1641,9 @@ sd_status_t sd_plan_get_features(sd_plan_t *plan, sd_features_t *out) {
         f.m_r = f.borrowed_bytes + f.plan_bytes + f.d_r;
         f.m_t = f.m_r + f.d_s;
         f.work_units = info.family == SD_MERGE ? (info.class_split ? info.num_segments : info.num_tiles)
-                                               : (info.family == SD_BSR_TC ? (info.M + 15) / 16 : info.M);
+                     : info.family == SD_BSR_TC ? (info.M + 15) / 16
+                     : info.family == SD_HYBRID ? info.num_segments + (info.M - info.num_tiles)
+                                                : info.M;
         f.sm_count = info.sm_count;
         f.l2_bytes = info.l2_bytes;
         plan->feat = f;
@@ -1398,6 +1668,28 @@ sd_status_t sd_plan_get_bsr(const sd_plan_t *plan, int32_t *browptr, int32_t *bc
     if (bcol && plan->nnzb)
         SD_CUDA_TRY(cudaMemcpy(bcol, plan->bcol, sizeof(int32_t) * plan->nnzb, cudaMemcpyDeviceToHost));
     if (bval && plan->nnzb) SD_CUDA_TRY(cudaMemcpy(bval, plan->bval, es * 256 * plan->nnzb, cudaMemcpyDeviceToHost));
+    return SD_OK;
+}
+
+sd_status_t sd_plan_get_hybrid(const sd_plan_t *plan, int32_t *heavy_rows, int32_t *chunk_ptr, int32_t *ranges,
+                               int32_t *order, int32_t *light_rows) {
+    if (!plan) {
+        set_error(SD_ERR_INVALID_ARG, "plan is null");
+        return SD_ERR_INVALID_ARG;
+    }
+    if (plan->info.family != SD_HYBRID) {
+        set_error(SD_ERR_UNSUPPORTED, "the plan's family is not SD_HYBRID");
+        return SD_ERR_UNSUPPORTED;
+    }
+    const int64_t nl = plan->h_nl, nc = plan->h_nc, nlight = plan->h_T > 0 ? plan->M - nl : 0;
+    if (heavy_rows && nl > 0) SD_CUDA_TRY(cudaMemcpy(heavy_rows, plan->h_rows, 4 * nl, cudaMemcpyDeviceToHost));
+    if (chunk_ptr) {
+        if (nl > 0) SD_CUDA_TRY(cudaMemcpy(chunk_ptr, plan->h_chunk_ptr, 4 * (nl + 1), cudaMemcpyDeviceToHost));
+        else chunk_ptr[0] = 0;
+    }
+    if (ranges && nc > 0) SD_CUDA_TRY(cudaMemcpy(ranges, plan->h_ranges, 8 * nc, cudaMemcpyDeviceToHost));
+    if (order && nc > 0) SD_CUDA_TRY(cudaMemcpy(order, plan->h_order, 4 * nc, cudaMemcpyDeviceToHost));
+    if (light_rows && nlight > 0) SD_CUDA_TRY(cudaMemcpy(light_rows, plan->h_light, 4 * nlight, cudaMemcpyDeviceToHost));
     return SD_OK;
 }
 
@@ -1641,6 +1933,59 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         if (ahead) SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_chunk.back(), 0));   // the caller's stream covers everything
         return SD_OK;
     }
+    case SD_HYBRID: {
+        const bool has_light = plan->h_nl < M, side = has_light && plan->h_nl > 0 && plan->aux[0] && !switches().no_side_streams;
+        cudaStream_t s_light = st;
+        if (side) {   // light rows and heavy rows write disjoint rows of C: side by side
+            s_light = plan->aux[0];
+            SD_CUDA_TRY(cudaEventRecord(plan->ev_fork, st));
+            SD_CUDA_TRY(cudaStreamWaitEvent(s_light, plan->ev_fork, 0));
+        }
+        if (plan->h_nl > 0) {
+            SpmmArgs ca = a;
+            ca.ranges = plan->h_ranges;
+            ca.order = plan->h_order;
+            ca.S = plan->h_nc;
+            ca.C = plan->chunk_out;
+            ca.ldc = N;
+            ca.alpha = 1.f;
+            ca.beta = 0.f;
+            SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, st));
+        }
+        cudaStream_t s_medium = st;
+        if (plan->h_nm > 0) {   // light rows of medium length: one lane group per row
+            if (side && plan->aux[1]) {
+                s_medium = plan->aux[1];
+                SD_CUDA_TRY(cudaStreamWaitEvent(s_medium, plan->ev_fork, 0));
+            }
+            SpmmArgs ma = a;
+            ma.seg_row = plan->h_light;
+            ma.S = plan->h_nm;
+            SD_CUDA_TRY(run_medium_rows(ma, plan->dtype, vec, s_medium));
+        }
+        if (M - plan->h_nl > plan->h_nm) {   // the short ones: several rows per lane group
+            SpmmArgs la = a;
+            la.seg_row = plan->h_light + plan->h_nm;
+            la.S = M - plan->h_nl - plan->h_nm;
+            SD_CUDA_TRY(run_light_rows(la, plan->dtype, vec, s_light));
+        }
+        if (plan->h_nl > 0) {
+            SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, 0, plan->h_nl, C, ldc,
+                                         static_cast<int32_t>(N), alpha, beta, st, plan->h_ng > 0 ? kGiantChunks : 0));
+            if (plan->h_ng > 0)
+                SD_CUDA_TRY(run_chunk_reduce_wide(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, plan->h_giant, plan->h_ng,
+                                                  C, ldc, static_cast<int32_t>(N), alpha, beta, st));
+        }
+        if (s_light != st) {
+            SD_CUDA_TRY(cudaEventRecord(plan->ev_join[0], s_light));
+            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[0], 0));
+        }
+        if (s_medium != st) {
+            SD_CUDA_TRY(cudaEventRecord(plan->ev_join[1], s_medium));
+            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[1], 0));
+        }
+        return SD_OK;
+    }
     case SD_BSR_TC: {
         BsrArgs b;
         b.browptr = plan->browptr;
@@ -1807,6 +2152,7 @@ sd_status_t sd_plan_save(const sd_plan_t *plan, void *buf, size_t cap, size_t *b
     h.nnzb = p->nnzb;
     h.bsr_nparts = p->bsr_nparts;
     h.has_coo = p->coo_row ? 1 : 0;
+    h.h_nl = p->h_nl; h.h_nc = p->h_nc; h.h_ng = p->h_ng; h.h_nm = p->h_nm; h.h_T = p->h_T;
     for (int i = 0; i < kBlobArrays; ++i) h.array_bytes[i] = arr[i].bytes;
     unsigned char *out = static_cast<unsigned char *>(buf);
     memset(out, 0, need);
@@ -1900,6 +2246,7 @@ sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, 
     p->ntiles = h.ntiles;
     p->nnzb = h.nnzb;
     p->bsr_nparts = h.bsr_nparts;
+    p->h_nl = h.h_nl; p->h_nc = h.h_nc; p->h_ng = h.h_ng; p->h_nm = h.h_nm; p->h_T = h.h_T;
     const unsigned char *in = static_cast<const unsigned char *>(blob);
     size_t off = pad16(sizeof(BlobHeader));
     p->wins.resize(h.nwins);
@@ -1951,6 +2298,11 @@ sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, 
             if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_row), sizeof(int32_t) * count3, "carry rows (level 2)"))) return fail(s);
             if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->coo_c2_val), sizeof(float) * count3 * p->N, "carry sums (level 2)"))) return fail(s);
         }
+    } else if (p->info.family == SD_HYBRID && p->h_T > 0) {
+        if (p->h_nl > 0 &&
+            (s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * p->h_nc * p->N, "chunk sums")))
+            return fail(s);
+        if ((s = create_split_streams(p, 1))) return fail(s);
     } else if (p->info.family == SD_BSR_TC) {
         if ((s = dev_alloc(p, &p->bval, es * 256 * p->nnzb, "bval"))) return fail(s);
         if ((s = dev_alloc(p, &p->bval_mma, (p->dtype == SD_BF16 ? 512 : 2048) * static_cast<size_t>(p->nnzb), "bval (tensor-core image)"))) return fail(s);

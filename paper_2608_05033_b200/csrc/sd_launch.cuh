@@ -22,6 +22,8 @@ struct MergeArgs {
 
 // Family (a).  `vec`: B, C, ldb, ldc and N allow 16-byte accesses.
 cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
+cudaError_t run_medium_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
+cudaError_t run_light_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
 
 // One lane group per segment (a.seg_row: output rows), or per chunk of a long segment
 // (`scratch`: chunk c writes its plain sum to row c of a.C).
@@ -33,7 +35,12 @@ cudaError_t run_single(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
 // Long segments of a window-major plan: segment s owns the scratch rows seg_chunk[s] ..
 // seg_chunk[s+1]-1 of chunk_out ([chunks][N]); their sum, taken in order, updates C[seg_row[s]].
 cudaError_t run_chunk_reduce(const float *chunk_out, const int32_t *seg_chunk, const int32_t *seg_row, int64_t seg_begin,
-                             int64_t seg_end, float *C, int64_t ldc, int32_t N, float alpha, float beta, cudaStream_t st);
+                             int64_t seg_end, float *C, int64_t ldc, int32_t N, float alpha, float beta, cudaStream_t st,
+                             int32_t skip_above = 0);
+constexpr int kGiantChunks = 64;   // segments of more chunks than this are summed by a whole CTA
+cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chunk, const int32_t *seg_row,
+                                  const int32_t *list, int64_t count, float *C, int64_t ldc, int32_t N, float alpha,
+                                  float beta, cudaStream_t st);
 
 // C = beta * C.
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st);

@@ -1,5 +1,6 @@
 #include "sd_launch.cuh"
 #include "sd_rowsplit.cuh"
+#include "sd_light.cuh"
 #include "sd_rowsplit_narrow.cuh"
 #include "sd_segment.cuh"
 
@@ -24,9 +25,21 @@ cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st
     return launch_rowsplit<__nv_bfloat16>(a, vec, st);
 }
 
+// Hybrid family, short rows: a.seg_row lists the rows (longest first), a.ptr is the row pointer array.
+cudaError_t run_light_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
+    if (dtype == SD_F32) return launch_light<float>(a, vec, st);
+    return launch_light<__nv_bfloat16>(a, vec, st);
+}
+
 cudaError_t run_segments(const SpmmArgs &a, int dtype, bool vec, bool scratch, cudaStream_t st) {
-    if (dtype == SD_F32) return launch_seg<float>(a, vec, scratch, st);
-    return launch_seg<__nv_bfloat16>(a, vec, scratch, st);
+    if (dtype == SD_F32) return launch_seg<float>(a, vec, scratch ? 1 : 0, st);
+    return launch_seg<__nv_bfloat16>(a, vec, scratch ? 1 : 0, st);
+}
+
+// Hybrid family, rows of medium length: a.seg_row lists the rows, a.ptr is the row pointer array.
+cudaError_t run_medium_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
+    if (dtype == SD_F32) return launch_seg<float>(a, vec, 2, st);
+    return launch_seg<__nv_bfloat16>(a, vec, 2, st);
 }
 
 cudaError_t run_single(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
@@ -35,14 +48,27 @@ cudaError_t run_single(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) 
 }
 
 cudaError_t run_chunk_reduce(const float *chunk_out, const int32_t *seg_chunk, const int32_t *seg_row, int64_t seg_begin,
-                             int64_t seg_end, float *C, int64_t ldc, int32_t N, float alpha, float beta, cudaStream_t st) {
+                             int64_t seg_end, float *C, int64_t ldc, int32_t N, float alpha, float beta, cudaStream_t st,
+                             int32_t skip_above) {
     const int64_t n = seg_end - seg_begin;
     if (N % 4 == 0)   // scratch rows are then 16-byte aligned
         chunk_reduce_kernel<4><<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, seg_begin,
-                                                                                 seg_end, C, ldc, N, alpha, beta, 0);
+                                                                                 seg_end, C, ldc, N, alpha, beta, skip_above);
     else
         chunk_reduce_kernel<1><<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, seg_begin,
-                                                                                 seg_end, C, ldc, N, alpha, beta, 0);
+                                                                                 seg_end, C, ldc, N, alpha, beta, skip_above);
+    return cudaGetLastError();
+}
+
+cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chunk, const int32_t *seg_row,
+                                  const int32_t *list, int64_t count, float *C, int64_t ldc, int32_t N, float alpha,
+                                  float beta, cudaStream_t st) {
+    if (N % 4 == 0)
+        chunk_reduce_wide_kernel<4><<<static_cast<unsigned>(count), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, list, C, ldc,
+                                                                                 N, alpha, beta);
+    else
+        chunk_reduce_wide_kernel<1><<<static_cast<unsigned>(count), 256, 0, st>>>(chunk_out, seg_chunk, seg_row, list, C, ldc,
+                                                                                 N, alpha, beta);
     return cudaGetLastError();
 }
 

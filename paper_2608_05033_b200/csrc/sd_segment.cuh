@@ -15,12 +15,16 @@ namespace sd {
 
 constexpr int kSegThreads = 256;
 
-// SCRATCH: the segments are chunks; chunk c writes its plain sum to row c of a.C (the scratch
-// matrix).  Otherwise a.seg_row gives the output row and whether an earlier window wrote it.
+// MODE 1 (SCRATCH): the segments are chunks; chunk c writes its plain sum to row c of a.C (the scratch
+// matrix).  MODE 0: a.seg_row gives the output row and whether an earlier window wrote it.
+// MODE 2: the segments are whole rows of the caller's CSR arrays named by the list a.seg_row (hybrid
+// family, rows of medium length); walked like chunks, written like segments.
 // Up to four lanes per row: six CTAs per SM (40 registers) measure 6 % faster; wider groups lose with that cap.
-template <typename T, int VW, int LPR, int NV, bool SCRATCH>
+template <typename T, int VW, int LPR, int NV, int MODE>
 __global__ void __launch_bounds__(kSegThreads, (LPR <= 4 && NV * VW < 8) ? 6 : 1)
 seg_kernel(const SpmmArgs a) {
+    constexpr bool SCRATCH = MODE == 1;   // output: scratch rows
+    constexpr bool STREAM = MODE != 0;    // walk: whole steps untested, next step's pairs requested ahead
     const int lane = threadIdx.x & 31;
     const int lg = threadIdx.x % LPR;
     const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << (lane & ~(LPR - 1)));
@@ -33,14 +37,30 @@ seg_kernel(const SpmmArgs a) {
     // gathers in flight per lane: the chunk kernel, which runs ahead of the rest on its own stream and is
     // bound by gather latency, takes all LPR of a step (measured: 12 % less time for the window-major
     // call); the short-segment kernel measures better with four and the higher occupancy
-    constexpr int QW = (NV * VW >= 8) ? 2 : (SCRATCH ? 8 : 4);
+    constexpr int QW = (NV * VW >= 8) ? 2 : (STREAM ? 8 : 4);
     constexpr int QU = LPR < QW ? LPR : QW;
 
     const int64_t gstride = static_cast<int64_t>(gridDim.x) * (kSegThreads / LPR);
     for (int64_t s = (static_cast<int64_t>(blockIdx.x) * kSegThreads + threadIdx.x) / LPR; s < a.S; s += gstride) {
-        const int p0 = __ldg(a.ptr + s), p1 = __ldg(a.ptr + s + 1);
+        int p0, p1;
+        int64_t out_row = s;   // SCRATCH: scratch row of this chunk
+        if (SCRATCH && a.ranges) {
+            // hybrid family: work item s is chunk order[s], a sub-range of one long row inside one column window
+            out_row = a.order ? __ldg(a.order + s) : s;
+            const int2 pr = __ldg(a.ranges + out_row);
+            p0 = pr.x;
+            p1 = pr.y;
+        } else if (MODE == 2) {
+            out_row = __ldg(a.seg_row + s);
+            p0 = __ldg(a.ptr + out_row);
+            p1 = __ldg(a.ptr + out_row + 1);
+        } else {
+            p0 = __ldg(a.ptr + s);
+            p1 = __ldg(a.ptr + s + 1);
+        }
         int32_t r = 0;
-        if (!SCRATCH) r = __ldg(a.seg_row + s);
+        if (MODE == 0) r = __ldg(a.seg_row + s);
+        if (MODE == 2) r = static_cast<int32_t>(out_row);
         float acc[NV][VW];
 #pragma unroll
         for (int v = 0; v < NV; ++v)
@@ -89,21 +109,37 @@ seg_kernel(const SpmmArgs a) {
             for (; p + STEP <= p1; p += STEP) step(p, std::true_type{});
             if (p < p1) step(p, std::false_type{});
         } else {
-            auto step = [&](int p, auto whole_tag) {
+            int myc = 0;
+            float myv = 0.f;
+            auto fetch = [&](int p, auto whole_tag) {   // the group's (column, value) pairs of the step that starts at p
                 constexpr bool WHOLE = decltype(whole_tag)::value;
-                int myc = 0;
-                float myv = 0.f;
+                myc = 0;
+                myv = 0.f;
                 if (WHOLE || p + lg < p1) {
                     myc = __ldg(a.colind + p + lg);
                     myv = to_float(vals[p + lg]);
+                }
+            };
+            auto step = [&](int p, auto whole_tag) {
+                constexpr bool WHOLE = decltype(whole_tag)::value;
+                int curc = myc;
+                float curv = myv;
+                if constexpr (STREAM) {
+                    // chunks: the next step's pairs are requested before this step's gathers, so that a step costs one
+                    // memory round trip instead of two (the chunk kernel is bound by that latency)
+                    fetch(p + LPR, std::false_type{});
+                } else {
+                    fetch(p, whole_tag);
+                    curc = myc;
+                    curv = myv;
                 }
                 for (int q0 = 0; q0 < LPR && (WHOLE || p + q0 < p1); q0 += QU) {
                     int cq[QU];
                     float aq[QU];
 #pragma unroll
                     for (int qq = 0; qq < QU; ++qq) {
-                        cq[qq] = (LPR == 1) ? myc : __shfl_sync(gmask, myc, q0 + qq, LPR);
-                        aq[qq] = (LPR == 1) ? myv : __shfl_sync(gmask, myv, q0 + qq, LPR);
+                        cq[qq] = (LPR == 1) ? curc : __shfl_sync(gmask, curc, q0 + qq, LPR);
+                        aq[qq] = (LPR == 1) ? curv : __shfl_sync(gmask, curv, q0 + qq, LPR);
                     }
                     float b[QU][NV][VW];
 #pragma unroll
@@ -129,7 +165,8 @@ seg_kernel(const SpmmArgs a) {
                 }
             };
             int p = p0;
-            if constexpr (SCRATCH) {
+            if constexpr (STREAM) {
+                fetch(p0, std::false_type{});
                 for (; p + LPR <= p1; p += LPR) step(p, std::true_type{});
                 if (p < p1) step(p, std::false_type{});
             } else {
@@ -138,7 +175,7 @@ seg_kernel(const SpmmArgs a) {
             }
         }
         if (SCRATCH) {
-            float *crow = a.C + s * a.ldc + cbase;
+            float *crow = a.C + out_row * a.ldc + cbase;
 #pragma unroll
             for (int v = 0; v < NV; ++v)
                 if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], 1.f, 0.f, 0);
@@ -210,7 +247,7 @@ template <int CW>
 __global__ void __launch_bounds__(256)
 chunk_reduce_kernel(const float *__restrict__ chunk_out, const int32_t *__restrict__ seg_chunk,
                     const int32_t *__restrict__ seg_row, int64_t seg_begin, int64_t seg_end, float *__restrict__ C,
-                    int64_t ldc, int32_t N, float alpha, float beta, int vec_c) {
+                    int64_t ldc, int32_t N, float alpha, float beta, int32_t skip_above) {
     const int lane = threadIdx.x & 31;
     const int64_t s = seg_begin + static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
     if (s >= seg_end) return;
@@ -219,6 +256,7 @@ chunk_reduce_kernel(const float *__restrict__ chunk_out, const int32_t *__restri
     while (lpc < 32 && lpc < units) lpc <<= 1;
     const int nchain = 32 / lpc, chain = lane / lpc, cl = lane % lpc;
     const int32_t c0 = __ldg(seg_chunk + s), c1 = __ldg(seg_chunk + s + 1);
+    if (skip_above > 0 && c1 - c0 > skip_above) return;   // left to chunk_reduce_wide_kernel
     const int32_t r = __ldg(seg_row + s);
     const bool accumulate = r < 0;
     float *crow = C + static_cast<int64_t>(r & 0x7FFFFFFF) * ldc;
@@ -252,43 +290,103 @@ chunk_reduce_kernel(const float *__restrict__ chunk_out, const int32_t *__restri
             }
         }
     }
-    (void)vec_c;
+}
+
+// Segments of very many chunks (list[]: their positions in seg_chunk / seg_row): one CTA each.  Warp w adds the chunks
+// c0 + w, c0 + w + 8, ... with the same chains as above; the eight warp sums meet in shared memory and warp 0 adds them
+// in warp order: a fixed order again.
+template <int CW>
+__global__ void __launch_bounds__(256)
+chunk_reduce_wide_kernel(const float *__restrict__ chunk_out, const int32_t *__restrict__ seg_chunk,
+                         const int32_t *__restrict__ seg_row, const int32_t *__restrict__ list, float *__restrict__ C,
+                         int64_t ldc, int32_t N, float alpha, float beta) {
+    __shared__ float part[8][32 * CW];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t s = __ldg(list + blockIdx.x);
+    const int units = (N + CW - 1) / CW;
+    int lpc = 1;
+    while (lpc < 32 && lpc < units) lpc <<= 1;
+    const int nchain = 32 / lpc, chain = lane / lpc, cl = lane % lpc;
+    const int32_t c0 = __ldg(seg_chunk + s), c1 = __ldg(seg_chunk + s + 1);
+    const int32_t r = __ldg(seg_row + s);
+    const bool accumulate = r < 0;
+    float *crow = C + static_cast<int64_t>(r & 0x7FFFFFFF) * ldc;
+    for (int ub = 0; ub < units; ub += lpc) {
+        const int col = (ub + cl) * CW;
+        float sum[CW];
+#pragma unroll
+        for (int e = 0; e < CW; ++e) sum[e] = 0.f;
+        if (col < N) {
+#pragma unroll 4
+            for (int32_t c = c0 + warp * nchain + chain; c < c1; c += 8 * nchain) {
+                const float *p = chunk_out + static_cast<int64_t>(c) * N + col;
+                if constexpr (CW == 4) {
+                    const float4 t = *reinterpret_cast<const float4 *>(p);
+                    sum[0] += t.x; sum[1] += t.y; sum[2] += t.z; sum[3] += t.w;
+                } else {
+                    sum[0] += *p;
+                }
+            }
+        }
+        for (int off = lpc; off < 32; off <<= 1)
+#pragma unroll
+            for (int e = 0; e < CW; ++e) sum[e] += __shfl_xor_sync(0xffffffffu, sum[e], off);
+        if (chain == 0)
+#pragma unroll
+            for (int e = 0; e < CW; ++e) part[warp][cl * CW + e] = sum[e];
+        __syncthreads();
+        if (warp == 0 && chain == 0 && col < N) {
+#pragma unroll
+            for (int e = 0; e < CW; ++e) {
+                float t = part[0][cl * CW + e];
+#pragma unroll
+                for (int w = 1; w < 8; ++w) t += part[w][cl * CW + e];
+                float v = alpha * t;
+                if (accumulate) v += crow[col + e];
+                else if (beta != 0.f) v = fmaf(beta, crow[col + e], v);
+                crow[col + e] = v;
+            }
+        }
+        __syncthreads();
+    }
 }
 
 template <typename T, int VW, int LPR, int NV>
-cudaError_t launch_seg_one(const SpmmArgs &a, bool scratch, cudaStream_t st) {
+cudaError_t launch_seg_one(const SpmmArgs &a, int mode, cudaStream_t st) {
     const int per_cta = kSegThreads / LPR;
     const int64_t need = (a.S + per_cta - 1) / per_cta;
     // persistent grid: exactly the CTAs that are resident together (the registers of an instance decide how
     // many of the eight 256-thread CTAs an SM takes); a larger grid would run a thin second wave
-    static std::atomic<int> occ_scratch[kMaxDevices], occ_plain[kMaxDevices];
-    const int occ = scratch ? occupancy_cached(occ_scratch, seg_kernel<T, VW, LPR, NV, true>, kSegThreads)
-                            : occupancy_cached(occ_plain, seg_kernel<T, VW, LPR, NV, false>, kSegThreads);
+    static std::atomic<int> occ_scratch[kMaxDevices], occ_plain[kMaxDevices], occ_rows[kMaxDevices];
+    const int occ = mode == 1 ? occupancy_cached(occ_scratch, seg_kernel<T, VW, LPR, NV, 1>, kSegThreads)
+                  : mode == 2 ? occupancy_cached(occ_rows, seg_kernel<T, VW, LPR, NV, 2>, kSegThreads)
+                              : occupancy_cached(occ_plain, seg_kernel<T, VW, LPR, NV, 0>, kSegThreads);
     const int64_t cap = static_cast<int64_t>(sm_count_cached()) * occ;
     dim3 grid(static_cast<unsigned>(need < cap ? need : cap),
               static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
-    if (scratch) seg_kernel<T, VW, LPR, NV, true><<<grid, kSegThreads, 0, st>>>(a);
-    else seg_kernel<T, VW, LPR, NV, false><<<grid, kSegThreads, 0, st>>>(a);
+    if (mode == 1) seg_kernel<T, VW, LPR, NV, 1><<<grid, kSegThreads, 0, st>>>(a);
+    else if (mode == 2) seg_kernel<T, VW, LPR, NV, 2><<<grid, kSegThreads, 0, st>>>(a);
+    else seg_kernel<T, VW, LPR, NV, 0><<<grid, kSegThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t launch_seg(const SpmmArgs &a, bool vec, bool scratch, cudaStream_t st) {
+cudaError_t launch_seg(const SpmmArgs &a, bool vec, int mode, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
     const LaneGeom g = lane_geometry(a.N, vec, VWV, false);
     if (vec && g.nv == 2) {
         switch (g.lpr) {
-        case 8: return launch_seg_one<T, VWV, 8, 2>(a, scratch, st);
-        case 16: return launch_seg_one<T, VWV, 16, 2>(a, scratch, st);
-        case 32: return launch_seg_one<T, VWV, 32, 2>(a, scratch, st);
+        case 8: return launch_seg_one<T, VWV, 8, 2>(a, mode, st);
+        case 16: return launch_seg_one<T, VWV, 16, 2>(a, mode, st);
+        case 32: return launch_seg_one<T, VWV, 32, 2>(a, mode, st);
         }
         return cudaErrorInvalidValue;
     }
 #define SD_SEG_CASE(L)                                                       \
     case L:                                                                  \
-        if (vec) return launch_seg_one<T, VWV, L, 1>(a, scratch, st);        \
-        return (g.nv == 4) ? launch_seg_one<T, 1, 32, 4>(a, scratch, st)     \
-                           : launch_seg_one<T, 1, L, 1>(a, scratch, st);
+        if (vec) return launch_seg_one<T, VWV, L, 1>(a, mode, st);        \
+        return (g.nv == 4) ? launch_seg_one<T, 1, 32, 4>(a, mode, st)     \
+                           : launch_seg_one<T, 1, L, 1>(a, mode, st);
     switch (g.lpr) {
         SD_SEG_CASE(1)
         SD_SEG_CASE(2)

@@ -35,14 +35,15 @@ def compare(w, plan):
     assert as_dict(got, COUNT_FIELDS) == as_dict(want, COUNT_FIELDS)
     pinfo = plan.info()
     # Eq. 11-12 for the plan as built
-    reads_csr = pinfo.family == sd.SD_ROWSPLIT or (pinfo.family == sd.SD_MERGE and not pinfo.class_split)
+    reads_csr = pinfo.family in (sd.SD_ROWSPLIT, sd.SD_HYBRID) or (pinfo.family == sd.SD_MERGE and not pinfo.class_split)
     assert got.borrowed_bytes == (oracle.csr_bytes(info, vb) if reads_csr else 0)
     assert got.plan_bytes == pinfo.plan_bytes
     m_r, m_t = oracle.working_set_bytes(got.borrowed_bytes + got.plan_bytes, info, vb)
     assert (got.m_r, got.m_t) == (m_r, m_t)
     assert (got.d_r, got.d_s) == (w.K * w.N * vb, 4 * w.M * w.N)
     units = {sd.SD_ROWSPLIT: w.M, sd.SD_MERGE: pinfo.num_segments if pinfo.class_split else pinfo.num_tiles,
-             sd.SD_BSR_TC: (w.M + 15) // 16}[pinfo.family]
+             sd.SD_BSR_TC: (w.M + 15) // 16,
+             sd.SD_HYBRID: pinfo.num_segments + w.M - pinfo.num_tiles}[pinfo.family]
     assert got.work_units == units
     assert (got.sm_count, got.l2_bytes) == (pinfo.sm_count, pinfo.l2_bytes)
     return got

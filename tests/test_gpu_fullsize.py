@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 CASES = [("tiny_uniform", 0, W.SD_F32, 1), ("stencil", 1, W.SD_F32, 1), ("gcn_rmat", 2, W.SD_F32, 2),
-         ("block16_f32", 3, W.SD_F32, 3), ("block16_bf16", 3, W.SD_BF16, 3), ("skewed", 4, W.SD_F32, 2),
+         ("block16_f32", 3, W.SD_F32, 3), ("block16_bf16", 3, W.SD_BF16, 3), ("skewed", 4, W.SD_F32, 4),
          # narrow dense operands of the two merge-family workloads (SpMV and four columns)
          ("skewed_spmv", 4, W.SD_F32, 2), ("gcn_rmat_n4", 2, W.SD_F32, 2)]
 NARROW = {"skewed_spmv": 1, "gcn_rmat_n4": 4}
@@ -32,8 +32,8 @@ def test_full_size_config_matches_oracle(name, ci, dtype, family):
     mine = info.as_dict()
     for k, v in ref.as_dict().items():
         assert mine[k] == v, k
-    assert info.family == oracle.decide(ref, dtype)
-    if info.family == sd.SD_MERGE:
+    assert info.family == oracle.decide_family(ref, dtype, info.l2_bytes)
+    if info.family in (sd.SD_MERGE, sd.SD_HYBRID):
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes)
     if name not in NARROW:   # extended analysis (quartiles, column degrees, SELL / BSR slots), every count exact
         fo = oracle.features(w.rowptr, w.colind, w.M, w.K, ref, 4 if dtype == W.SD_F32 else 2)

@@ -181,7 +181,7 @@ def test_scaled_configs_auto_plan_and_plan_parity(name):
     mine = info.as_dict()
     for k, v in ref.as_dict().items():
         assert mine[k] == v, k
-    assert info.family == oracle.decide(ref, w.dtype) == EXPECTED_FAMILY[name]
+    assert info.family == oracle.decide_family(ref, w.dtype, info.l2_bytes) == EXPECTED_FAMILY[name]
     if info.family == sd.SD_MERGE:
         assert bool(info.class_split) == (info.windows > 1 or oracle.decide_class_split(ref, w.dtype))
     if info.family == sd.SD_MERGE and not info.class_split:

@@ -26,6 +26,8 @@ def _cases():
     yield "merge_class_split", W.random_csr(1500, 4000, 32, rng.permutation(skew), seed=2), dict(family=2, windows=-1), "segments"
     yield "merge_windows", W.random_csr(1500, 4000, 32, rng.permutation(skew), seed=3, beta=-1.0), dict(family=2, windows=4), "segments"
     yield "merge_narrow", W.random_csr(1500, 4000, 2, rng.permutation(skew), seed=4), dict(family=2, windows=1), "tiles"
+    yield "hybrid", W.random_csr(1500, 4000, 32, rng.permutation(skew), seed=5, beta=0.25), dict(family=4, windows=4, heavy_len=40), "hybrid"
+    yield "hybrid_giant_row", W.random_csr(300, 9500, 64, np.r_[9000, rng.integers(0, 5, 299)], seed=6, dtype=W.SD_BF16), dict(family=4, windows=2), "hybrid"
     yield "blocks_bf16", W.g4_block(Mb=48, Kb=64, N=256, nblocks=150, dtype=W.SD_BF16), dict(family=3), "bsr"
     yield "blocks_fp32", W.g4_block(Mb=48, Kb=64, N=128, nblocks=150, dtype=W.SD_F32), dict(family=3), "bsr"
     yield "automatic", W.g1_tiny_uniform(), dict(), None
@@ -36,6 +38,8 @@ def _representation(plan, kind):
         return [sd.sd_plan_get_tiles(plan.handle)]
     if kind == "segments":
         return list(sd.sd_plan_get_segments(plan.handle))
+    if kind == "hybrid":
+        return list(sd.sd_plan_get_hybrid(plan.handle))
     if kind == "bsr":
         return list(sd.sd_plan_get_bsr(plan.handle))
     return []

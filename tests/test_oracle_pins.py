@@ -656,3 +656,69 @@ def test_o5_shape_class_on_designed_distributions():
     assert cls(W.random_csr(4000, 5000, 1, two, seed=1)) == "bimodal"
     geo = np.minimum(rng.geometric(1 / 9.0, 4000) - 1, 4000)                        # CV^2 = 1 / (1 - p) > 1, no heavy tail
     assert cls(W.random_csr(4000, 5000, 1, geo, seed=2)) == "skewed"
+
+
+def test_o4_hybrid_schedule_against_python_sets():
+    """The hybrid schedule from dictionaries and sorts: heavy rows, their (row, window) pieces cut into runs,
+    the window-major walk, and the light rows by falling length."""
+    rng = np.random.default_rng(21)
+    M, K, Wn, T, CH = 80, 333, 4, 9, 5
+    lengths = rng.integers(0, 9, size=M)
+    lengths[[3, 40, 41, 79]] = [60, 9, 8, 200]
+    lengths[17] = 0
+    wl = W.random_csr(M, K, 1, lengths, seed=4)
+    heavy, chunk_ptr, ranges, order, light = oracle.hybrid_schedule(wl.rowptr, wl.colind, M, K, Wn, T, CH)
+    wcols = -(-K // Wn)
+    assert heavy.tolist() == [i for i in range(M) if lengths[i] >= T] and 40 in heavy and 41 not in heavy
+    want_ranges, want_win, want_ptr = [], [], []
+    for i in heavy:
+        want_ptr.append(len(want_ranges))
+        pieces = {}
+        for p in range(wl.rowptr[i], wl.rowptr[i + 1]):
+            pieces.setdefault(int(wl.colind[p]) // wcols, []).append(p)
+        for win in sorted(pieces):
+            ps = pieces[win]
+            assert ps == list(range(ps[0], ps[-1] + 1))           # columns ascend: a piece is a range
+            for j in range(0, len(ps), CH):
+                want_ranges.append([ps[j], ps[min(j + CH, len(ps)) - 1] + 1])
+                want_win.append(win)
+    want_ptr.append(len(want_ranges))
+    assert ranges.tolist() == want_ranges and chunk_ptr.tolist() == want_ptr
+    # every nonzero of a heavy row lies in exactly one chunk, no chunk is longer than CH
+    covered = np.concatenate([np.arange(a, b) for a, b in ranges]) if len(ranges) else np.zeros(0, int)
+    heavy_nz = np.concatenate([np.arange(wl.rowptr[i], wl.rowptr[i + 1]) for i in heavy])
+    assert np.array_equal(np.sort(covered), heavy_nz) and np.all(np.diff(ranges, axis=1) <= CH)
+    # the walk: a stable sort of the chunk numbers by window
+    assert order.tolist() == sorted(range(len(want_ranges)), key=lambda c: (want_win[c], c))
+    assert light.tolist() == sorted((i for i in range(M) if lengths[i] < T), key=lambda i: (-lengths[i], i))
+    assert sorted(heavy.tolist() + light.tolist()) == list(range(M))
+    # one window: the walk is the numbering itself; a threshold above every row: nothing is heavy
+    h1, p1, r1, o1, l1 = oracle.hybrid_schedule(wl.rowptr, wl.colind, M, K, 1, T, CH)
+    assert o1.tolist() == list(range(len(r1))) and h1.tolist() == heavy.tolist()
+    h2, p2, r2, o2, l2 = oracle.hybrid_schedule(wl.rowptr, wl.colind, M, K, Wn, 1000, CH)
+    assert h2.size == 0 and r2.shape[0] == 0 and p2.tolist() == [0] and l2.size == M
+
+
+def test_o4_hybrid_rule():
+    """Hybrid in place of the windowed class split: only with column windows, ascending columns and rows of B
+    of more than 64 and at most 128 bytes; the family rule applies it on top of the merge decision."""
+    info = oracle.Info()
+    info.M, info.K, info.nnz, info.unsorted_rows = 1 << 20, 1 << 22, 5 << 20, 0
+    for dtype, es in ((oracle.F32, 4), (oracle.BF16, 2)):
+        for N in (8, 16, 17, 24, 32, 33, 48, 64, 65, 128):
+            info.N = N
+            want = 64 < N * es <= 128
+            assert oracle.decide_hybrid(info, dtype, 8) == want, (dtype, N)
+            assert not oracle.decide_hybrid(info, dtype, 1)
+    info.N, info.unsorted_rows = 32, 3
+    assert not oracle.decide_hybrid(info, oracle.F32, 8)
+    # the family rule: a skewed summary whose B exceeds the L2 budget
+    info.unsorted_rows, info.max_r, info.nnz_long_rows, info.sum_r2 = 0, 5000, info.nnz, 1 << 40
+    info.nnzb16 = info.nnz                                         # one entry per 16x16 block: no block form
+    l2 = 126 << 20
+    assert oracle.decide(info, oracle.F32) == oracle.MERGE and oracle.decide_windows(info, oracle.F32, l2) == 8
+    assert oracle.decide_family(info, oracle.F32, l2) == oracle.HYBRID
+    info.N = 128
+    assert oracle.decide_family(info, oracle.F32, l2) == oracle.MERGE
+    info.N, info.K = 32, 1 << 18                                   # B fits in L2: no windows, no hybrid
+    assert oracle.decide_family(info, oracle.F32, l2) == oracle.MERGE

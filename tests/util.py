@@ -21,10 +21,10 @@ class DeviceWorkload:
         self.colind = dev(w.colind) if w.colind.size else torch.zeros(1, dtype=torch.int32, device="cuda")
         self.vals = dev(w.vals) if w.vals.size else torch.zeros(1, dtype=torch.float32, device="cuda")
 
-    def plan(self, family=sd.SD_AUTO, windows=0, validate=False, N=None):
+    def plan(self, family=sd.SD_AUTO, windows=0, validate=False, N=None, heavy_len=0):
         w = self.w
         return sd.Plan(self.rowptr, self.colind, self.vals, w.M, w.K, w.N if N is None else N,
-                       dtype=w.dtype, family=family, windows=windows, validate=validate)
+                       dtype=w.dtype, family=family, windows=windows, validate=validate, heavy_len=heavy_len)
 
 
 def run_spmm(plan, w: W.Workload, pad_b=0, pad_c=0, offset=0, c_fill=None, alpha=None, beta=None):
