@@ -403,8 +403,8 @@ int sdo_summary(int64_t M, int64_t K, int64_t N, const int32_t *rowptr, const in
  *             compaction and fill-in costs").  rho_max is where the block form stops
  *             paying on the target GPU, by dense width and value type:
  *                        N < 128   128 <= N < 256   N >= 256
- *               fp32       9/8          2              11/4
- *               bf16       9/4          4              7
+ *               fp32       9/8          2              3
+ *               bf16       3            7              10
  *   MERGE     (max r >= 256 and rows >= 256 hold >= 10 % of nnz) or CV^2 >= 4
  *   ROWSPLIT  otherwise
  * CV^2 = M sum r^2 / nnz^2 - 1 >= 4  <=>  M sum r^2 >= 5 nnz^2. */
@@ -412,22 +412,19 @@ int sdo_decide(const sdo_info_t *o, int dtype)
 {
     int64_t num, den = 1;
     if (dtype == SDO_BF16) {
-        if (o->N < 128) {
-            num = 9;
-            den = 4;
-        } else if (o->N < 256) {
-            num = 4;
-        } else {
+        if (o->N < 128)
+            num = 3;
+        else if (o->N < 256)
             num = 7;
-        }
+        else
+            num = 10;
     } else if (o->N < 128) {
         num = 9;
         den = 8;
     } else if (o->N < 256) {
         num = 2;
     } else {
-        num = 11;
-        den = 4;
+        num = 3;
     }
     int64_t group = dtype == SDO_BF16 ? 64 : 32;
     if (o->N >= 64 && o->N % group == 0 && o->nnz > 0 && o->unsorted_rows == 0 &&

@@ -527,25 +527,17 @@ struct TempBuf {   // frees temporary device memory on every exit path
 // depends on the number of blocks only, the CSR kernels' time on the number of nonzeros; the
 // measured cross-over (random 16x16 blocks thinned to a given fill) by width and value type:
 //              N < 128   128 <= N < 256   N >= 256
-//     fp32       9/8          2              11/4
-//     bf16       9/4          4              7
+//     fp32       9/8          2              3
+//     bf16       3            7              10
 static int decide_family(const sd_plan_info_t &s, int dtype) {
     int64_t num, den = 1;
     if (dtype == SD_BF16) {
-        if (s.N < 128) {
-            num = 9;
-            den = 4;
-        } else {
-            num = s.N < 256 ? 4 : 7;
-        }
+        num = s.N < 128 ? 3 : (s.N < 256 ? 7 : 10);
     } else if (s.N < 128) {
         num = 9;
         den = 8;
-    } else if (s.N < 256) {
-        num = 2;
     } else {
-        num = 11;
-        den = 4;
+        num = s.N < 256 ? 2 : 3;
     }
     // the tensor-core kernel serves dense widths that are whole 128-byte groups of columns; at any other
     // width the block form would run its SIMT kernel, which is slower than the CSR kernels at every width

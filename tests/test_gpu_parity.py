@@ -591,7 +591,7 @@ def test_bsr_tensor_core_block_row_partition(dtype):
 @pytest.mark.parametrize("fill", [0.5, 0.2])
 def test_partially_filled_blocks_take_the_block_form_while_it_pays(dtype, fill):
     # 16x16 blocks thinned to a given fill: the automatic rule keeps the tensor-core block form down to
-    # a fill of 1/rho_max(dtype, N) -- at N = 256: 36 % for fp32, 14 % for bf16 -- and the result is
+    # a fill of 1/rho_max(dtype, N) -- at N = 256: 33 % for fp32, 10 % for bf16 -- and the result is
     # right either way
     base = W.g4_block(Mb=96, Kb=80, N=256, nblocks=700, seed=9, dtype=W.SD_F32)
     rng = np.random.default_rng(int(fill * 100))

@@ -408,8 +408,8 @@ def test_o4_merge_coords_match_closed_form():
 def test_o4_block_rule_thresholds_by_width_and_value_type():
     # the block form is taken while 256 * nnzb <= rho_max * nnz; rho_max by dense width and value type
     # (integer arithmetic: the boundary itself is inside)
-    table = {(oracle.F32, 64): (9, 8), (oracle.F32, 96): (9, 8), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (11, 4), (oracle.F32, 1024): (11, 4),
-             (oracle.BF16, 64): (9, 4), (oracle.BF16, 128): (4, 1), (oracle.BF16, 192): (4, 1), (oracle.BF16, 256): (7, 1)}
+    table = {(oracle.F32, 64): (9, 8), (oracle.F32, 96): (9, 8), (oracle.F32, 128): (2, 1), (oracle.F32, 256): (3, 1), (oracle.F32, 1024): (3, 1),
+             (oracle.BF16, 64): (3, 1), (oracle.BF16, 128): (7, 1), (oracle.BF16, 192): (7, 1), (oracle.BF16, 256): (10, 1)}
     w = W.g4_block(Mb=16, Kb=16, N=4, nblocks=30)
     base = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
     for (dt, N), (num, den) in table.items():
