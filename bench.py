@@ -701,13 +701,13 @@ def regret_rows(level: str, device_index: int = 0, log=None):
                 rows.append(point("family: blocks on tensor cores vs CSR kernels", w, f"block fill {fill:g}",
                                   {"bsr_tc": dict(family=sd.SD_BSR_TC), "rowsplit": dict(family=sd.SD_ROWSPLIT),
                                    "merge": dict(family=sd.SD_MERGE)}, reps))
-    # (B) merge family: class split or merge-path tiles, by dense width
+    # (B) skewed rows without column windows: merge-path tiles, class split or hybrid family, by dense width
     for dt in (W.SD_F32, W.SD_BF16):
-        for N in ((8, 16, 32, 64, 128) if full else (8, 32, 128)):
+        for N in ((5, 8, 16, 32, 64, 96, 128, 256) if full else (8, 32, 128)):
             w = W.config(2, dtype=dt, N=N, **({} if full else dict(scale=18)))
-            rows.append(point("merge family: class split vs tiles", w, "R-MAT scale %d" % (20 if full else 18),
-                              {"tiles": dict(family=sd.SD_MERGE, windows=1), "class_split": dict(family=sd.SD_MERGE, windows=-1)},
-                              reps))
+            rows.append(point("skewed rows, no column windows: tiles, class split or hybrid", w, "R-MAT scale %d" % (20 if full else 18),
+                              {"tiles": dict(family=sd.SD_MERGE, windows=1), "class_split": dict(family=sd.SD_MERGE, windows=-1),
+                               "hybrid": dict(family=sd.SD_HYBRID, windows=1)}, reps))
     # (C) column windows of the skewed workload: none, the rule's count, twice that
     w = W.config(4, **({} if full else dict(M=1 << 20, scale_c=2.4e7 / 4, cap=50000)))
     rule_w = 8 if full else 2

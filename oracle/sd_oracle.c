@@ -563,21 +563,27 @@ int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const i
     return S;
 }
 
-/* Hybrid family in place of the windowed class split (this build's rule, parity unpinned): a
- * merge-family matrix that would run with column windows (sdo_decide_windows > 1) takes the hybrid
- * schedule instead when one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns,
- * 48 or 64 bf16 columns): measured on the target GPU on the rank-size matrix, the hybrid schedule
- * takes 0.92 to 0.97 of the windowed schedule's time there and is behind it at narrower rows (1.05)
- * and at wider ones (1.03 to 1.30: the light rows then gather wide rows of B from DRAM, which the
- * windowed schedule finds in L2). */
+/* Hybrid family in place of the merge family's own schedules (this build's rule, parity unpinned;
+ * measured on the target GPU).  Needs ascending columns.  Without column windows: from 5 columns up
+ * to rows of B of 256 bytes (64 fp32 / 128 bf16 columns), where it takes 0.80 to 0.94 of the better of
+ * merge-path tiles and class split on the R-MAT matrix and is level with the class split on the
+ * rank-size matrix.  With column windows (sdo_decide_windows > 1): where one row of B is more than 64
+ * and at most 128 bytes (24 or 32 fp32 columns, 48 or 64 bf16 columns): 0.92 to 0.97 of the windowed
+ * class split's time on the rank-size matrix; behind it at narrower rows (1.06 to 1.28) and at wider
+ * ones (1.03 to 1.07: the light rows then gather wide rows of B from DRAM, which the windowed
+ * schedule finds in L2). */
 int sdo_decide_hybrid(const sdo_info_t *o, int dtype, int windows)
 {
     int64_t row_bytes = o->N * (dtype == SDO_F32 ? 4 : 2);
-    return windows > 1 && o->unsorted_rows == 0 && row_bytes > 64 && row_bytes <= 128;
+    if (o->unsorted_rows != 0)
+        return 0;
+    if (windows > 1)
+        return row_bytes > 64 && row_bytes <= 128;
+    return o->N >= 5 && row_bytes <= 256;
 }
 
-/* The family a plan is built with: sdo_decide, then the hybrid family in place of a merge family
- * that would use column windows (l2_bytes: the L2 size the window rule works with). */
+/* The family a plan is built with: sdo_decide, then the hybrid family in place of the merge family
+ * where sdo_decide_hybrid says so (l2_bytes: the L2 size the window rule works with). */
 int sdo_decide_family(const sdo_info_t *o, int dtype, int64_t l2_bytes)
 {
     int family = sdo_decide(o, dtype);

@@ -576,14 +576,21 @@ static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
     return s.unsorted_rows == 0 && s.nnz > 0 && s.N >= narrowest && s.N <= widest;
 }
 
-// The hybrid family in place of the windowed class split: where the merge family would run with column windows and
-// one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns, 48 or 64 bf16 columns).  Measured on the
-// rank-size matrix (`bench.py --regret`): 0.92 to 0.97 of the windowed class split's time there (4 launches instead of
-// 32, a tenth of the plan memory); behind it at 64 bytes and below (1.05) and beyond 128 bytes (1.03 to 1.30), where
-// the light rows gather wide rows of B from DRAM that the windowed schedule finds in L2.
+// The hybrid family in place of the merge family's own schedules, for matrices with ascending columns (measured,
+// `bench.py --regret`):
+//   without column windows: from 5 columns up to rows of B of 256 bytes (64 fp32 / 128 bf16 columns).  On the R-MAT
+//     matrix it takes 0.80 to 0.94 of the better of merge-path tiles and class split at every such width (fp32 5 to 64
+//     columns, bf16 8 to 128) and is level with the class split on the rank-size matrix; at 512-byte rows the tiles are
+//     ahead (1.12 against 1.27 ms), at 384 bytes it depends on the value type.
+//   with column windows: where one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns, 48 or 64 bf16
+//     columns): 0.92 to 0.97 of the windowed class split's time on the rank-size matrix (5 launches instead of 32, a
+//     tenth of the plan memory); behind it at 64 bytes and below (1.06 to 1.28) and beyond 128 bytes (1.03 to 1.07),
+//     where the light rows gather wide rows of B from DRAM that the windowed schedule finds in L2.
 static bool decide_hybrid(const sd_plan_info_t &s, int dtype, int windows) {
     const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
-    return windows > 1 && s.unsorted_rows == 0 && row_bytes > 64 && row_bytes <= 128;
+    if (s.unsorted_rows != 0) return false;
+    if (windows > 1) return row_bytes > 64 && row_bytes <= 128;
+    return s.N > kCooMaxN && row_bytes <= 256;
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {
@@ -762,7 +769,7 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     return SD_OK;
 }
 
-static sd_status_t create_split_streams(sd_plan *p, int W);
+static sd_status_t create_split_streams(sd_plan *p, int W, bool chunks_first = false);
 
 // `split`: the segments are re-bucketed by (window, class) and run through the chunk / segment / single
 // kernels; always so with W > 1, and with W = 1 when the class split alone pays (decide_class_split).
@@ -1008,7 +1015,7 @@ static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
     SD_CUDA_TRY(cudaStreamSynchronize(st));
     p->h_nl = nl;
     p->h_nc = 0;
-    if ((s = create_split_streams(p, 1))) return s;
+    if ((s = create_split_streams(p, 1, true))) return s;
     p->info.windows = W;
     p->info.launches = 1;
     if (nl > 0) {
@@ -1462,13 +1469,22 @@ static void blob_arrays(sd_plan *p, BlobArray (&arr)[kBlobArrays]) {
     set(18, &p->h_light, (hyb && p->h_nl < p->M) ? 4 * (p->M - p->h_nl) : 0, "light rows");
 }
 
-static sd_status_t create_split_streams(sd_plan *p, int W) {
+// chunks_first: the chunk stream gets the highest priority, so that when its persistent kernel and the kernels of the
+// side streams become runnable at the same moment (calls queued back to back) the chunk kernel's CTAs are placed first.
+static sd_status_t create_split_streams(sd_plan *p, int W, bool chunks_first) {
+    SD_CUDA_TRY(preload_stream_kernels(p->dtype, static_cast<int32_t>(p->N), chunks_first));   // before the streams exist
     for (int i = 0; i < 2; ++i) {
         SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
         SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
     }
     SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
-    SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
+    if (chunks_first) {
+        int least = 0, greatest = 0;
+        SD_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+        SD_CUDA_TRY(cudaStreamCreateWithPriority(&p->chunk_stream, cudaStreamNonBlocking, greatest));
+    } else {
+        SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
+    }
     p->ev_chunk.assign(W, nullptr);
     for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
     return SD_OK;
@@ -1927,11 +1943,15 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
     }
     case SD_HYBRID: {
         const bool has_light = plan->h_nl < M, side = has_light && plan->h_nl > 0 && plan->aux[0] && !switches().no_side_streams;
-        cudaStream_t s_light = st;
+        cudaStream_t s_light = st, s_heavy = st;
         if (side) {   // light rows and heavy rows write disjoint rows of C: side by side
             s_light = plan->aux[0];
             SD_CUDA_TRY(cudaEventRecord(plan->ev_fork, st));
             SD_CUDA_TRY(cudaStreamWaitEvent(s_light, plan->ev_fork, 0));
+            if (plan->chunk_stream && !switches().no_chunk_ahead) {   // the chunk kernel on the high-priority stream
+                s_heavy = plan->chunk_stream;
+                SD_CUDA_TRY(cudaStreamWaitEvent(s_heavy, plan->ev_fork, 0));
+            }
         }
         if (plan->h_nl > 0) {
             SpmmArgs ca = a;
@@ -1942,7 +1962,7 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
             ca.ldc = N;
             ca.alpha = 1.f;
             ca.beta = 0.f;
-            SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, st));
+            SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, s_heavy));
         }
         cudaStream_t s_medium = st;
         if (plan->h_nm > 0) {   // light rows of medium length: one lane group per row
@@ -1963,10 +1983,14 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         }
         if (plan->h_nl > 0) {
             SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, 0, plan->h_nl, C, ldc,
-                                         static_cast<int32_t>(N), alpha, beta, st, plan->h_ng > 0 ? kGiantChunks : 0));
+                                         static_cast<int32_t>(N), alpha, beta, s_heavy, plan->h_ng > 0 ? kGiantChunks : 0));
             if (plan->h_ng > 0)
                 SD_CUDA_TRY(run_chunk_reduce_wide(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, plan->h_giant, plan->h_ng,
-                                                  C, ldc, static_cast<int32_t>(N), alpha, beta, st));
+                                                  C, ldc, static_cast<int32_t>(N), alpha, beta, s_heavy));
+        }
+        if (s_heavy != st) {
+            SD_CUDA_TRY(cudaEventRecord(plan->ev_chunk[0], s_heavy));
+            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_chunk[0], 0));
         }
         if (s_light != st) {
             SD_CUDA_TRY(cudaEventRecord(plan->ev_join[0], s_light));
@@ -2294,7 +2318,7 @@ sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, 
         if (p->h_nl > 0 &&
             (s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * p->h_nc * p->N, "chunk sums")))
             return fail(s);
-        if ((s = create_split_streams(p, 1))) return fail(s);
+        if ((s = create_split_streams(p, 1, true))) return fail(s);
     } else if (p->info.family == SD_BSR_TC) {
         if ((s = dev_alloc(p, &p->bval, es * 256 * p->nnzb, "bval"))) return fail(s);
         if ((s = dev_alloc(p, &p->bval_mma, (p->dtype == SD_BF16 ? 512 : 2048) * static_cast<size_t>(p->nnzb), "bval (tensor-core image)"))) return fail(s);

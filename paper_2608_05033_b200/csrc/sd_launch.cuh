@@ -43,6 +43,7 @@ cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chu
                                   float beta, cudaStream_t st);
 
 // C = beta * C.
+cudaError_t preload_stream_kernels(int dtype, int32_t N, bool hybrid);
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st);
 
 // Family (b): tile kernel, then the carry-out fix-up for the listed tiles (short chains one per

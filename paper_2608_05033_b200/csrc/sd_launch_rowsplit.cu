@@ -72,6 +72,33 @@ cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chu
     return cudaGetLastError();
 }
 
+// Loads every kernel instance that the multi-stream schedules of a plan of this value type and dense width can launch
+// (both the 16-byte-vector and the scalar forms: which one runs depends on the operands' alignment at call time).
+// With lazy module loading a kernel is otherwise loaded at its first launch; when that happens in the middle of a
+// call that has just forked the plan's side streams, that plan's calls queued back to back stay 25 % slower for its
+// whole life (measured: 0.311 against 0.246 ms at 8 columns on the R-MAT matrix; loading eagerly or at plan creation
+// removes it).
+cudaError_t preload_stream_kernels(int dtype, int32_t N, bool hybrid) {
+    SpmmArgs a{};
+    a.N = N;
+    a.load_only = true;
+    const int vw = dtype == SD_F32 ? 4 : 8;
+    for (int v = 0; v < 2; ++v) {
+        const bool vec = v == 1;
+        if (vec && N % vw != 0) continue;
+        cudaError_t e = run_segments(a, dtype, vec, true, nullptr);
+        if (e == cudaSuccess) e = hybrid ? run_medium_rows(a, dtype, vec, nullptr) : run_segments(a, dtype, vec, false, nullptr);
+        if (e == cudaSuccess) e = hybrid ? run_light_rows(a, dtype, vec, nullptr) : run_single(a, dtype, vec, nullptr);
+        if (e != cudaSuccess) return e;
+    }
+    cudaFuncAttributes at;
+    cudaError_t e = cudaFuncGetAttributes(&at, chunk_reduce_kernel<4>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_kernel<1>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_wide_kernel<4>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_wide_kernel<1>);
+    return e;
+}
+
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st) {
     const int64_t total = M * N;
     const int blocks = static_cast<int>(std::min<int64_t>((total + 255) / 256, 148 * 16));

@@ -94,6 +94,10 @@ light_rows_kernel(const SpmmArgs a) {
 template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_light_one(const SpmmArgs &a, cudaStream_t st) {
     constexpr int R = (NV * VW >= 8) ? 2 : 4;
+    if (a.load_only) {
+        cudaFuncAttributes at;
+        return cudaFuncGetAttributes(&at, light_rows_kernel<T, VW, LPR, NV, R>);
+    }
     const int64_t groups = (a.S + R - 1) / R;
     const int per_cta = kLightThreads / LPR;
     dim3 grid(static_cast<unsigned>((groups + per_cta - 1) / per_cta),

@@ -353,6 +353,12 @@ chunk_reduce_wide_kernel(const float *__restrict__ chunk_out, const int32_t *__r
 
 template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_seg_one(const SpmmArgs &a, int mode, cudaStream_t st) {
+    if (a.load_only) {
+        cudaFuncAttributes at;
+        return mode == 1 ? cudaFuncGetAttributes(&at, seg_kernel<T, VW, LPR, NV, 1>)
+             : mode == 2 ? cudaFuncGetAttributes(&at, seg_kernel<T, VW, LPR, NV, 2>)
+                         : cudaFuncGetAttributes(&at, seg_kernel<T, VW, LPR, NV, 0>);
+    }
     const int per_cta = kSegThreads / LPR;
     const int64_t need = (a.S + per_cta - 1) / per_cta;
     // persistent grid: exactly the CTAs that are resident together (the registers of an instance decide how
@@ -401,6 +407,10 @@ cudaError_t launch_seg(const SpmmArgs &a, bool vec, int mode, cudaStream_t st) {
 
 template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_single_one(const SpmmArgs &a, cudaStream_t st) {
+    if (a.load_only) {
+        cudaFuncAttributes at;
+        return cudaFuncGetAttributes(&at, single_kernel<T, VW, LPR, NV>);
+    }
     const int per_cta = kSegThreads / LPR * kSingleBatch;
     dim3 grid(static_cast<unsigned>((a.S + per_cta - 1) / per_cta),
               static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));

@@ -167,7 +167,7 @@ def small_configs():
     }
 
 
-EXPECTED_FAMILY = {"tiny_uniform": 1, "stencil": 1, "gcn_rmat": 2, "block16_f32": 3, "block16_bf16": 3, "skewed": 2}
+EXPECTED_FAMILY = {"tiny_uniform": 1, "stencil": 1, "gcn_rmat": 2, "block16_f32": 3, "block16_bf16": 3, "skewed": 4}
 
 
 @pytest.mark.parametrize("name", list(EXPECTED_FAMILY))
@@ -193,6 +193,11 @@ def test_scaled_configs_auto_plan_and_plan_parity(name):
         rp, rr, perm, rw = oracle.window_segments(w.rowptr, w.colind, w.M, w.K, info.windows)
         assert np.array_equal(seg_ptr, rp) and np.array_equal(seg_row, rr) and np.array_equal(win_seg, rw)
         assert np.array_equal(colind, w.colind[perm]) and vals.tobytes() == w.vals[perm].tobytes()
+    if info.family == sd.SD_HYBRID:
+        assert info.windows == oracle.decide_windows(ref, w.dtype, info.l2_bytes) and info.heavy_len == 256
+        got_s = sd.sd_plan_get_hybrid(plan.handle)
+        ref_s = oracle.hybrid_schedule(w.rowptr, w.colind, w.M, w.K, info.windows, 256)
+        assert all(np.array_equal(a, b) for a, b in zip(got_s, ref_s))
     if info.family == sd.SD_BSR_TC:
         browptr, bcol, bval = sd.sd_plan_get_bsr(plan.handle)
         rb, rc, rv = oracle.bsr16(w.rowptr, w.colind, w.vals, w.M, w.K)
@@ -248,20 +253,20 @@ def test_unsorted_and_duplicate_columns():
 
 def test_long_all_positive_row_stays_inside_tolerance():
     # 200,000 same-sign terms in one row: sequential fp32 summation would drift to the edge of
-    # 1e-5; the tiled summation of the merge family must stay well inside
+    # 1e-5; the tiled summation of the merge family and the chunked one of the hybrid family must stay well inside
     M, K, N = 64, 262144, 32
     r = np.full(M, 3, np.int64)
     r[17] = 200_000
     w = W.random_csr(M, K, N, r, seed=31, positive=True)
     dw = DeviceWorkload(w)
-    for fam in (sd.SD_MERGE, sd.SD_ROWSPLIT):
+    for fam in (sd.SD_MERGE, sd.SD_HYBRID, sd.SD_ROWSPLIT):
         plan = dw.plan(family=fam)
         got, _ = run_spmm(plan, w)
         res = check(w, got)
-        if fam == sd.SD_MERGE:
+        if fam != sd.SD_ROWSPLIT:
             assert res["max_ratio"] < 0.5
         plan.close()
-    assert dw.plan().info().family == sd.SD_MERGE
+    assert dw.plan().info().family == sd.SD_HYBRID
 
 
 def test_one_row_holds_every_nonzero_and_rows_straddle_many_tiles():
@@ -696,20 +701,32 @@ def test_merge_class_split_with_one_window(kind, N, dtype):
     plan.close()
 
 
-def test_automatic_class_split_matches_the_rule():
+def test_automatic_schedule_of_a_skewed_matrix_matches_the_rules():
+    """Without column windows: the hybrid family from 5 columns up to 256-byte rows of B, else the merge family
+    (tiles; the COO reduction up to 4 columns).  A forced merge plan still takes its class split by the width rule."""
     for N, dtype in ((32, W.SD_F32), (16, W.SD_F32), (24, W.SD_F32), (64, W.SD_F32), (128, W.SD_F32), (32, W.SD_BF16), (64, W.SD_BF16),
-                     (8, W.SD_F32)):
+                     (128, W.SD_BF16), (256, W.SD_BF16), (8, W.SD_F32), (5, W.SD_F32), (4, W.SD_F32)):
         w = W.config(2, scale=12, N=N, dtype=dtype)
         dw = DeviceWorkload(w)
         plan = dw.plan()
         info = plan.info()
         ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
-        assert info.family == sd.SD_MERGE == oracle.decide(ref, dtype)
+        assert oracle.decide(ref, dtype) == oracle.MERGE
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes) == 1
-        assert bool(info.class_split) == oracle.decide_class_split(ref, dtype) == (16 <= N <= (64 if dtype == W.SD_F32 else 32))
+        hybrid = N >= 5 and N * (4 if dtype == W.SD_F32 else 2) <= 256
+        assert info.family == oracle.decide_family(ref, dtype, info.l2_bytes) == (sd.SD_HYBRID if hybrid else sd.SD_MERGE)
+        if not hybrid:
+            assert info.class_split == 0
         got, _ = run_spmm(plan, w)
         check(w, got)
         plan.close()
+        forced = dw.plan(family=sd.SD_MERGE)
+        fi = forced.info()
+        assert fi.family == sd.SD_MERGE
+        assert bool(fi.class_split) == oracle.decide_class_split(ref, dtype) == ((16 if dtype == W.SD_F32 else 8) <= N <= (64 if dtype == W.SD_F32 else 32))
+        got, _ = run_spmm(forced, w)
+        check(w, got)
+        forced.close()
 
 
 def test_automatic_window_choice_matches_the_rule():
