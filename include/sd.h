@@ -67,10 +67,11 @@ typedef enum {
                         several rows per lane group, longest first; every heavy row is cut, column window by
                         column window, into chunks of at most 128 nonzeros of the caller's own CSR arrays
                         (no re-bucketed copy of A), the chunks are summed window-major into scratch rows
-                        and one warp (or CTA) per heavy row adds its scratch rows in order.  Four launches
+                        and one warp (or CTA) per heavy row adds its scratch rows in order.  Five launches
                         at most, plan memory of a few bytes per row.  Needs ascending columns.  AUTO takes
-                        it in place of the windowed class split where the rows of B are 128 bytes
-                        (measured; see sd_plan_info_t.family) */
+                        it in place of SD_MERGE (measured rule): without column windows from 5 columns up to
+                        rows of B of 256 bytes, with column windows where a row of B is more than 64 and at
+                        most 128 bytes */
 } sd_family_t;
 
 /* Options of sd_plan_create_ex.  Zero-initialise, then set fields. */
@@ -153,8 +154,11 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
  * 16-byte aligned B/C with N, ldb, ldc multiples of the vector width take the
  * vectorised kernels; anything else takes scalar kernels (never an error).
  * With column windows the call issues one kernel sequence per window, in order, and C is
- * updated window by window.  A plan must not run concurrently on two streams (it owns
- * carry-out scratch).
+ * updated window by window.  Window-major and hybrid plans run part of their kernels on plan-owned
+ * streams that are forked from `stream` and joined back into it before the call returns, so that
+ * everything is ordered after what `stream` held before the call and before what is queued on it
+ * afterwards.  A plan must not run concurrently on two streams or from two host threads (it owns
+ * scratch, streams and events).
  * Results are run-to-run bit-identical (no floating-point atomics). */
 sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc,
                     float alpha, float beta, void *stream);
