@@ -464,6 +464,7 @@ struct sd_plan {
     int64_t h_ng = 0;
     int32_t *h_light = nullptr;      // [M - h_nl] light rows, longest first, ascending inside a length
     int64_t h_nm = 0;                // the first h_nm of them have at least kHybridMedium nonzeros: one lane group per row
+    int4 *h_desc = nullptr;          // [M - h_nl] per light row, in list order: {row, first nonzero, its column, length} (rebuilt at load)
     int64_t h_nl = 0, h_nc = 0;
     int32_t h_T = 0;
 
@@ -982,6 +983,27 @@ hybrid_light_key_kernel(const int32_t *__restrict__ rowptr, int64_t M, int32_t T
     id[r] = static_cast<int32_t>(r);
 }
 
+// Descriptors of the light rows: everything the first gather of a row needs, in one 16-byte load.
+__global__ void __launch_bounds__(256)
+hybrid_desc_kernel(const int32_t *__restrict__ rowptr, const int32_t *__restrict__ colind, const int32_t *__restrict__ rows,
+                   int64_t n, int4 *__restrict__ desc) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t r = rows[i], p0 = rowptr[r], len = rowptr[r + 1] - p0;
+    desc[i] = make_int4(r, p0, len > 0 ? colind[p0] : 0, len);
+}
+
+static sd_status_t build_light_desc(sd_plan *p, cudaStream_t st) {
+    const int64_t n = p->M - p->h_nl;
+    if (n <= 0) return SD_OK;
+    sd_status_t s;
+    if ((s = dev_alloc(p, reinterpret_cast<void **>(&p->h_desc), sizeof(int4) * n, "light row descriptors"))) return s;
+    hybrid_desc_kernel<<<ceil_div(n, 256), 256, 0, st>>>(p->rowptr, p->colind, p->h_light, n, p->h_desc);
+    SD_CUDA_TRY(cudaGetLastError());
+    SD_CUDA_TRY(cudaStreamSynchronize(st));
+    return SD_OK;
+}
+
 // Number of entries of the ascending array `key` that are <= v (one thread).
 __global__ void count_not_above_kernel(const int32_t *__restrict__ key, int64_t n, int32_t v, int64_t *__restrict__ out) {
     int64_t lo = 0, hi = n;
@@ -1109,6 +1131,7 @@ static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
         SD_CUDA_TRY(cudaStreamSynchronize(st));
         p->h_nm = upto - nl;
         p->info.launches += (p->h_nm > 0 ? 1 : 0) - (p->h_nm == p->M - nl ? 1 : 0);   // medium rows add a launch; no shorter rows: one less
+        if ((s = build_light_desc(p, st))) return s;
     }
     p->num_chunks = p->h_nc;
     p->info.num_segments = p->h_nc;
@@ -1338,6 +1361,7 @@ static void free_plan(sd_plan *p) {
     cudaFree(p->h_ranges);
     cudaFree(p->h_order);
     cudaFree(p->h_light);
+    cudaFree(p->h_desc);
     cudaFree(p->h_giant);
     cudaFree(p->coo_row);
     cudaFree(p->coo_c1_row);
@@ -1971,13 +1995,13 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
                 SD_CUDA_TRY(cudaStreamWaitEvent(s_medium, plan->ev_fork, 0));
             }
             SpmmArgs ma = a;
-            ma.seg_row = plan->h_light;
+            ma.desc = plan->h_desc;
             ma.S = plan->h_nm;
             SD_CUDA_TRY(run_medium_rows(ma, plan->dtype, vec, s_medium));
         }
         if (M - plan->h_nl > plan->h_nm) {   // the short ones: several rows per lane group
             SpmmArgs la = a;
-            la.seg_row = plan->h_light + plan->h_nm;
+            la.desc = plan->h_desc + plan->h_nm;
             la.S = M - plan->h_nl - plan->h_nm;
             SD_CUDA_TRY(run_light_rows(la, plan->dtype, vec, s_light));
         }
@@ -2318,6 +2342,7 @@ sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, 
         if (p->h_nl > 0 &&
             (s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * p->h_nc * p->N, "chunk sums")))
             return fail(s);
+        if ((s = build_light_desc(p, nullptr))) return fail(s);
         if ((s = create_split_streams(p, 1, true))) return fail(s);
     } else if (p->info.family == SD_BSR_TC) {
         if ((s = dev_alloc(p, &p->bval, es * 256 * p->nnzb, "bval"))) return fail(s);

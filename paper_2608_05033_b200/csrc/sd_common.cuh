@@ -156,6 +156,7 @@ struct SpmmArgs {
     int64_t mean_len;       // mean row length rounded up if known (0: unknown): lanes per row of the narrow row-split kernel
     // hybrid family (light rows row-wise, heavy rows as chunks):
     bool load_only = false;          // host side only: the launcher loads the kernel instance it would launch and returns
+    const int4 *desc = nullptr;      // light-rows kernel: {row, first nonzero, its column, length} of every row it takes
     const int2 *ranges = nullptr;    // chunk kernel: nonzero range [x, y) of every chunk (in the caller's CSR arrays) ...
     const int32_t *order = nullptr;  // ... and the order in which the chunks are taken (column-window-major); work item i is chunk order[i]
 };

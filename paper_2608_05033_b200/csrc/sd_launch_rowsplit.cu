@@ -25,7 +25,7 @@ cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st
     return launch_rowsplit<__nv_bfloat16>(a, vec, st);
 }
 
-// Hybrid family, short rows: a.seg_row lists the rows (longest first), a.ptr is the row pointer array.
+// Hybrid family, short rows: a.desc holds their descriptors (longest rows first).
 cudaError_t run_light_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
     if (dtype == SD_F32) return launch_light<float>(a, vec, st);
     return launch_light<__nv_bfloat16>(a, vec, st);
@@ -36,7 +36,7 @@ cudaError_t run_segments(const SpmmArgs &a, int dtype, bool vec, bool scratch, c
     return launch_seg<__nv_bfloat16>(a, vec, scratch ? 1 : 0, st);
 }
 
-// Hybrid family, rows of medium length: a.seg_row lists the rows, a.ptr is the row pointer array.
+// Hybrid family, rows of medium length: a.desc holds their descriptors.
 cudaError_t run_medium_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
     if (dtype == SD_F32) return launch_seg<float>(a, vec, 2, st);
     return launch_seg<__nv_bfloat16>(a, vec, 2, st);

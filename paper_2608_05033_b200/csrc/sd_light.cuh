@@ -1,10 +1,12 @@
 // Short rows of the hybrid family (a handful of nonzeros, most of them one or two), named by a list
 // that is sorted by falling length.  A group of LPR lanes owns R consecutive list entries at once, so
-// that R gathers (one per row) are in flight per lane at every step and the dependent chain
-// row pointer -> column index -> row of B is paid once per R rows; rows of similar length share a
-// warp.  The lanes of a group read the same (column, value) pair with one broadcast load: at these
-// lengths that is cheaper than loading LPR pairs and shuffling them.  Rows without nonzeros are
-// written too (C = beta * C).
+// that R gathers (one per row) are in flight per lane at every step; rows of similar length share a
+// warp.  Every list entry is a plan-time descriptor {row, first nonzero, column of the first nonzero,
+// length}: the first gather of a row depends on nothing but its descriptor (two dependent memory
+// round trips per one-nonzero row: descriptor, row of B; four without it: list, row pointer, column
+// index, row of B), and the (column, value) pair of step j + 1 is requested before the gathers of step j.
+// The lanes of a group read the same pair with one broadcast load: at these lengths that is cheaper
+// than loading LPR pairs and shuffling them.  Rows without nonzeros are written too (C = beta * C).
 #pragma once
 
 #include "sd_common.cuh"
@@ -28,21 +30,22 @@ light_rows_kernel(const SpmmArgs a) {
 #pragma unroll
     for (int v = 0; v < NV; ++v) colok[v] = cbase + (v * LPR + lg) * VW < a.N;
 
-    // a.seg_row: the list of rows, longest first; nullptr: all rows in order
-    int p[R], len[R], maxlen = 0;
+    int p[R], len[R], cn[R], maxlen = 0;
+    float vn[R];
     int64_t row[R];
     bool mine[R];
 #pragma unroll
     for (int u = 0; u < R; ++u) {
         mine[u] = r0 + u < a.S;
-        row[u] = !mine[u] ? 0 : a.seg_row ? __ldg(a.seg_row + r0 + u) : r0 + u;
-    }
-#pragma unroll
-    for (int u = 0; u < R; ++u) {
-        p[u] = mine[u] ? __ldg(a.ptr + row[u]) : 0;
-        len[u] = mine[u] ? __ldg(a.ptr + row[u] + 1) - p[u] : 0;
+        const int4 d = mine[u] ? __ldg(a.desc + r0 + u) : make_int4(0, 0, 0, 0);
+        row[u] = d.x;
+        p[u] = d.y;
+        cn[u] = d.z;
+        len[u] = d.w;
         maxlen = max(maxlen, len[u]);
     }
+#pragma unroll
+    for (int u = 0; u < R; ++u) vn[u] = len[u] > 0 ? to_float(vals[p[u]]) : 0.f;
     float acc[R][NV][VW];
 #pragma unroll
     for (int u = 0; u < R; ++u)
@@ -56,9 +59,11 @@ light_rows_kernel(const SpmmArgs a) {
         float av[R];
 #pragma unroll
         for (int u = 0; u < R; ++u) {
-            const bool ok = j < len[u];
-            c[u] = ok ? __ldg(a.colind + p[u] + j) : 0;
-            av[u] = ok ? to_float(vals[p[u] + j]) : 0.f;
+            c[u] = cn[u];
+            av[u] = vn[u];
+            const bool more = j + 1 < len[u];   // the next step's pair, requested before this step's gathers
+            cn[u] = more ? __ldg(a.colind + p[u] + j + 1) : 0;
+            vn[u] = more ? to_float(vals[p[u] + j + 1]) : 0.f;
         }
         float b[R][NV][VW];
 #pragma unroll

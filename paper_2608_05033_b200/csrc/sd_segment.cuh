@@ -17,7 +17,7 @@ constexpr int kSegThreads = 256;
 
 // MODE 1 (SCRATCH): the segments are chunks; chunk c writes its plain sum to row c of a.C (the scratch
 // matrix).  MODE 0: a.seg_row gives the output row and whether an earlier window wrote it.
-// MODE 2: the segments are whole rows of the caller's CSR arrays named by the list a.seg_row (hybrid
+// MODE 2: the segments are whole rows of the caller's CSR arrays named by the descriptors a.desc (hybrid
 // family, rows of medium length); walked like chunks, written like segments.
 // Up to four lanes per row: six CTAs per SM (40 registers) measure 6 % faster; wider groups lose with that cap.
 template <typename T, int VW, int LPR, int NV, int MODE>
@@ -51,9 +51,10 @@ seg_kernel(const SpmmArgs a) {
             p0 = pr.x;
             p1 = pr.y;
         } else if (MODE == 2) {
-            out_row = __ldg(a.seg_row + s);
-            p0 = __ldg(a.ptr + out_row);
-            p1 = __ldg(a.ptr + out_row + 1);
+            const int4 d = __ldg(a.desc + s);   // {row, first nonzero, its column, length}
+            out_row = d.x;
+            p0 = d.y;
+            p1 = d.y + d.w;
         } else {
             p0 = __ldg(a.ptr + s);
             p1 = __ldg(a.ptr + s + 1);
