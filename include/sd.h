@@ -157,8 +157,9 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
  * updated window by window.  Window-major and hybrid plans run part of their kernels on plan-owned
  * streams that are forked from `stream` and joined back into it before the call returns, so that
  * everything is ordered after what `stream` held before the call and before what is queued on it
- * afterwards.  A plan must not run concurrently on two streams or from two host threads (it owns
- * scratch, streams and events).
+ * afterwards (a stream capture of `stream` therefore takes the whole call into its graph).  A plan
+ * must not run concurrently on two streams or from two host threads (it owns scratch, streams and
+ * events).
  * Results are run-to-run bit-identical (no floating-point atomics). */
 sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C, int64_t ldc,
                     float alpha, float beta, void *stream);

@@ -169,3 +169,29 @@ def test_auto_takes_the_hybrid_family_where_the_rule_says_so():
         got, _ = run_spmm(plan, w)
         check(w, got)
         plan.close()
+
+
+@pytest.mark.parametrize("family,windows", [(4, 4), (2, 4)], ids=["hybrid", "windowed_class_split"])
+def test_calls_of_multi_stream_plans_can_be_captured_into_a_cuda_graph(family, windows):
+    """The plan-owned side streams are forked from and joined back into the caller's stream with events, so a stream
+    capture takes them in: two calls captured (the second adds to the first's result), replayed, checked."""
+    rng = np.random.default_rng(3)
+    M, K, N = 3000, 5000, 32
+    w = W.random_csr(M, K, N, lengths_of("skewed", M, K, rng), seed=5)
+    plan = DeviceWorkload(w).plan(family=family, windows=windows, heavy_len=64 if family == 4 else 0)
+    B = dev(w.B)
+    C = torch.full((M, N), float("nan"), device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        plan.spmm(B, C, 1.0, 0.0, side)                 # first call outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        plan.spmm(B, C, 1.0, 0.0, torch.cuda.current_stream())
+        plan.spmm(B, C, 1.0, 1.0, torch.cuda.current_stream())
+    for _ in range(2):
+        C.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        check(w, C.cpu().numpy() / np.float32(2.0))      # C = A B + (A B): halving is exact
+    plan.close()
