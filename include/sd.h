@@ -70,8 +70,7 @@ typedef enum {
                         and one warp (or CTA) per heavy row adds its scratch rows in order.  Five launches
                         at most, plan memory of a few bytes per row.  Needs ascending columns.  AUTO takes
                         it in place of SD_MERGE (measured rule): without column windows from 5 columns up to
-                        rows of B of 256 bytes, with column windows where a row of B is more than 64 and at
-                        most 128 bytes */
+                        rows of B of 384 bytes, with column windows where a row of B is 64 to 192 bytes */
 } sd_family_t;
 
 /* Options of sd_plan_create_ex.  Zero-initialise, then set fields. */

@@ -579,19 +579,21 @@ static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
 
 // The hybrid family in place of the merge family's own schedules, for matrices with ascending columns (measured,
 // `bench.py --regret`):
-//   without column windows: from 5 columns up to rows of B of 256 bytes (64 fp32 / 128 bf16 columns).  On the R-MAT
-//     matrix it takes 0.80 to 0.94 of the better of merge-path tiles and class split at every such width (fp32 5 to 64
-//     columns, bf16 8 to 128) and is level with the class split on the rank-size matrix; at 512-byte rows the tiles are
-//     ahead (1.12 against 1.27 ms), at 384 bytes it depends on the value type.
-//   with column windows: where one row of B is more than 64 and at most 128 bytes (24 or 32 fp32 columns, 48 or 64 bf16
-//     columns): 0.92 to 0.97 of the windowed class split's time on the rank-size matrix (5 launches instead of 32, a
-//     tenth of the plan memory); behind it at 64 bytes and below (1.06 to 1.28) and beyond 128 bytes (1.03 to 1.07),
-//     where the light rows gather wide rows of B from DRAM that the windowed schedule finds in L2.
+//   without column windows: from 5 columns up to rows of B of 384 bytes (96 fp32 / 192 bf16 columns).  On the R-MAT
+//     matrix it takes 0.80 to 0.94 of the better of merge-path tiles and class split at every width up to 256 bytes
+//     (fp32 5 to 64 columns, bf16 5 to 128) and is level with the class split on the rank-size matrix; at 384 bytes
+//     0.90 of the tiles' time with fp32 values and 1.02 with bf16 values; at 512-byte rows the tiles are ahead
+//     (1.12 against 1.19 ms).
+//   with column windows: where one row of B is 64 to 192 bytes (16 to 48 fp32 columns, 32 to 96 bf16 columns): on the
+//     rank-size matrix 0.90 to 0.93 of the windowed class split's time at 96 and 128 bytes and level with it (0.99 to
+//     1.005) at 64 and 192 bytes, with 5 launches instead of 16 to 64 and a quarter of the plan memory; behind it at
+//     32 bytes (1.28) and from 256 bytes on (1.01 to 1.05), where the light rows gather wide rows of B from DRAM that
+//     the windowed schedule finds in L2.
 static bool decide_hybrid(const sd_plan_info_t &s, int dtype, int windows) {
     const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
     if (s.unsorted_rows != 0) return false;
-    if (windows > 1) return row_bytes > 64 && row_bytes <= 128;
-    return s.N > kCooMaxN && row_bytes <= 256;
+    if (windows > 1) return row_bytes >= 64 && row_bytes <= 192;
+    return s.N > kCooMaxN && row_bytes <= 384;
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {

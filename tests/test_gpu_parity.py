@@ -702,10 +702,10 @@ def test_merge_class_split_with_one_window(kind, N, dtype):
 
 
 def test_automatic_schedule_of_a_skewed_matrix_matches_the_rules():
-    """Without column windows: the hybrid family from 5 columns up to 256-byte rows of B, else the merge family
+    """Without column windows: the hybrid family from 5 columns up to 384-byte rows of B, else the merge family
     (tiles; the COO reduction up to 4 columns).  A forced merge plan still takes its class split by the width rule."""
     for N, dtype in ((32, W.SD_F32), (16, W.SD_F32), (24, W.SD_F32), (64, W.SD_F32), (128, W.SD_F32), (32, W.SD_BF16), (64, W.SD_BF16),
-                     (128, W.SD_BF16), (256, W.SD_BF16), (8, W.SD_F32), (5, W.SD_F32), (4, W.SD_F32)):
+                     (128, W.SD_BF16), (256, W.SD_BF16), (8, W.SD_F32), (5, W.SD_F32), (4, W.SD_F32), (96, W.SD_F32), (192, W.SD_BF16)):
         w = W.config(2, scale=12, N=N, dtype=dtype)
         dw = DeviceWorkload(w)
         plan = dw.plan()
@@ -713,7 +713,7 @@ def test_automatic_schedule_of_a_skewed_matrix_matches_the_rules():
         ref = oracle.summary(w.rowptr, w.colind, w.M, w.K, w.N)
         assert oracle.decide(ref, dtype) == oracle.MERGE
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes) == 1
-        hybrid = N >= 5 and N * (4 if dtype == W.SD_F32 else 2) <= 256
+        hybrid = N >= 5 and N * (4 if dtype == W.SD_F32 else 2) <= 384
         assert info.family == oracle.decide_family(ref, dtype, info.l2_bytes) == (sd.SD_HYBRID if hybrid else sd.SD_MERGE)
         if not hybrid:
             assert info.class_split == 0

@@ -700,16 +700,16 @@ def test_o4_hybrid_schedule_against_python_sets():
 
 
 def test_o4_hybrid_rule():
-    """Hybrid in place of the merge family's schedules: ascending columns; with column windows rows of B of more
-    than 64 and at most 128 bytes, without them 5 columns and more up to 256-byte rows; the family rule applies it on
-    top of the merge decision."""
+    """Hybrid in place of the merge family's schedules: ascending columns; with column windows rows of B of 64 to
+    192 bytes, without them 5 columns and more up to 384-byte rows; the family rule applies it on top of the merge
+    decision."""
     info = oracle.Info()
     info.M, info.K, info.nnz, info.unsorted_rows = 1 << 20, 1 << 22, 5 << 20, 0
     for dtype, es in ((oracle.F32, 4), (oracle.BF16, 2)):
         for N in (1, 4, 5, 8, 16, 17, 24, 32, 33, 48, 64, 65, 96, 128, 129, 256):
             info.N = N
-            assert oracle.decide_hybrid(info, dtype, 8) == (64 < N * es <= 128), (dtype, N)
-            assert oracle.decide_hybrid(info, dtype, 1) == (N >= 5 and N * es <= 256), (dtype, N)
+            assert oracle.decide_hybrid(info, dtype, 8) == (64 <= N * es <= 192), (dtype, N)
+            assert oracle.decide_hybrid(info, dtype, 1) == (N >= 5 and N * es <= 384), (dtype, N)
     info.N, info.unsorted_rows = 32, 3
     assert not oracle.decide_hybrid(info, oracle.F32, 8) and not oracle.decide_hybrid(info, oracle.F32, 1)
     # the family rule: a skewed summary whose B exceeds the L2 budget
@@ -720,7 +720,7 @@ def test_o4_hybrid_rule():
     assert oracle.decide_family(info, oracle.F32, l2) == oracle.HYBRID
     info.N = 128                                                   # 512-byte rows, 32 windows: the windowed class split
     assert oracle.decide_family(info, oracle.F32, l2) == oracle.MERGE
-    info.N, info.K = 32, 1 << 18                                   # B fits in L2: no windows, hybrid up to 256-byte rows
+    info.N, info.K = 32, 1 << 18                                   # B fits in L2: no windows, hybrid up to 384-byte rows
     assert oracle.decide_windows(info, oracle.F32, l2) == 1 and oracle.decide_family(info, oracle.F32, l2) == oracle.HYBRID
     info.N = 128
     assert oracle.decide_family(info, oracle.F32, l2) == oracle.MERGE
