@@ -17,7 +17,10 @@ PATHS = {0: "plain loads, 4 in flight per lane", 1: "plain loads, 8 in flight", 
          5: "tile order, indices staged in shared memory, evict-last", 6: "half warp per row, two vectors per lane",
          7: "bulk-copy ring (cp.async.bulk, 512 B per copy) + shared loads",
          8: "hub rows in distributed shared memory, cluster of 4", 9: "hub rows in distributed shared memory, cluster of 8",
-         10: "hub rows in distributed shared memory, cluster of 16"}
+         10: "hub rows in distributed shared memory, cluster of 16",
+         11: "cp.async 16-byte copies into a per-warp shared-memory ring, 16 rows in flight per warp, L1 bypassed",
+         12: "cp.async ring, 16 rows in flight per warp, through L1",
+         13: "cp.async ring, 32 rows in flight per warp, L1 bypassed"}
 HUB_CLUSTER = {8: 4, 9: 8, 10: 16}
 HUB_ROWS_PER_CTA = 256
 

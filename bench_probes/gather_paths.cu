@@ -220,6 +220,53 @@ __global__ void __launch_bounds__(32 * (kBulkCons + 1)) bulk_ring_kernel(const i
     sink[(long)blockIdx.x * blockDim.x + tid] = acc;
 }
 
+// ---- asynchronous 16-byte copies (cp.async) into a per-warp shared-memory ring: a gather in flight holds a ring slot
+// instead of registers, so a warp can keep D rows (D * 512 bytes) in flight; every lane copies and later reads back
+// its own 16 bytes of a row, so the warp needs no barrier.  Batches of WB rows are one commit group; NB = D / WB
+// groups are in flight.  CG: copies bypass L1 (cp.async.cg), else they allocate in it (cp.async.ca) -----------------
+template <int D, int WB, bool CG>
+__global__ void __launch_bounds__(256) async_ring_kernel(const int *__restrict__ idx, long count, const char *__restrict__ table,
+                                                        float4 *__restrict__ sink) {
+    extern __shared__ __align__(16) char ring_mem[];
+    constexpr int NB = D / WB;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    char *ring = ring_mem + (size_t)w * D * 512 + lane * 16;
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+    const char *base = table + lane * 16;
+    const long g = (long)blockIdx.x * 8 + w, G = (long)gridDim.x * 8;
+    const long nbatch_all = (count + WB - 1) / WB;
+    const long nb = nbatch_all > g ? (nbatch_all - g + G - 1) / G : 0;   // batches of this warp: g, g + G, ...
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto issue = [&](long k) {
+        if (k < nb) {
+            const long i = (g + k * G) * WB;
+            int r[WB];
+#pragma unroll
+            for (int u = 0; u < WB; ++u) r[u] = (i + u < count) ? __ldg(idx + i + u) : -1;
+#pragma unroll
+            for (int u = 0; u < WB; ++u) {
+                if (r[u] < 0) continue;
+                const uint32_t dst = ring_s + (uint32_t)(((k % NB) * WB + u) * 512);
+                const char *src = base + (uint64_t)(uint32_t)r[u] * 512u;
+                if constexpr (CG) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+                else asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");   // one group per call, also when empty: uniform counting
+    };
+    for (long k = 0; k < NB; ++k) issue(k);
+    for (long k = 0; k < nb; ++k) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(NB - 1) : "memory");   // batch k has landed
+        const long i = (g + k * G) * WB;
+#pragma unroll
+        for (int u = 0; u < WB; ++u)
+            if (i + u < count) add4(acc, *reinterpret_cast<const float4 *>(ring + ((k % NB) * WB + u) * 512));
+        issue(k + NB);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    sink[(long)blockIdx.x * blockDim.x + threadIdx.x] = acc;
+}
+
 // ---- hub rows in distributed shared memory: a cluster of CL CTAs (one per SM) keeps CL * kHubRows hot rows; an
 // index with bit 31 set names hub slot (idx & 0x7fffffff), held by CTA slot / kHubRows of the cluster ------------
 constexpr int kHubRows = 256;   // 128 KB of 512-byte rows per CTA
@@ -289,6 +336,7 @@ extern "C" {
 // Paths: 0 plain loads, 4 in flight per lane (any row size 16..512 bytes); the others take 512-byte rows only:
 //   1 plain x8   2 plain x16   3 L2 evict-last x4   4 L1 no-allocate x4   5 tile order, staged indices, evict-last
 //   6 half warp per row, two vectors per lane   7 bulk-copy ring   8 / 9 / 10 hub rows in a cluster of 4 / 8 / 16 CTAs
+//   11 / 12 cp.async ring, 16 rows in flight per warp, bypassing / through L1   13 the same with 32 rows (L1 bypassed)
 // Floats the sink must hold for any path.
 long gp_sink_floats(void) { return (long)sm_count() * 8 * 1024 * 4; }
 
@@ -370,6 +418,19 @@ int gp_gather(int path, const int *idx, long count, const void *table_, int row_
         if (e != cudaSuccess) return (int)e;
         break;
     }
+#define GP_ASYNC(D, CGF)                                                                           \
+    {                                                                                              \
+        auto k = async_ring_kernel<D, 4, CGF>;                                                     \
+        const size_t sm = (size_t)8 * D * 512;                                                     \
+        cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);             \
+        const int o = resident(k, 256, sm);                                                        \
+        if (info) *info = o;                                                                       \
+        k<<<sm_count() * o, 256, sm, st>>>(idx, count, table, sink);                               \
+    }
+    case 11: GP_ASYNC(16, true) break;
+    case 12: GP_ASYNC(16, false) break;
+    case 13: GP_ASYNC(32, true) break;
+#undef GP_ASYNC
     default: return -1;
     }
 #undef GP_STRIDE

@@ -35,7 +35,7 @@ def test_plain_path_sums_any_row_size(row_bytes, count):
     assert np.array_equal(got, table[idx].astype(np.float64).sum(axis=0))
 
 
-@pytest.mark.parametrize("path", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13])
 @pytest.mark.parametrize("count", [5, 70_003])
 def test_every_512_byte_path_fetches_every_row(path, count):
     bp = _probes()
