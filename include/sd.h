@@ -67,8 +67,9 @@ typedef enum {
                         several rows per lane group, longest first; every heavy row is cut, column window by
                         column window, into chunks of at most 128 nonzeros of the caller's own CSR arrays
                         (no re-bucketed copy of A), the chunks are summed window-major into scratch rows
-                        and one warp (or CTA) per heavy row adds its scratch rows in order.  Five launches
-                        at most, plan memory of a few bytes per row.  Needs ascending columns.  AUTO takes
+                        and one warp (or CTA) per heavy row adds its scratch rows in order.  Three launches
+                        at most (one kernel for all rows, then the chunk sums), on the caller's stream only;
+                        plan memory of a few tens of bytes per row.  Needs ascending columns.  AUTO takes
                         it in place of SD_MERGE (measured rule): without column windows from 5 columns up to
                         rows of B of 384 bytes, with column windows where a row of B is 64 to 192 bytes */
 } sd_family_t;
@@ -153,7 +154,7 @@ sd_status_t sd_plan_create_ex(const sd_plan_desc_t *desc, sd_plan_t **out);
  * 16-byte aligned B/C with N, ldb, ldc multiples of the vector width take the
  * vectorised kernels; anything else takes scalar kernels (never an error).
  * With column windows the call issues one kernel sequence per window, in order, and C is
- * updated window by window.  Window-major and hybrid plans run part of their kernels on plan-owned
+ * updated window by window.  Window-major plans run part of their kernels on plan-owned
  * streams that are forked from `stream` and joined back into it before the call returns, so that
  * everything is ordered after what `stream` held before the call and before what is queued on it
  * afterwards (a stream capture of `stream` therefore takes the whole call into its graph).  A plan

@@ -565,7 +565,9 @@ int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const i
 
 /* Hybrid family in place of the merge family's own schedules (this build's rule, parity unpinned;
  * measured on the target GPU).  Needs ascending columns.  Without column windows: from 5 columns up
- * to rows of B of 384 bytes (96 fp32 / 192 bf16 columns): up to 256 bytes it takes 0.80 to 0.94 of the
+ * to rows of B of 384 bytes (96 fp32 / 192 bf16 columns) when the call gathers at least 256 MiB
+ * (nnz times the bytes of a row of B; smaller calls keep the merge family, whose three or four launches
+ * weigh less): up to 256 bytes it takes 0.80 to 0.94 of the
  * better of merge-path tiles and class split on the R-MAT matrix and is level with the class split on
  * the rank-size matrix; at 384 bytes 0.90 (fp32) and 1.02 (bf16) of the tiles' time; at 512 bytes the
  * tiles are ahead.  With column windows (sdo_decide_windows > 1): where one row of B is 64 to 192
@@ -580,7 +582,7 @@ int sdo_decide_hybrid(const sdo_info_t *o, int dtype, int windows)
         return 0;
     if (windows > 1)
         return row_bytes >= 64 && row_bytes <= 192;
-    return o->N >= 5 && row_bytes <= 384;
+    return o->N >= 5 && row_bytes <= 384 && o->nnz * row_bytes >= ((int64_t)1 << 28);
 }
 
 /* The family a plan is built with: sdo_decide, then the hybrid family in place of the merge family

@@ -579,7 +579,10 @@ static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
 
 // The hybrid family in place of the merge family's own schedules, for matrices with ascending columns (measured,
 // `bench.py --regret`):
-//   without column windows: from 5 columns up to rows of B of 384 bytes (96 fp32 / 192 bf16 columns).  On the R-MAT
+//   without column windows: from 5 columns up to rows of B of 384 bytes (96 fp32 / 192 bf16 columns), when the call
+//     gathers at least 256 MiB (nnz x bytes of a row of B): below that its five launches and two stream joins weigh
+//     too much (R-MAT scale 18 at 8 columns, 126 / 252 MB gathered: 1.27 / 1.04 to 1.13 of the tiles' time; at 32 fp32
+//     columns, 1 GB: 0.78 of the class split's).  On the R-MAT
 //     matrix it takes 0.80 to 0.94 of the better of merge-path tiles and class split at every width up to 256 bytes
 //     (fp32 5 to 64 columns, bf16 5 to 128) and is level with the class split on the rank-size matrix; at 384 bytes
 //     0.90 of the tiles' time with fp32 values and 1.02 with bf16 values; at 512-byte rows the tiles are ahead
@@ -593,7 +596,7 @@ static bool decide_hybrid(const sd_plan_info_t &s, int dtype, int windows) {
     const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
     if (s.unsorted_rows != 0) return false;
     if (windows > 1) return row_bytes >= 64 && row_bytes <= 192;
-    return s.N > kCooMaxN && row_bytes <= 384;
+    return s.N > kCooMaxN && row_bytes <= 384 && s.nnz * row_bytes >= (int64_t{1} << 28);
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {
@@ -772,7 +775,7 @@ static sd_status_t build_windows(sd_plan *p, int W, std::vector<int64_t> &bounds
     return SD_OK;
 }
 
-static sd_status_t create_split_streams(sd_plan *p, int W, bool chunks_first = false);
+static sd_status_t create_split_streams(sd_plan *p, int W);
 
 // `split`: the segments are re-bucketed by (window, class) and run through the chunk / segment / single
 // kernels; always so with W > 1, and with W = 1 when the class split alone pays (decide_class_split).
@@ -1039,7 +1042,6 @@ static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
     SD_CUDA_TRY(cudaStreamSynchronize(st));
     p->h_nl = nl;
     p->h_nc = 0;
-    if ((s = create_split_streams(p, 1, true))) return s;
     p->info.windows = W;
     p->info.launches = 1;
     if (nl > 0) {
@@ -1098,7 +1100,7 @@ static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
             SD_CUDA_TRY(cudaMemcpyAsync(p->h_giant, sel.p, sizeof(int32_t) * ng, cudaMemcpyDeviceToDevice, st));
             SD_CUDA_TRY(cudaStreamSynchronize(st));
         }
-        p->info.launches = (nl < p->M ? 1 : 0) + 2 + (ng > 0 ? 1 : 0);
+        p->info.launches = 2 + (ng > 0 ? 1 : 0);   // the fused kernel, the chunk sums, the chunk sums of very long rows
     }
     if (nl < p->M) {   // the light rows, longest first
         TempBuf key, key_out, id, id_out, tmp3;
@@ -1132,7 +1134,6 @@ static sd_status_t build_hybrid(sd_plan *p, int W, int32_t T, cudaStream_t st) {
         }
         SD_CUDA_TRY(cudaStreamSynchronize(st));
         p->h_nm = upto - nl;
-        p->info.launches += (p->h_nm > 0 ? 1 : 0) - (p->h_nm == p->M - nl ? 1 : 0);   // medium rows add a launch; no shorter rows: one less
         if ((s = build_light_desc(p, st))) return s;
     }
     p->num_chunks = p->h_nc;
@@ -1495,22 +1496,14 @@ static void blob_arrays(sd_plan *p, BlobArray (&arr)[kBlobArrays]) {
     set(18, &p->h_light, (hyb && p->h_nl < p->M) ? 4 * (p->M - p->h_nl) : 0, "light rows");
 }
 
-// chunks_first: the chunk stream gets the highest priority, so that when its persistent kernel and the kernels of the
-// side streams become runnable at the same moment (calls queued back to back) the chunk kernel's CTAs are placed first.
-static sd_status_t create_split_streams(sd_plan *p, int W, bool chunks_first) {
-    SD_CUDA_TRY(preload_stream_kernels(p->dtype, static_cast<int32_t>(p->N), chunks_first));   // before the streams exist
+static sd_status_t create_split_streams(sd_plan *p, int W) {
+    SD_CUDA_TRY(preload_stream_kernels(p->dtype, static_cast<int32_t>(p->N)));   // before the streams exist
     for (int i = 0; i < 2; ++i) {
         SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->aux[i], cudaStreamNonBlocking));
         SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_join[i], cudaEventDisableTiming));
     }
     SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
-    if (chunks_first) {
-        int least = 0, greatest = 0;
-        SD_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
-        SD_CUDA_TRY(cudaStreamCreateWithPriority(&p->chunk_stream, cudaStreamNonBlocking, greatest));
-    } else {
-        SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
-    }
+    SD_CUDA_TRY(cudaStreamCreateWithFlags(&p->chunk_stream, cudaStreamNonBlocking));
     p->ev_chunk.assign(W, nullptr);
     for (int w = 0; w < W; ++w) SD_CUDA_TRY(cudaEventCreateWithFlags(&p->ev_chunk[w], cudaEventDisableTiming));
     return SD_OK;
@@ -1968,63 +1961,26 @@ sd_status_t sd_spmm(const sd_plan_t *plan, const void *B, int64_t ldb, float *C,
         return SD_OK;
     }
     case SD_HYBRID: {
-        const bool has_light = plan->h_nl < M, side = has_light && plan->h_nl > 0 && plan->aux[0] && !switches().no_side_streams;
-        cudaStream_t s_light = st, s_heavy = st;
-        if (side) {   // light rows and heavy rows write disjoint rows of C: side by side
-            s_light = plan->aux[0];
-            SD_CUDA_TRY(cudaEventRecord(plan->ev_fork, st));
-            SD_CUDA_TRY(cudaStreamWaitEvent(s_light, plan->ev_fork, 0));
-            if (plan->chunk_stream && !switches().no_chunk_ahead) {   // the chunk kernel on the high-priority stream
-                s_heavy = plan->chunk_stream;
-                SD_CUDA_TRY(cudaStreamWaitEvent(s_heavy, plan->ev_fork, 0));
-            }
-        }
-        if (plan->h_nl > 0) {
-            SpmmArgs ca = a;
-            ca.ranges = plan->h_ranges;
-            ca.order = plan->h_order;
-            ca.S = plan->h_nc;
-            ca.C = plan->chunk_out;
-            ca.ldc = N;
-            ca.alpha = 1.f;
-            ca.beta = 0.f;
-            SD_CUDA_TRY(run_segments(ca, plan->dtype, vec, true, s_heavy));
-        }
-        cudaStream_t s_medium = st;
-        if (plan->h_nm > 0) {   // light rows of medium length: one lane group per row
-            if (side && plan->aux[1]) {
-                s_medium = plan->aux[1];
-                SD_CUDA_TRY(cudaStreamWaitEvent(s_medium, plan->ev_fork, 0));
-            }
-            SpmmArgs ma = a;
-            ma.desc = plan->h_desc;
-            ma.S = plan->h_nm;
-            SD_CUDA_TRY(run_medium_rows(ma, plan->dtype, vec, s_medium));
-        }
-        if (M - plan->h_nl > plan->h_nm) {   // the short ones: several rows per lane group
-            SpmmArgs la = a;
-            la.desc = plan->h_desc + plan->h_nm;
-            la.S = M - plan->h_nl - plan->h_nm;
-            SD_CUDA_TRY(run_light_rows(la, plan->dtype, vec, s_light));
-        }
+        // one launch for the chunks of the heavy rows, the rows of medium length and the short rows; then the chunk sums
+        SpmmArgs ca = a, ma = a, la = a;
+        ca.ranges = plan->h_ranges;
+        ca.order = plan->h_order;
+        ca.S = plan->h_nc;
+        ca.C = plan->chunk_out;
+        ca.ldc = N;
+        ca.alpha = 1.f;
+        ca.beta = 0.f;
+        ma.desc = plan->h_desc;
+        ma.S = plan->h_nm;
+        la.desc = plan->h_desc + plan->h_nm;
+        la.S = M - plan->h_nl - plan->h_nm;
+        SD_CUDA_TRY(run_hybrid_fused(ca, ma, la, plan->dtype, vec, st));
         if (plan->h_nl > 0) {
             SD_CUDA_TRY(run_chunk_reduce(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, 0, plan->h_nl, C, ldc,
-                                         static_cast<int32_t>(N), alpha, beta, s_heavy, plan->h_ng > 0 ? kGiantChunks : 0));
+                                         static_cast<int32_t>(N), alpha, beta, st, plan->h_ng > 0 ? kGiantChunks : 0));
             if (plan->h_ng > 0)
-                SD_CUDA_TRY(run_chunk_reduce_wide(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, plan->h_giant, plan->h_ng,
-                                                  C, ldc, static_cast<int32_t>(N), alpha, beta, s_heavy));
-        }
-        if (s_heavy != st) {
-            SD_CUDA_TRY(cudaEventRecord(plan->ev_chunk[0], s_heavy));
-            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_chunk[0], 0));
-        }
-        if (s_light != st) {
-            SD_CUDA_TRY(cudaEventRecord(plan->ev_join[0], s_light));
-            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[0], 0));
-        }
-        if (s_medium != st) {
-            SD_CUDA_TRY(cudaEventRecord(plan->ev_join[1], s_medium));
-            SD_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_join[1], 0));
+                SD_CUDA_TRY(run_chunk_reduce_wide(plan->chunk_out, plan->h_chunk_ptr, plan->h_rows, plan->h_giant,
+                                                  plan->h_ng, C, ldc, static_cast<int32_t>(N), alpha, beta, st));
         }
         return SD_OK;
     }
@@ -2345,7 +2301,6 @@ sd_status_t sd_plan_load(const void *blob, size_t bytes, const int32_t *rowptr, 
             (s = dev_alloc(p, reinterpret_cast<void **>(&p->chunk_out), sizeof(float) * p->h_nc * p->N, "chunk sums")))
             return fail(s);
         if ((s = build_light_desc(p, nullptr))) return fail(s);
-        if ((s = create_split_streams(p, 1, true))) return fail(s);
     } else if (p->info.family == SD_BSR_TC) {
         if ((s = dev_alloc(p, &p->bval, es * 256 * p->nnzb, "bval"))) return fail(s);
         if ((s = dev_alloc(p, &p->bval_mma, (p->dtype == SD_BF16 ? 512 : 2048) * static_cast<size_t>(p->nnzb), "bval (tensor-core image)"))) return fail(s);

@@ -166,7 +166,7 @@ struct SpmmArgs {
 struct Switches {
     bool no_coo;           // SD_NO_COO: generic merge kernel at one to four columns
     bool no_side_streams;  // SD_NO_SIDE_STREAMS: the classes of a window on one stream
-    bool no_chunk_ahead;   // SD_NO_CHUNK_AHEAD: chunk kernels in window order; hybrid family: chunk kernel on the caller's stream
+    bool no_chunk_ahead;   // SD_NO_CHUNK_AHEAD: chunk kernels in window order
     bool bsr_simt;         // SD_BSR_SIMT: SIMT block kernel instead of the tensor-core one
     bool no_narrow;        // SD_NO_NARROW: wide row-split kernel at one to four columns
     int geom_nv;           // SD_GEOM_NV: 1 forces one vector per lane

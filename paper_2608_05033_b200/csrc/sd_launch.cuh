@@ -22,8 +22,7 @@ struct MergeArgs {
 
 // Family (a).  `vec`: B, C, ldb, ldc and N allow 16-byte accesses.
 cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
-cudaError_t run_medium_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
-cudaError_t run_light_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st);
+cudaError_t run_hybrid_fused(const SpmmArgs &ca, const SpmmArgs &ma, const SpmmArgs &la, int dtype, bool vec, cudaStream_t st);
 
 // One lane group per segment (a.seg_row: output rows), or per chunk of a long segment
 // (`scratch`: chunk c writes its plain sum to row c of a.C).
@@ -43,7 +42,7 @@ cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chu
                                   float beta, cudaStream_t st);
 
 // C = beta * C.
-cudaError_t preload_stream_kernels(int dtype, int32_t N, bool hybrid);
+cudaError_t preload_stream_kernels(int dtype, int32_t N);
 cudaError_t run_scale_c(float *C, int64_t ldc, int64_t M, int32_t N, float beta, cudaStream_t st);
 
 // Family (b): tile kernel, then the carry-out fix-up for the listed tiles (short chains one per

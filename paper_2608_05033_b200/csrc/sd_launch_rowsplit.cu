@@ -25,21 +25,15 @@ cudaError_t run_rowsplit(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st
     return launch_rowsplit<__nv_bfloat16>(a, vec, st);
 }
 
-// Hybrid family, short rows: a.desc holds their descriptors (longest rows first).
-cudaError_t run_light_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
-    if (dtype == SD_F32) return launch_light<float>(a, vec, st);
-    return launch_light<__nv_bfloat16>(a, vec, st);
+// Hybrid family in one launch: chunks of the heavy rows (ca), rows of medium length (ma), short rows (la).
+cudaError_t run_hybrid_fused(const SpmmArgs &ca, const SpmmArgs &ma, const SpmmArgs &la, int dtype, bool vec, cudaStream_t st) {
+    if (dtype == SD_F32) return launch_hybrid<float>(ca, ma, la, vec, st);
+    return launch_hybrid<__nv_bfloat16>(ca, ma, la, vec, st);
 }
 
 cudaError_t run_segments(const SpmmArgs &a, int dtype, bool vec, bool scratch, cudaStream_t st) {
     if (dtype == SD_F32) return launch_seg<float>(a, vec, scratch ? 1 : 0, st);
     return launch_seg<__nv_bfloat16>(a, vec, scratch ? 1 : 0, st);
-}
-
-// Hybrid family, rows of medium length: a.desc holds their descriptors.
-cudaError_t run_medium_rows(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
-    if (dtype == SD_F32) return launch_seg<float>(a, vec, 2, st);
-    return launch_seg<__nv_bfloat16>(a, vec, 2, st);
 }
 
 cudaError_t run_single(const SpmmArgs &a, int dtype, bool vec, cudaStream_t st) {
@@ -76,9 +70,9 @@ cudaError_t run_chunk_reduce_wide(const float *chunk_out, const int32_t *seg_chu
 // (both the 16-byte-vector and the scalar forms: which one runs depends on the operands' alignment at call time).
 // With lazy module loading a kernel is otherwise loaded at its first launch; when that happens in the middle of a
 // call that has just forked the plan's side streams, that plan's calls queued back to back stay 25 % slower for its
-// whole life (measured: 0.311 against 0.246 ms at 8 columns on the R-MAT matrix; loading eagerly or at plan creation
-// removes it).
-cudaError_t preload_stream_kernels(int dtype, int32_t N, bool hybrid) {
+// whole life (measured on an earlier multi-stream form of the hybrid family: 0.311 against 0.246 ms at 8 columns on
+// the R-MAT matrix; loading eagerly or at plan creation removes it).
+cudaError_t preload_stream_kernels(int dtype, int32_t N) {
     SpmmArgs a{};
     a.N = N;
     a.load_only = true;
@@ -87,15 +81,13 @@ cudaError_t preload_stream_kernels(int dtype, int32_t N, bool hybrid) {
         const bool vec = v == 1;
         if (vec && N % vw != 0) continue;
         cudaError_t e = run_segments(a, dtype, vec, true, nullptr);
-        if (e == cudaSuccess) e = hybrid ? run_medium_rows(a, dtype, vec, nullptr) : run_segments(a, dtype, vec, false, nullptr);
-        if (e == cudaSuccess) e = hybrid ? run_light_rows(a, dtype, vec, nullptr) : run_single(a, dtype, vec, nullptr);
+        if (e == cudaSuccess) e = run_segments(a, dtype, vec, false, nullptr);
+        if (e == cudaSuccess) e = run_single(a, dtype, vec, nullptr);
         if (e != cudaSuccess) return e;
     }
     cudaFuncAttributes at;
     cudaError_t e = cudaFuncGetAttributes(&at, chunk_reduce_kernel<4>);
     if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_kernel<1>);
-    if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_wide_kernel<4>);
-    if (e == cudaSuccess) e = cudaFuncGetAttributes(&at, chunk_reduce_wide_kernel<1>);
     return e;
 }
 

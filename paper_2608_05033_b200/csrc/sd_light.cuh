@@ -11,16 +11,16 @@
 
 #include "sd_common.cuh"
 #include "sd_rowsplit.cuh"
+#include "sd_segment.cuh"
 
 namespace sd {
 
 constexpr int kLightThreads = 256;
 
 template <typename T, int VW, int LPR, int NV, int R>
-__global__ void __launch_bounds__(kLightThreads)
-light_rows_kernel(const SpmmArgs a) {
+__device__ __forceinline__ void light_rows_body(const SpmmArgs &a, const unsigned bx) {
     const int lg = threadIdx.x % LPR;
-    const int64_t g = (static_cast<int64_t>(blockIdx.x) * kLightThreads + threadIdx.x) / LPR;
+    const int64_t g = (static_cast<int64_t>(bx) * kLightThreads + threadIdx.x) / LPR;
     const int64_t r0 = g * R;
     if (r0 >= a.S) return;
     const int cbase = blockIdx.y * (LPR * NV * VW);
@@ -96,47 +96,71 @@ light_rows_kernel(const SpmmArgs a) {
     }
 }
 
+// The hybrid family in one launch: the first `gc` CTAs walk the chunks of the heavy rows (persistent, grid-stride), the
+// next `gm` the rows of medium length (likewise), the rest the short rows (a batch of rows per lane group each).  CTAs
+// are placed in index order, so the chunk CTAs take the SMs first and the others fill in as they retire: what side
+// streams and a high stream priority would give, without depending on how streams map to the GPU's hardware queues
+// (two of a plan's streams landing on the same queue serialised them: 0.20 against 0.15 ms per call for every third
+// and fourth plan instance of a process) and without an order race between the kernels of calls queued back to back.
+template <typename T, int VW, int LPR, int NV, int R>
+__global__ void __launch_bounds__(kSegThreads, 4)
+hybrid_fused_kernel(const SpmmArgs chunks, const SpmmArgs medium, const SpmmArgs light, const unsigned gc, const unsigned gm) {
+    static_assert(kSegThreads == kLightThreads, "one CTA size for all roles");
+    if (blockIdx.x < gc) seg_body<T, VW, LPR, NV, 1>(chunks, blockIdx.x, gc);
+    else if (blockIdx.x < gc + gm) seg_body<T, VW, LPR, NV, 2>(medium, blockIdx.x - gc, gm);
+    else light_rows_body<T, VW, LPR, NV, R>(light, blockIdx.x - gc - gm);
+}
+
 template <typename T, int VW, int LPR, int NV>
-cudaError_t launch_light_one(const SpmmArgs &a, cudaStream_t st) {
-    constexpr int R = (NV * VW >= 8) ? 2 : 4;
-    if (a.load_only) {
+cudaError_t launch_hybrid_one(const SpmmArgs &ca, const SpmmArgs &ma, const SpmmArgs &la, cudaStream_t st) {
+    // four rows per lane group at four CTAs per SM (64 registers, a few spilled words in the short-row role): measured
+    // against 2, 6 and 8 rows and against 3 and 5 CTAs per SM, 4 to 20 % ahead of each on four workloads
+    constexpr int R = 4;
+    auto kernel = hybrid_fused_kernel<T, VW, LPR, NV, R>;
+    if (ca.load_only) {
         cudaFuncAttributes at;
-        return cudaFuncGetAttributes(&at, light_rows_kernel<T, VW, LPR, NV, R>);
+        return cudaFuncGetAttributes(&at, kernel);
     }
-    const int64_t groups = (a.S + R - 1) / R;
-    const int per_cta = kLightThreads / LPR;
-    dim3 grid(static_cast<unsigned>((groups + per_cta - 1) / per_cta),
-              static_cast<unsigned>((a.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
-    light_rows_kernel<T, VW, LPR, NV, R><<<grid, kLightThreads, 0, st>>>(a);
+    static std::atomic<int> occ_cache[kMaxDevices];
+    const int64_t cap = static_cast<int64_t>(sm_count_cached()) * occupancy_cached(occ_cache, kernel, kSegThreads);
+    const int per_cta = kSegThreads / LPR;
+    const int64_t need_c = (ca.S + per_cta - 1) / per_cta, need_m = (ma.S + per_cta - 1) / per_cta;
+    const int64_t need_l = ((la.S + R - 1) / R + per_cta - 1) / per_cta;
+    const unsigned gc = static_cast<unsigned>(need_c < cap ? need_c : cap), gm = static_cast<unsigned>(need_m < cap ? need_m : cap);
+    const int64_t total = static_cast<int64_t>(gc) + gm + need_l;
+    if (total == 0) return cudaSuccess;
+    if (total > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    dim3 grid(static_cast<unsigned>(total), static_cast<unsigned>((ca.N + LPR * NV * VW - 1) / (LPR * NV * VW)));
+    kernel<<<grid, kSegThreads, 0, st>>>(ca, ma, la, gc, gm);
     return cudaGetLastError();
 }
 
 template <typename T>
-cudaError_t launch_light(const SpmmArgs &a, bool vec, cudaStream_t st) {
+cudaError_t launch_hybrid(const SpmmArgs &ca, const SpmmArgs &ma, const SpmmArgs &la, bool vec, cudaStream_t st) {
     constexpr int VWV = vec_width<T>::value;
-    const LaneGeom g = lane_geometry(a.N, vec, VWV, false);
+    const LaneGeom g = lane_geometry(ca.N, vec, VWV, false);
     if (vec && g.nv == 2) {
         switch (g.lpr) {
-        case 8: return launch_light_one<T, VWV, 8, 2>(a, st);
-        case 16: return launch_light_one<T, VWV, 16, 2>(a, st);
-        case 32: return launch_light_one<T, VWV, 32, 2>(a, st);
+        case 8: return launch_hybrid_one<T, VWV, 8, 2>(ca, ma, la, st);
+        case 16: return launch_hybrid_one<T, VWV, 16, 2>(ca, ma, la, st);
+        case 32: return launch_hybrid_one<T, VWV, 32, 2>(ca, ma, la, st);
         }
         return cudaErrorInvalidValue;
     }
-#define SD_LT_CASE(L)                                               \
-    case L:                                                         \
-        if (vec) return launch_light_one<T, VWV, L, 1>(a, st);      \
-        return (g.nv == 4) ? launch_light_one<T, 1, 32, 4>(a, st)   \
-                           : launch_light_one<T, 1, L, 1>(a, st);
+#define SD_HY_CASE(L)                                                        \
+    case L:                                                                  \
+        if (vec) return launch_hybrid_one<T, VWV, L, 1>(ca, ma, la, st);     \
+        return (g.nv == 4) ? launch_hybrid_one<T, 1, 32, 4>(ca, ma, la, st)  \
+                           : launch_hybrid_one<T, 1, L, 1>(ca, ma, la, st);
     switch (g.lpr) {
-        SD_LT_CASE(1)
-        SD_LT_CASE(2)
-        SD_LT_CASE(4)
-        SD_LT_CASE(8)
-        SD_LT_CASE(16)
-        SD_LT_CASE(32)
+        SD_HY_CASE(1)
+        SD_HY_CASE(2)
+        SD_HY_CASE(4)
+        SD_HY_CASE(8)
+        SD_HY_CASE(16)
+        SD_HY_CASE(32)
     }
-#undef SD_LT_CASE
+#undef SD_HY_CASE
     return cudaErrorInvalidValue;
 }
 

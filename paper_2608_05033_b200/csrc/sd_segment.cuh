@@ -20,9 +20,10 @@ constexpr int kSegThreads = 256;
 // MODE 2: the segments are whole rows of the caller's CSR arrays named by the descriptors a.desc (hybrid
 // family, rows of medium length); walked like chunks, written like segments.
 // Up to four lanes per row: six CTAs per SM (40 registers) measure 6 % faster; wider groups lose with that cap.
+// seg_body is the kernel's body for CTA number `bx` of `nbx` (a kernel of its own, or one role of the fused kernel
+// of the hybrid family).
 template <typename T, int VW, int LPR, int NV, int MODE>
-__global__ void __launch_bounds__(kSegThreads, (LPR <= 4 && NV * VW < 8) ? 6 : 1)
-seg_kernel(const SpmmArgs a) {
+__device__ __forceinline__ void seg_body(const SpmmArgs &a, const unsigned bx, const unsigned nbx) {
     constexpr bool SCRATCH = MODE == 1;   // output: scratch rows
     constexpr bool STREAM = MODE != 0;    // walk: whole steps untested, next step's pairs requested ahead
     const int lane = threadIdx.x & 31;
@@ -40,8 +41,8 @@ seg_kernel(const SpmmArgs a) {
     constexpr int QW = (NV * VW >= 8) ? 2 : (STREAM ? 8 : 4);
     constexpr int QU = LPR < QW ? LPR : QW;
 
-    const int64_t gstride = static_cast<int64_t>(gridDim.x) * (kSegThreads / LPR);
-    for (int64_t s = (static_cast<int64_t>(blockIdx.x) * kSegThreads + threadIdx.x) / LPR; s < a.S; s += gstride) {
+    const int64_t gstride = static_cast<int64_t>(nbx) * (kSegThreads / LPR);
+    for (int64_t s = (static_cast<int64_t>(bx) * kSegThreads + threadIdx.x) / LPR; s < a.S; s += gstride) {
         int p0, p1;
         int64_t out_row = s;   // SCRATCH: scratch row of this chunk
         if (SCRATCH && a.ranges) {
@@ -187,6 +188,12 @@ seg_kernel(const SpmmArgs a) {
                 if (colok[v]) store_cols<VW>(crow + (v * LPR + lg) * VW, acc[v], a.alpha, a.beta, r < 0 ? 1 : 0);
         }
     }
+}
+
+template <typename T, int VW, int LPR, int NV, int MODE>
+__global__ void __launch_bounds__(kSegThreads, (LPR <= 4 && NV * VW < 8) ? 6 : 1)
+seg_kernel(const SpmmArgs a) {
+    seg_body<T, VW, LPR, NV, MODE>(a, blockIdx.x, gridDim.x);
 }
 
 constexpr int kSingleBatch = 4;   // segments per lane group: their loads are all in flight together

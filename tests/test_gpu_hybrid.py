@@ -58,9 +58,7 @@ def test_schedule_is_the_sequential_definition(kind, M, K, windows):
     assert np.array_equal(ranges, rr) and np.array_equal(order, ro) and np.array_equal(light, rl)
     assert (info.num_tiles, info.num_segments) == (rh.size, rr.shape[0])
     giants = int(np.sum(np.diff(rc) > 64)) if rh.size else 0
-    lens = np.diff(w.rowptr)[rl]
-    medium, short = int(np.sum(lens >= 16)), int(np.sum(lens < 16))   # one lane group per row / several rows per group
-    assert info.launches == (1 if medium else 0) + (1 if short else 0) + (2 if rh.size else 0) + (1 if giants else 0)
+    assert info.launches == 1 + (1 if rh.size else 0) + (1 if giants else 0)   # fused kernel, chunk sums, those of very long rows
     got, intact = run_spmm(plan, w)
     assert intact
     check(w, got)
@@ -162,7 +160,7 @@ def test_auto_takes_the_hybrid_family_where_the_rule_says_so():
         assert windows > 1 and info.windows == windows
         assert info.family == oracle.decide_family(ref, dtype, info.l2_bytes) == want
         if want == sd.SD_HYBRID:
-            assert info.heavy_len == 256 and info.launches <= 5
+            assert info.heavy_len == 256 and info.launches <= 3
             got = sd.sd_plan_get_hybrid(plan.handle)
             ref_s = oracle.hybrid_schedule(w.rowptr, w.colind, M, K, windows, 256)
             assert all(np.array_equal(a, b) for a, b in zip(got, ref_s))
@@ -172,9 +170,10 @@ def test_auto_takes_the_hybrid_family_where_the_rule_says_so():
 
 
 @pytest.mark.parametrize("family,windows", [(4, 4), (2, 4)], ids=["hybrid", "windowed_class_split"])
-def test_calls_of_multi_stream_plans_can_be_captured_into_a_cuda_graph(family, windows):
-    """The plan-owned side streams are forked from and joined back into the caller's stream with events, so a stream
-    capture takes them in: two calls captured (the second adds to the first's result), replayed, checked."""
+def test_calls_can_be_captured_into_a_cuda_graph(family, windows):
+    """The hybrid family launches on the caller's stream only; the windowed class split forks plan-owned side streams
+    from it and joins them back with events, so a stream capture takes them in: two calls captured (the second adds to
+    the first's result), replayed, checked."""
     rng = np.random.default_rng(3)
     M, K, N = 3000, 5000, 32
     w = W.random_csr(M, K, N, lengths_of("skewed", M, K, rng), seed=5)
