@@ -71,7 +71,8 @@ typedef enum {
                         at most (one kernel for all rows, then the chunk sums), on the caller's stream only;
                         plan memory of a few tens of bytes per row.  Needs ascending columns.  AUTO takes
                         it in place of SD_MERGE (measured rule): without column windows from 5 columns up to
-                        rows of B of 384 bytes, with column windows where a row of B is 64 to 192 bytes */
+                        rows of B of 384 bytes (fp32 values) or 256 bytes (bf16 values) when the call gathers
+                        at least 256 MiB, with column windows where a row of B is 64 to 192 (128) bytes */
 } sd_family_t;
 
 /* Options of sd_plan_create_ex.  Zero-initialise, then set fields. */

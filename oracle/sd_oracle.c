@@ -565,24 +565,24 @@ int64_t sdo_window_segments(int64_t M, int64_t K, const int32_t *rowptr, const i
 
 /* Hybrid family in place of the merge family's own schedules (this build's rule, parity unpinned;
  * measured on the target GPU).  Needs ascending columns.  Without column windows: from 5 columns up
- * to rows of B of 384 bytes (96 fp32 / 192 bf16 columns) when the call gathers at least 256 MiB
- * (nnz times the bytes of a row of B; smaller calls keep the merge family, whose three or four launches
- * weigh less): up to 256 bytes it takes 0.80 to 0.94 of the
- * better of merge-path tiles and class split on the R-MAT matrix and is level with the class split on
- * the rank-size matrix; at 384 bytes 0.90 (fp32) and 1.02 (bf16) of the tiles' time; at 512 bytes the
- * tiles are ahead.  With column windows (sdo_decide_windows > 1): where one row of B is 64 to 192
- * bytes (16 to 48 fp32 columns, 32 to 96 bf16 columns): 0.90 to 0.93 of the windowed class split's
- * time on the rank-size matrix at 96 and 128 bytes, level with it at 64 and 192 bytes with a fraction
- * of its launches and plan memory; behind it at 32 bytes (1.28) and from 256 bytes on (1.01 to 1.05:
- * the light rows then gather wide rows of B from DRAM, which the windowed schedule finds in L2). */
+ * to rows of B of 384 bytes with fp32 values (96 columns) or 256 bytes with bf16 values (128 columns),
+ * when the call gathers at least 256 MiB (nnz times the bytes of a row of B; smaller calls keep the
+ * merge family, whose launches weigh less): 0.70 to 0.90 of the better of merge-path tiles and class
+ * split on the R-MAT matrix; the tiles are ahead at 128 fp32 and 192 bf16 columns.  With column
+ * windows (sdo_decide_windows > 1): where one row of B is 64 to 192 bytes with fp32 values (16 to 48
+ * columns) or 64 to 128 bytes with bf16 values (32 to 64 columns): 0.84 to 0.93 of the windowed class
+ * split's time on the rank-size matrix at 96 and 128 bytes, level with it at the ends of the band
+ * with a fraction of its launches and plan memory; behind it at wider rows (the light rows then
+ * gather wide rows of B from DRAM, which the windowed schedule finds in L2). */
 int sdo_decide_hybrid(const sdo_info_t *o, int dtype, int windows)
 {
-    int64_t row_bytes = o->N * (dtype == SDO_F32 ? 4 : 2);
+    int f32 = dtype == SDO_F32;
+    int64_t row_bytes = o->N * (f32 ? 4 : 2);
     if (o->unsorted_rows != 0)
         return 0;
     if (windows > 1)
-        return row_bytes >= 64 && row_bytes <= 192;
-    return o->N >= 5 && row_bytes <= 384 && o->nnz * row_bytes >= ((int64_t)1 << 28);
+        return row_bytes >= 64 && row_bytes <= (f32 ? 192 : 128);
+    return o->N >= 5 && row_bytes <= (f32 ? 384 : 256) && o->nnz * row_bytes >= ((int64_t)1 << 28);
 }
 
 /* The family a plan is built with: sdo_decide, then the hybrid family in place of the merge family

@@ -578,25 +578,24 @@ static bool decide_class_split(const sd_plan_info_t &s, int dtype) {
 }
 
 // The hybrid family in place of the merge family's own schedules, for matrices with ascending columns (measured,
-// `bench.py --regret`):
-//   without column windows: from 5 columns up to rows of B of 384 bytes (96 fp32 / 192 bf16 columns), when the call
-//     gathers at least 256 MiB (nnz x bytes of a row of B): below that its five launches and two stream joins weigh
-//     too much (R-MAT scale 18 at 8 columns, 126 / 252 MB gathered: 1.27 / 1.04 to 1.13 of the tiles' time; at 32 fp32
-//     columns, 1 GB: 0.78 of the class split's).  On the R-MAT
-//     matrix it takes 0.80 to 0.94 of the better of merge-path tiles and class split at every width up to 256 bytes
-//     (fp32 5 to 64 columns, bf16 5 to 128) and is level with the class split on the rank-size matrix; at 384 bytes
-//     0.90 of the tiles' time with fp32 values and 1.02 with bf16 values; at 512-byte rows the tiles are ahead
-//     (1.12 against 1.19 ms).
-//   with column windows: where one row of B is 64 to 192 bytes (16 to 48 fp32 columns, 32 to 96 bf16 columns): on the
-//     rank-size matrix 0.90 to 0.93 of the windowed class split's time at 96 and 128 bytes and level with it (0.99 to
-//     1.005) at 64 and 192 bytes, with 5 launches instead of 16 to 64 and a quarter of the plan memory; behind it at
-//     32 bytes (1.28) and from 256 bytes on (1.01 to 1.05), where the light rows gather wide rows of B from DRAM that
-//     the windowed schedule finds in L2.
+// `bench.py --regret`; fp32 values allow wider rows than bf16 values, whose lanes hold eight accumulators per row):
+//   without column windows: from 5 columns up to rows of B of 384 bytes with fp32 values (96 columns) and 256 bytes with
+//     bf16 values (128 columns), when the call gathers at least 256 MiB (nnz x bytes of a row of B): below that its
+//     launches weigh too much (R-MAT scale 18 at 8 columns, 126 / 252 MB gathered: 1.27 / 1.04 to 1.13 of the tiles'
+//     time).  On the R-MAT matrix it takes 0.70 to 0.90 of the better of merge-path tiles and class split up to 256-byte
+//     rows (bf16 at 256 bytes: level), 0.87 of the tiles' time at 96 fp32 columns, and is behind them at 128 fp32
+//     columns (1.06) and 192 bf16 columns (1.16).
+//   with column windows: where one row of B is 64 to 192 bytes with fp32 values (16 to 48 columns) and 64 to 128 bytes
+//     with bf16 values (32 to 64 columns): on the rank-size matrix 0.84 to 0.93 of the windowed class split's time at 96
+//     and 128 bytes and level with it (0.99 to 1.01) at the ends of the band, with 3 launches instead of 16 to 64 and a
+//     quarter of the plan memory; behind it at 64 fp32 columns (1.07) and 96 or 128 bf16 columns (1.2), where the light
+//     rows gather wide rows of B from DRAM that the windowed schedule finds in L2.
 static bool decide_hybrid(const sd_plan_info_t &s, int dtype, int windows) {
-    const int64_t row_bytes = s.N * (dtype == SD_F32 ? 4 : 2);
+    const bool f32 = dtype == SD_F32;
+    const int64_t row_bytes = s.N * (f32 ? 4 : 2);
     if (s.unsorted_rows != 0) return false;
-    if (windows > 1) return row_bytes >= 64 && row_bytes <= 192;
-    return s.N > kCooMaxN && row_bytes <= 384 && s.nnz * row_bytes >= (int64_t{1} << 28);
+    if (windows > 1) return row_bytes >= 64 && row_bytes <= (f32 ? 192 : 128);
+    return s.N > kCooMaxN && row_bytes <= (f32 ? 384 : 256) && s.nnz * row_bytes >= (int64_t{1} << 28);
 }
 
 __global__ void iota_kernel(int32_t *out, int64_t n) {

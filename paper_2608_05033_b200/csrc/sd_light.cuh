@@ -114,8 +114,9 @@ hybrid_fused_kernel(const SpmmArgs chunks, const SpmmArgs medium, const SpmmArgs
 template <typename T, int VW, int LPR, int NV>
 cudaError_t launch_hybrid_one(const SpmmArgs &ca, const SpmmArgs &ma, const SpmmArgs &la, cudaStream_t st) {
     // four rows per lane group at four CTAs per SM (64 registers, a few spilled words in the short-row role): measured
-    // against 2, 6 and 8 rows and against 3 and 5 CTAs per SM, 4 to 20 % ahead of each on four workloads
-    constexpr int R = 4;
+    // against 2, 6 and 8 rows and against 3 and 5 CTAs per SM, 4 to 20 % ahead of each on four workloads (fp32 values, one
+    // 16-byte vector per lane); lanes that hold eight accumulators per row take two rows
+    constexpr int R = (NV * VW >= 8) ? 2 : 4;
     auto kernel = hybrid_fused_kernel<T, VW, LPR, NV, R>;
     if (ca.load_only) {
         cudaFuncAttributes at;

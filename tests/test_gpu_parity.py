@@ -702,8 +702,8 @@ def test_merge_class_split_with_one_window(kind, N, dtype):
 
 
 def test_automatic_schedule_of_a_skewed_matrix_matches_the_rules():
-    """Without column windows: the hybrid family from 5 columns up to 384-byte rows of B when the call gathers at least
-    256 MiB, else the merge family (tiles; the COO reduction up to 4 columns).  A forced merge plan still takes its
+    """Without column windows: the hybrid family from 5 columns up to 384-byte (fp32 values) or 256-byte (bf16 values)
+    rows of B when the call gathers at least 256 MiB, else the merge family (tiles; the COO reduction up to 4 columns).  A forced merge plan still takes its
     class split by the width rule."""
     rng = np.random.default_rng(77)
     M, K = 20_000, 30_000
@@ -718,7 +718,7 @@ def test_automatic_schedule_of_a_skewed_matrix_matches_the_rules():
         assert oracle.decide(ref, dtype) == oracle.MERGE
         assert info.windows == oracle.decide_windows(ref, dtype, info.l2_bytes) == 1
         row_bytes = N * (4 if dtype == W.SD_F32 else 2)
-        hybrid = N >= 5 and row_bytes <= 384 and w.nnz * row_bytes >= 1 << 28
+        hybrid = N >= 5 and row_bytes <= (384 if dtype == W.SD_F32 else 256) and w.nnz * row_bytes >= 1 << 28
         assert info.family == oracle.decide_family(ref, dtype, info.l2_bytes) == (sd.SD_HYBRID if hybrid else sd.SD_MERGE), (N, dtype)
         got, _ = run_spmm(plan, w)
         check(w, got)

@@ -701,17 +701,18 @@ def test_o4_hybrid_schedule_against_python_sets():
 
 def test_o4_hybrid_rule():
     """Hybrid in place of the merge family's schedules: ascending columns; with column windows rows of B of 64 to
-    192 bytes, without them 5 columns and more up to 384-byte rows and at least 256 MiB gathered per call; the family
-    rule applies it on top of the merge decision."""
+    192 bytes (fp32 values) or 128 bytes (bf16 values), without them 5 columns and more up to 384-byte (256-byte) rows
+    and at least 256 MiB gathered per call; the family rule applies it on top of the merge decision."""
     info = oracle.Info()
     info.M, info.K, info.nnz, info.unsorted_rows = 1 << 20, 1 << 22, 5 << 20, 0
     for dtype, es in ((oracle.F32, 4), (oracle.BF16, 2)):
         for N in (1, 4, 5, 8, 16, 17, 24, 32, 33, 48, 64, 65, 96, 128, 129, 256):
             info.N = N
-            assert oracle.decide_hybrid(info, dtype, 8) == (64 <= N * es <= 192), (dtype, N)
+            assert oracle.decide_hybrid(info, dtype, 8) == (64 <= N * es <= (192 if es == 4 else 128)), (dtype, N)
             for nnz in (5 << 20, 40 << 20):      # without windows the call must also gather at least 256 MiB
                 info.nnz = nnz
-                assert oracle.decide_hybrid(info, dtype, 1) == (N >= 5 and N * es <= 384 and nnz * N * es >= 1 << 28), (dtype, N)
+                cap = 384 if es == 4 else 256
+                assert oracle.decide_hybrid(info, dtype, 1) == (N >= 5 and N * es <= cap and nnz * N * es >= 1 << 28), (dtype, N)
             info.nnz = 5 << 20
     info.N, info.nnz = 64, (1 << 20) - 1             # 256-byte rows: one nonzero short of 256 MiB
     assert not oracle.decide_hybrid(info, oracle.F32, 1)
