@@ -608,8 +608,9 @@ constexpr int kShortSegment = 32;   // segments up to this many nonzeros go to t
 constexpr int kHybridHeavy = 256;   // hybrid family: rows of at least this many nonzeros run as chunks: the long-row threshold
                                     // of the paper's appendix listing; measured on the rank-size matrix at 128-byte rows of
                                     // B, 64 / 128 / 192 / 256 give 1.054 / 0.987 / 0.956 / 0.950 ms
-constexpr int kHybridMedium = 16;   // light rows of at least this many nonzeros take one lane group each, a step of nonzeros
+constexpr int kHybridMedium = 4;    // light rows of at least this many nonzeros take one lane group each, a step of nonzeros
                                     // at a time; shorter ones run several rows per lane group, a nonzero at a time
+                                    // (2 / 3 / 4 / 8 / 16 / 32 measured on six workloads: 4 is best or level on five)
 constexpr int kHybridHeavyMax = 256;   // upper limit: a light row is one running sum
 
 // Re-buckets the nonzeros by column window and builds the (row, window) segment list, ordered by
